@@ -1,0 +1,163 @@
+/* zipml.h -- C ABI of the B200 (sm_100a) library for double-sampled low-precision SGD on linear
+ * models (ZipML, arxiv 1611.05402).
+ *
+ * Conventions
+ *   - C linkage, plain pointers and sizes.  Every function returns an int status: ZIPML_OK (0) or
+ *     a negative ZIPML_ERR_* value; zipml_strerror() names it.  No exceptions, no abort, no device
+ *     trap.
+ *   - Unless a parameter says HOST, data pointers are DEVICE pointers owned by the caller and must
+ *     stay valid until the work is complete.  The library allocates only its own workspace, inside
+ *     the context (it may grow on a call that needs more).
+ *   - Work is enqueued on the context's CUDA stream and the call returns without waiting.
+ *     Argument errors are reported by the call itself; errors found on the device (non-finite
+ *     input, a grid barrier that ran out of patience) are reported by zipml_sync().
+ *   - Matrices are row-major with 64-bit sizes and an explicit leading dimension in elements.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with
+ *     ZIPML_ERR_CUDA.
+ *
+ * Packed sample layout ("plane"): row-major, `row_bytes` bytes per row, row_bytes a multiple of 16
+ * and >= zipml_row_bytes(n, bits).  Feature j occupies cb bits at bit position j*cb of its row,
+ * low bits first, where the container width cb is 2, 4, 4, 8 for bits = 2, 3, 4, 8.  Padding bits
+ * are zero.  A double-sampled dataset is two such planes (two independent quantizations of every
+ * sample, Eq. (double) of the paper) plus what turns a code back into a value: per-feature
+ * (lo_j, step_j) for a uniform grid, value = lo_j + code * step_j, or an n x 2^bits table of
+ * ascending levels.
+ */
+#ifndef ZIPML_H_
+#define ZIPML_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    ZIPML_OK = 0,
+    ZIPML_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad stride or alignment        */
+    ZIPML_ERR_UNSUPPORTED = -2, /* bits not in {2,3,4,8}, a level table with 8 bits, ...            */
+    ZIPML_ERR_NONFINITE = -3,   /* the sample matrix holds a NaN or an infinity (seen on device)   */
+    ZIPML_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, out of memory, ...)       */
+    ZIPML_ERR_TIMEOUT = -5,     /* a device-side wait gave up; the context stays usable            */
+    ZIPML_ERR_WORKSPACE = -6    /* the problem does not fit the kernels' on-chip or scratch limits */
+};
+
+enum { ZIPML_LEVELS_UNIFORM = 0, ZIPML_LEVELS_TABLE = 1 };
+enum { ZIPML_LOSS_DENSE = 0, ZIPML_LOSS_CODES = 1 };
+/* How zipml_sgd_epoch runs its minibatch chain.  Results do not depend on the choice. */
+enum {
+    ZIPML_ENGINE_AUTO = 0,
+    ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
+    ZIPML_ENGINE_PERSISTENT = 2 /* one cooperative launch per call, grid barriers between the phases */
+};
+
+typedef struct zipml_ctx zipml_ctx;
+
+/* A double-sampled, bit-packed dataset in device memory. */
+typedef struct zipml_dataset {
+    uint32_t struct_size;   /* sizeof(zipml_dataset), for ABI evolution                              */
+    int32_t bits;           /* 2, 3, 4 or 8                                                          */
+    int32_t level_mode;     /* ZIPML_LEVELS_UNIFORM or ZIPML_LEVELS_TABLE                            */
+    int32_t reserved;
+    int64_t m, n;           /* samples, features                                                     */
+    int64_t row_bytes;      /* stride of both planes                                                 */
+    const uint8_t* plane1;  /* m * row_bytes bytes, 16-byte aligned                                  */
+    const uint8_t* plane2;
+    const float* feat_lo;   /* n; UNIFORM                                                            */
+    const float* feat_step; /* n; UNIFORM                                                            */
+    const float* levels;    /* n * 2^bits ascending; TABLE                                           */
+} zipml_dataset;
+
+/* Parameters of one zipml_sgd_epoch call. */
+typedef struct zipml_sgd_params {
+    uint32_t struct_size;       /* sizeof(zipml_sgd_params)                                          */
+    int32_t model_bits;         /* 0: gradients see the fp32 model; 2..8: see Q3(x), redrawn per step */
+    int32_t grad_bits;          /* 0: fp32 gradient; 2..8: the update uses Q4(g)                     */
+    int32_t engine;             /* ZIPML_ENGINE_*                                                    */
+    int64_t batch;              /* minibatch size B; batch t holds rows [t*B, min(m, (t+1)*B))       */
+    int64_t epoch;              /* keys the Q3/Q4 random draws together with the step index          */
+    int64_t first_step;         /* the call executes positions first_step .. first_step+num_steps-1  */
+    int64_t num_steps;          /* of the batch order; num_steps < 0 means "to the end"              */
+    uint64_t seed;              /* keys the Q3/Q4 random draws                                       */
+    const int32_t* batch_order; /* HOST pointer or NULL: T = ceil(m/B) batch indices; NULL = 0..T-1  */
+    float lr;                   /* step length gamma, constant within the call                       */
+    int32_t grid_feature_parts; /* tuning, 0 = automatic: CTAs along the features                    */
+    int32_t grid_row_parts;     /* tuning, 0 = automatic: CTAs along the rows of a minibatch         */
+    int32_t reserved;
+} zipml_sgd_params;
+
+/* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default
+ * stream) and a workspace.  One context must not be used from two threads at once. */
+int zipml_create(zipml_ctx** ctx_out, int device, void* cuda_stream);
+int zipml_destroy(zipml_ctx* ctx);
+/* Waits for the stream and returns the first device-side error since the previous zipml_sync
+ * (ZIPML_OK if none), clearing it. */
+int zipml_sync(zipml_ctx* ctx);
+const char* zipml_strerror(int status);
+/* Smallest legal row stride for n features: ceil(n*cb/8) rounded up to 16; 0 if bits is unsupported. */
+int64_t zipml_row_bytes(int64_t n, int32_t bits);
+
+/* Stochastic quantization with double sampling (paper Section 2.1, Eq. (double); Supplement
+ * "Randomized Quantization", "Column Scaling").
+ *   A          m x n fp32, leading dimension lda >= n.
+ *   bits       2, 3, 4 or 8: L = 2^bits levels, s = L-1 intervals.
+ *   level_mode UNIFORM: levels lo_j + i*(hi_j-lo_j)/s on the feature's own range [lo_j, hi_j]
+ *              (found by this call).  TABLE: `levels` (n x L ascending, levels[j][0] <= every value
+ *              of feature j <= levels[j][L-1], e.g. from zipml_optimal_levels); bits = 8 unsupported.
+ *   seed       each element (row k, feature j) is rounded twice, to the lower or upper neighbouring
+ *              level with the probabilities that make the expectation equal to the value, using
+ *              two 24-bit uniforms from Philox4x32-10 keyed by (seed, k, j, copy).
+ * Out: plane1, plane2 (m * row_bytes bytes each, fully written including zero padding),
+ *      feat_lo (n; the per-feature minimum), feat_step (n; UNIFORM only, may be NULL for TABLE).
+ * A NaN or infinity in A makes the next zipml_sync() return ZIPML_ERR_NONFINITE (outputs undefined). */
+int zipml_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
+                   int32_t level_mode, const float* levels, uint64_t seed, uint8_t* plane1,
+                   uint8_t* plane2, int64_t row_bytes, float* feat_lo, float* feat_step);
+
+/* Variance-optimal level placement (paper Section 3: the problem statement, the recursion
+ * T(k,m) = min_j T(k-1,j) + V(j,m), and "Dynamic Programming with Candidate Points").
+ * Per feature: normalise to [0,1] by its range, count the values in `hist_bins` equal bins (one
+ * pass over A), and choose the s-1 interior endpoints among the bin edges that minimise the total
+ * quantization variance of the bin centres; exact integer arithmetic, ties to the smaller edge.
+ *   bits 2, 3 or 4; s = 2^bits - 1 <= hist_bins <= 1024; m <= 10^9.
+ * Out: levels_out n x 2^bits fp32 ascending with first = lo_j and last = hi_j;
+ *      objective_out (n uint64, may be NULL): 4 * hist_bins^2 * (sum of variances), normalised units. */
+int zipml_optimal_levels(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda,
+                         int32_t bits, int32_t hist_bins, float* levels_out, uint64_t* objective_out);
+
+/* Mini-batch SGD over the stored double samples (Supplement "Double Sampling", the averaged form of
+ * its footnote; "End-to-end Quantization" for the optional model and gradient quantizers):
+ *   g = 1/(2 B_t) sum_{k in batch} [ Q1(a_k)(Q2(a_k)^T x~ - b_k) + Q2(a_k)(Q1(a_k)^T x~ - b_k) ],
+ *   x~ = Q3(x) or x,  g^ = Q4(g) or g,  x <- x - lr * g^   (update in fp32).
+ * Q3 and Q4 are l2-scaled sign-magnitude stochastic quantizers with 2^(bits-1)-1 magnitude levels,
+ * keyed by (seed, epoch, step position, coordinate).
+ *   b        m labels;  x  n, read and updated in place.
+ *   grad_out NULL or 2n floats: the last executed step's gradient before and after Q4.
+ * ZIPML_ERR_WORKSPACE if n is too large for the kernels' shared memory plan. */
+int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, float* x,
+                    const zipml_sgd_params* params, float* grad_out);
+
+/* Training loss (paper Eq. (leastsquares) with l = a^T x - b): 1/(2m) sum_k (a_k^T x - b_k)^2.
+ *   ZIPML_LOSS_DENSE  on the fp32 samples A (m x n, lda); `data` ignored.
+ *   ZIPML_LOSS_CODES  the unbiased estimate 1/(2m) sum (Q1(a_k)^T x - b_k)(Q2(a_k)^T x - b_k) from
+ *                     `data`; A, m, n, lda ignored (sizes come from `data`).
+ * Out: loss_out, one double in device memory.  Deterministic for a given device and shape. */
+int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t n, int64_t lda,
+               const zipml_dataset* data, const float* b, const float* x, double* loss_out);
+
+/* Whole path from HOST buffers, for callers that hold their data in host memory: copies A and b to
+ * the device, quantizes (UNIFORM, or TABLE with levels from zipml_optimal_levels when
+ * optimal_levels != 0), runs `epochs` epochs of zipml_sgd_epoch (epoch index e = 0..epochs-1, step
+ * length lr, or lr/(e+1) when lr_decay != 0: the paper's alpha/epoch schedule), evaluates the dense
+ * loss, copies x and the loss back and waits.  Everything in `params` except epoch, first_step and
+ * num_steps is honoured.
+ *   A_host m x n fp32 (lda), b_host m, x_host n in/out, loss_out_host one double: all HOST. */
+int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, int64_t lda,
+                     const float* b_host, float* x_host, int32_t bits, int32_t optimal_levels,
+                     int32_t hist_bins, uint64_t quantize_seed, const zipml_sgd_params* params,
+                     int32_t epochs, int32_t lr_decay, double* loss_out_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIPML_H_ */

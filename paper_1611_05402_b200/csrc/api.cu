@@ -1,0 +1,295 @@
+// C-ABI entry points: argument validation, workspace management and the order of kernel launches.
+#include <new>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace zipml {
+
+int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return ZIPML_OK;
+    (void)cudaGetLastError();
+    return ZIPML_ERR_CUDA;
+}
+
+static int grow(unsigned char** buf, size_t* have, size_t want, cudaStream_t stream) {
+    if (want <= *have) return ZIPML_OK;
+    // earlier work on the stream may still use the old buffer
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    if (*buf) { e = cudaFree(*buf); *buf = nullptr; *have = 0; if (e != cudaSuccess) return cuda_status(e); }
+    const size_t bytes = (want + (1u << 20) - 1) >> 20 << 20;
+    e = cudaMalloc(reinterpret_cast<void**>(buf), bytes);
+    if (e != cudaSuccess) { *buf = nullptr; return cuda_status(e); }
+    *have = bytes;
+    return ZIPML_OK;
+}
+
+int ws_reserve(zipml_ctx* ctx, size_t bytes) { return grow(&ctx->ws, &ctx->ws_bytes, bytes, ctx->stream); }
+int stage_reserve(zipml_ctx* ctx, size_t bytes) { return grow(&ctx->stage, &ctx->stage_bytes, bytes, ctx->stream); }
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int device) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { (void)cudaGetLastError(); prev = -1; }
+        ok = cudaSetDevice(device) == cudaSuccess;
+        if (!ok) (void)cudaGetLastError();
+    }
+    ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
+};
+
+static int check_dataset(const zipml_dataset* d) {
+    if (!d || d->struct_size != sizeof(zipml_dataset)) return ZIPML_ERR_INVALID_ARG;
+    const int cb = container_bits(d->bits);
+    if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
+    if (d->level_mode != ZIPML_LEVELS_UNIFORM && d->level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
+    if (d->level_mode == ZIPML_LEVELS_TABLE && d->bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (d->m <= 0 || d->n <= 0) return ZIPML_ERR_INVALID_ARG;
+    if (d->n > 0x7fffffffLL / 8) return ZIPML_ERR_WORKSPACE;
+    if (!d->plane1 || !d->plane2 || !aligned16(d->plane1) || !aligned16(d->plane2)) return ZIPML_ERR_INVALID_ARG;
+    if (d->row_bytes % 16 != 0 || d->row_bytes < zipml_row_bytes(d->n, d->bits)) return ZIPML_ERR_INVALID_ARG;
+    if (d->level_mode == ZIPML_LEVELS_UNIFORM && (!d->feat_lo || !d->feat_step)) return ZIPML_ERR_INVALID_ARG;
+    if (d->level_mode == ZIPML_LEVELS_TABLE && !d->levels) return ZIPML_ERR_INVALID_ARG;
+    return ZIPML_OK;
+}
+
+constexpr int kLossPartials = 4096;
+
+}  // namespace zipml
+
+using namespace zipml;
+
+extern "C" {
+
+const char* zipml_strerror(int status) {
+    switch (status) {
+        case ZIPML_OK: return "ok";
+        case ZIPML_ERR_INVALID_ARG: return "invalid argument";
+        case ZIPML_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ZIPML_ERR_NONFINITE: return "non-finite value in the input";
+        case ZIPML_ERR_CUDA: return "CUDA runtime error (no device, out of memory or failed launch)";
+        case ZIPML_ERR_TIMEOUT: return "a device-side wait gave up";
+        case ZIPML_ERR_WORKSPACE: return "problem does not fit the kernels' shared memory or scratch limits";
+        default: return "unknown status";
+    }
+}
+
+int64_t zipml_row_bytes(int64_t n, int32_t bits) {
+    const int cb = container_bits(bits);
+    if (cb == 0 || n <= 0) return 0;
+    return ((n * cb + 7) / 8 + 15) / 16 * 16;
+}
+
+int zipml_create(zipml_ctx** ctx_out, int device, void* cuda_stream) {
+    if (!ctx_out) return ZIPML_ERR_INVALID_ARG;
+    *ctx_out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        (void)cudaGetLastError();
+        return ZIPML_ERR_CUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    zipml_ctx* ctx = new (std::nothrow) zipml_ctx();
+    if (!ctx) return ZIPML_ERR_CUDA;
+    ctx->device = device;
+    ctx->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->cooperative, cudaDevAttrCooperativeLaunch, device);
+    if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(DeviceStatus), ctx->stream);
+    if (e != cudaSuccess) { if (ctx->d_status) (void)cudaFree(ctx->d_status); delete ctx; return cuda_status(e); }
+    *ctx_out = ctx;
+    return ZIPML_OK;
+}
+
+int zipml_destroy(zipml_ctx* ctx) {
+    if (!ctx) return ZIPML_OK;
+    DeviceGuard guard(ctx->device);
+    (void)cudaStreamSynchronize(ctx->stream);
+    if (ctx->ws) (void)cudaFree(ctx->ws);
+    if (ctx->stage) (void)cudaFree(ctx->stage);
+    if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    (void)cudaGetLastError();
+    delete ctx;
+    return ZIPML_OK;
+}
+
+int zipml_sync(zipml_ctx* ctx) {
+    if (!ctx) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    DeviceStatus host{0, 0};
+    cudaError_t e = cudaMemcpyAsync(&host, ctx->d_status, sizeof(host), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    if (host.code != 0) {
+        e = cudaMemsetAsync(ctx->d_status, 0, sizeof(DeviceStatus), ctx->stream);
+        if (e != cudaSuccess) return cuda_status(e);
+    }
+    return host.code;
+}
+
+int zipml_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
+                   int32_t level_mode, const float* levels, uint64_t seed, uint8_t* plane1, uint8_t* plane2,
+                   int64_t row_bytes, float* feat_lo, float* feat_step) {
+    if (!ctx) return ZIPML_ERR_INVALID_ARG;
+    const int cb = container_bits(bits);
+    if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
+    if (level_mode != ZIPML_LEVELS_UNIFORM && level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
+    if (level_mode == ZIPML_LEVELS_TABLE && bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (!A || !plane1 || !plane2 || !feat_lo || m <= 0 || n <= 0 || lda < n) return ZIPML_ERR_INVALID_ARG;
+    if (level_mode == ZIPML_LEVELS_TABLE && !levels) return ZIPML_ERR_INVALID_ARG;
+    if (level_mode == ZIPML_LEVELS_UNIFORM && !feat_step) return ZIPML_ERR_INVALID_ARG;
+    if (row_bytes % 16 != 0 || row_bytes < zipml_row_bytes(n, bits)) return ZIPML_ERR_INVALID_ARG;
+    if (!aligned16(plane1) || !aligned16(plane2)) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    const int s = (1 << bits) - 1;
+    int rc = ws_reserve(ctx, carve_size(sizeof(uint32_t) * 2 * (size_t)n) + 2 * carve_size(sizeof(float) * (size_t)n));
+    if (rc != ZIPML_OK) return rc;
+    Carver cv(ctx->ws);
+    uint32_t* keys = cv.take<uint32_t>(2 * (size_t)n);
+    float* inv = cv.take<float>((size_t)n);
+    float* step_tmp = cv.take<float>((size_t)n);
+    rc = launch_column_range(ctx, A, m, n, lda, s, keys, feat_lo, nullptr, inv, feat_step ? feat_step : step_tmp);
+    if (rc != ZIPML_OK) return rc;
+    return launch_quantize(ctx, A, m, n, lda, bits, level_mode, feat_lo, inv, levels, seed, plane1, plane2, row_bytes);
+}
+
+int zipml_optimal_levels(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
+                         int32_t hist_bins, float* levels_out, uint64_t* objective_out) {
+    if (!ctx) return ZIPML_ERR_INVALID_ARG;
+    if (bits != 2 && bits != 3 && bits != 4) return ZIPML_ERR_UNSUPPORTED;
+    const int s = (1 << bits) - 1;
+    if (!A || !levels_out || m <= 0 || n <= 0 || lda < n) return ZIPML_ERR_INVALID_ARG;
+    if (hist_bins < s || hist_bins > 1024 || m > 1000000000LL) return ZIPML_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    int rc = ws_reserve(ctx, carve_size(sizeof(uint32_t) * 2 * (size_t)n) + 3 * carve_size(sizeof(float) * (size_t)n) +
+                                 carve_size(sizeof(uint32_t) * (size_t)n * hist_bins));
+    if (rc != ZIPML_OK) return rc;
+    Carver cv(ctx->ws);
+    uint32_t* keys = cv.take<uint32_t>(2 * (size_t)n);
+    float* lo = cv.take<float>((size_t)n);
+    float* hi = cv.take<float>((size_t)n);
+    float* inv = cv.take<float>((size_t)n);
+    uint32_t* counts = cv.take<uint32_t>((size_t)n * hist_bins);
+    rc = launch_column_range(ctx, A, m, n, lda, hist_bins, keys, lo, hi, inv, nullptr);
+    if (rc != ZIPML_OK) return rc;
+    rc = launch_histogram(ctx, A, m, n, lda, hist_bins, lo, inv, counts);
+    if (rc != ZIPML_OK) return rc;
+    return launch_levels_dp(ctx, counts, n, hist_bins, s, lo, hi, levels_out, objective_out);
+}
+
+int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, float* x,
+                    const zipml_sgd_params* params, float* grad_out) {
+    if (!ctx || !params || params->struct_size != sizeof(zipml_sgd_params)) return ZIPML_ERR_INVALID_ARG;
+    int rc = check_dataset(data);
+    if (rc != ZIPML_OK) return rc;
+    if (!b || !x || params->batch <= 0) return ZIPML_ERR_INVALID_ARG;
+    if (params->model_bits != 0 && (params->model_bits < 2 || params->model_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
+    if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
+    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_PERSISTENT) return ZIPML_ERR_INVALID_ARG;
+    if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
+    const int64_t T = (data->m + params->batch - 1) / params->batch;
+    const int64_t first = params->first_step;
+    const int64_t count = params->num_steps < 0 ? T - first : params->num_steps;
+    if (first < 0 || first > T || count < 0 || first + count > T) return ZIPML_ERR_INVALID_ARG;
+    if (params->batch_order)
+        for (int64_t i = 0; i < T; ++i)
+            if (params->batch_order[i] < 0 || params->batch_order[i] >= T) return ZIPML_ERR_INVALID_ARG;
+    if (count == 0) return ZIPML_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    return launch_sgd_epoch(ctx, data, b, x, params, first, count, grad_out);
+}
+
+int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t n, int64_t lda,
+               const zipml_dataset* data, const float* b, const float* x, double* loss_out) {
+    if (!ctx || !b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
+    if (mode != ZIPML_LOSS_DENSE && mode != ZIPML_LOSS_CODES) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    if (mode == ZIPML_LOSS_DENSE) {
+        if (!A || m <= 0 || n <= 0 || lda < n) return ZIPML_ERR_INVALID_ARG;
+        int rc = ws_reserve(ctx, carve_size(sizeof(double) * kLossPartials));
+        if (rc != ZIPML_OK) return rc;
+        return launch_loss_dense(ctx, A, m, n, lda, b, x, reinterpret_cast<double*>(ctx->ws), kLossPartials, loss_out);
+    }
+    int rc = check_dataset(data);
+    if (rc != ZIPML_OK) return rc;
+    const size_t tab = (data->level_mode == ZIPML_LEVELS_TABLE ? ((size_t)1 << data->bits) : 1) * (size_t)data->n;
+    rc = ws_reserve(ctx, carve_size(sizeof(double) * (kLossPartials + 2) + sizeof(float) * tab));
+    if (rc != ZIPML_OK) return rc;
+    return launch_loss_codes(ctx, data, b, x, reinterpret_cast<double*>(ctx->ws), kLossPartials, loss_out);
+}
+
+int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, int64_t lda, const float* b_host,
+                     float* x_host, int32_t bits, int32_t optimal_levels, int32_t hist_bins, uint64_t quantize_seed,
+                     const zipml_sgd_params* params, int32_t epochs, int32_t lr_decay, double* loss_out_host) {
+    if (!ctx || !params || params->struct_size != sizeof(zipml_sgd_params)) return ZIPML_ERR_INVALID_ARG;
+    if (!A_host || !b_host || !x_host || !loss_out_host || m <= 0 || n <= 0 || lda < n || epochs < 0)
+        return ZIPML_ERR_INVALID_ARG;
+    const int64_t rb = zipml_row_bytes(n, bits);
+    if (rb == 0) return ZIPML_ERR_UNSUPPORTED;
+    if (optimal_levels && bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    const size_t L = (size_t)1 << bits;
+    size_t total = 0;
+    auto piece = [&](size_t bytes) { const size_t off = total; total += carve_size(bytes); return off; };
+    const size_t oA = piece(sizeof(float) * (size_t)m * n), ob = piece(sizeof(float) * (size_t)m);
+    const size_t ox = piece(sizeof(float) * (size_t)n), op1 = piece((size_t)m * rb), op2 = piece((size_t)m * rb);
+    const size_t olo = piece(sizeof(float) * (size_t)n), ostep = piece(sizeof(float) * (size_t)n);
+    const size_t olev = piece(sizeof(float) * (size_t)n * L), oloss = piece(sizeof(double));
+    int rc = stage_reserve(ctx, total);
+    if (rc != ZIPML_OK) return rc;
+    unsigned char* s = ctx->stage;
+    float* dA = reinterpret_cast<float*>(s + oA);
+    float* db = reinterpret_cast<float*>(s + ob);
+    float* dx = reinterpret_cast<float*>(s + ox);
+    float* dlev = reinterpret_cast<float*>(s + olev);
+    double* dloss = reinterpret_cast<double*>(s + oloss);
+    cudaError_t e = cudaMemcpy2DAsync(dA, sizeof(float) * n, A_host, sizeof(float) * lda, sizeof(float) * n, (size_t)m,
+                                      cudaMemcpyHostToDevice, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(db, b_host, sizeof(float) * m, cudaMemcpyHostToDevice, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dx, x_host, sizeof(float) * n, cudaMemcpyHostToDevice, ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+
+    zipml_dataset d{};
+    d.struct_size = sizeof(zipml_dataset);
+    d.bits = bits; d.m = m; d.n = n; d.row_bytes = rb;
+    d.plane1 = s + op1; d.plane2 = s + op2;
+    d.feat_lo = reinterpret_cast<float*>(s + olo);
+    d.feat_step = reinterpret_cast<float*>(s + ostep);
+    d.levels = nullptr;
+    d.level_mode = optimal_levels ? ZIPML_LEVELS_TABLE : ZIPML_LEVELS_UNIFORM;
+    if (optimal_levels) {
+        rc = zipml_optimal_levels(ctx, dA, m, n, n, bits, hist_bins, dlev, nullptr);
+        if (rc != ZIPML_OK) return rc;
+        d.levels = dlev;
+    }
+    rc = zipml_quantize(ctx, dA, m, n, n, bits, d.level_mode, d.levels, quantize_seed, s + op1, s + op2, rb,
+                        reinterpret_cast<float*>(s + olo), reinterpret_cast<float*>(s + ostep));
+    if (rc != ZIPML_OK) return rc;
+    zipml_sgd_params p = *params;
+    for (int32_t ep = 0; ep < epochs; ++ep) {
+        p.epoch = ep; p.first_step = 0; p.num_steps = -1;
+        p.lr = lr_decay ? params->lr / (float)(ep + 1) : params->lr;
+        rc = zipml_sgd_epoch(ctx, &d, db, dx, &p, nullptr);
+        if (rc != ZIPML_OK) return rc;
+    }
+    rc = zipml_loss(ctx, ZIPML_LOSS_DENSE, dA, m, n, n, nullptr, db, dx, dloss);
+    if (rc != ZIPML_OK) return rc;
+    e = cudaMemcpyAsync(x_host, dx, sizeof(float) * n, cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(loss_out_host, dloss, sizeof(double), cudaMemcpyDeviceToHost, ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    return zipml_sync(ctx);
+}
+
+}  // extern "C"

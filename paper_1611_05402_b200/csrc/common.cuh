@@ -1,0 +1,123 @@
+// Device helpers shared by the kernels: the counter-based random numbers, the pinned fp32
+// rounding decision, container widths and a few warp/block reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/zipml.h"
+
+namespace zipml {
+
+// Device-side status word values (ORed is not needed: first error wins).
+struct DeviceStatus {
+    int code;          // ZIPML_OK or a ZIPML_ERR_* value, set with atomicCAS from 0
+    int detail;        // where a wait gave up, or 0
+};
+
+__device__ __forceinline__ void set_status(DeviceStatus* st, int code, int detail) {
+    if (atomicCAS(&st->code, 0, code) == 0) st->detail = detail;
+}
+
+__host__ __device__ __forceinline__ int container_bits(int bits) {
+    return bits == 2 ? 2 : (bits == 3 || bits == 4) ? 4 : bits == 8 ? 8 : 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11), written from its published round function.
+// ---------------------------------------------------------------------------------------------
+struct Philox4 {
+    uint32_t v[4];
+};
+
+__device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                 uint32_t k0, uint32_t k1) {
+    constexpr uint32_t kMul0 = 0xD2511F53u, kMul1 = 0xCD9E8D57u;
+    constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(kMul0, c0), lo0 = kMul0 * c0;
+        const uint32_t hi1 = __umulhi(kMul1, c2), lo1 = kMul1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += kWeyl0;
+        k1 += kWeyl1;
+    }
+    Philox4 out;
+    out.v[0] = c0; out.v[1] = c1; out.v[2] = c2; out.v[3] = c3;
+    return out;
+}
+
+// Random block of the sample feature pair (2p, 2p+1) of row `row`: words {2p copy 1, 2p copy 2,
+// 2p+1 copy 1, 2p+1 copy 2}; the top 24 bits of a word are the uniform integer.
+__device__ __forceinline__ Philox4 sample_block(uint64_t seed, uint64_t row, uint32_t pair) {
+    return philox4x32_10((uint32_t)row, (uint32_t)(row >> 32), pair, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+}
+
+// Uniform 24-bit integer for coordinate `coord` of the model (stream 3) / gradient (stream 4)
+// quantizer at (epoch, step).
+__device__ __forceinline__ uint32_t vector_u24(uint64_t seed, uint32_t epoch, uint32_t step, uint32_t coord,
+                                               uint32_t stream) {
+    const Philox4 b = philox4x32_10(coord >> 2, step, epoch, stream, (uint32_t)seed, (uint32_t)(seed >> 32));
+    return b.v[coord & 3u] >> 8;
+}
+
+// up <=> u24 * 2^-24 < p, both sides fp32 (the product is exact).
+__device__ __forceinline__ uint32_t round_up_if(uint32_t cell, float p, uint32_t word) {
+    const float u = __fmul_rn((float)(word >> 8), 5.9604644775390625e-08f);
+    return cell + (u < p ? 1u : 0u);
+}
+
+// Cell and up-probability on a uniform grid of s intervals: t = (v - lo) * inv with every
+// operation rounded on its own (no contraction into an FMA).
+__device__ __forceinline__ void uniform_cell(float v, float lo, float inv, int s, uint32_t& cell, float& p) {
+    const float t = __fmul_rn(__fsub_rn(v, lo), inv);
+    float fl = floorf(t);
+    fl = fl < 0.0f ? 0.0f : fl;                    // a NaN falls through both comparisons ...
+    fl = fl > (float)(s - 1) ? (float)(s - 1) : fl;
+    cell = (fl == fl) ? (uint32_t)fl : 0u;         // ... and lands in cell 0
+    p = __fsub_rn(t, fl);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum over the block in a fixed order (warp results combined by thread 0); every thread gets the
+// result.  `scratch` holds at least 33 doubles.  Ends with the block synchronised.
+__device__ __forceinline__ double block_sum(double v, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < nwarps; ++w) t += scratch[w];
+        scratch[32] = t;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+// Order-preserving map float -> uint32 so that integer atomicMin/Max order floats (-0 < +0).
+__device__ __forceinline__ uint32_t float_order_key(float f) {
+    const uint32_t b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ float float_from_order_key(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+}  // namespace zipml

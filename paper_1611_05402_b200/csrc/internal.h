@@ -1,0 +1,77 @@
+// Host-side internals of the library: the context and the kernel launchers that the C-ABI entry
+// points call.  Not part of the public interface.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/zipml.h"
+
+namespace zipml {
+struct DeviceStatus;
+}
+
+struct zipml_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int sm_count = 0;
+    int smem_optin = 0;             // max dynamic shared memory per block (opt-in), bytes
+    int cooperative = 0;            // device supports cooperative launch
+    unsigned char* ws = nullptr;    // general workspace
+    size_t ws_bytes = 0;
+    zipml::DeviceStatus* d_status = nullptr;
+    // staging buffers of zipml_train_host (grown on demand)
+    unsigned char* stage = nullptr;
+    size_t stage_bytes = 0;
+};
+
+namespace zipml {
+
+// Status helpers -------------------------------------------------------------------------------
+int cuda_status(cudaError_t e);                       // ZIPML_OK or ZIPML_ERR_CUDA (clears the sticky error)
+int ws_reserve(zipml_ctx* ctx, size_t bytes);         // grow ctx->ws to at least `bytes`
+int stage_reserve(zipml_ctx* ctx, size_t bytes);
+
+// Simple bump carving of the workspace: 256-byte aligned pieces.
+struct Carver {
+    unsigned char* base;
+    size_t off = 0;
+    explicit Carver(unsigned char* b) : base(b) {}
+    template <typename T>
+    T* take(size_t count) {
+        T* p = reinterpret_cast<T*>(base + off);
+        off += (count * sizeof(T) + 255) / 256 * 256;
+        return p;
+    }
+};
+inline size_t carve_size(size_t bytes) { return (bytes + 255) / 256 * 256; }
+
+// Launchers (each enqueues on ctx->stream and returns a status) -------------------------------
+// Column range: lo/hi per feature, inv = s/(hi-lo) and step = (hi-lo)/s for a grid of s intervals.
+// Any of hi_out, inv_out, step_out may be null.  Sets NONFINITE in the device status.
+int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int s,
+                        uint32_t* key_scratch /* 2n */, float* lo_out, float* hi_out, float* inv_out,
+                        float* step_out);
+
+int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
+                    const float* lo, const float* inv, const float* levels, uint64_t seed, uint8_t* plane1,
+                    uint8_t* plane2, int64_t row_bytes);
+
+int launch_histogram(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bins,
+                     const float* lo, const float* inv, uint32_t* counts /* n x bins, zeroed here */);
+
+int launch_levels_dp(zipml_ctx* ctx, const uint32_t* counts, int64_t n, int bins, int s, const float* lo,
+                     const float* hi, float* levels_out, uint64_t* objective_out);
+
+int launch_loss_dense(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, const float* b,
+                      const float* x, double* partials, int max_partials, double* loss_out);
+
+int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, const float* x, double* partials,
+                      int max_partials, double* loss_out);
+
+size_t sgd_workspace_bytes(const zipml_ctx* ctx, const zipml_dataset* d, const zipml_sgd_params* p);
+int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                     int64_t first_step, int64_t num_steps, float* grad_out);
+
+}  // namespace zipml

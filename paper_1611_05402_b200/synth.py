@@ -3,7 +3,7 @@
 The paper's datasets (its dataset table: Synthetic 10/100/1000, YearPrediction, cadata, cpusmall,
 cod-rna, gisette, a 128-projection tomography volume) are not available here; the five workloads
 below stand in for their shapes.  This module holds no arithmetic of the method itself: it only
-draws A, x*, b = A x* + noise.  The same arrays feed the CUDA path and the CPU oracle.
+draws A, x*, b = A x* + noise.  The same arrays feed the CUDA path and whatever checks it.
 
 Every generator takes (m, n) overrides so that tests can run reduced sizes with the same
 distributions, and a torch device so that full sizes can be drawn directly in device memory.

@@ -1,0 +1,335 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Tolerances (from the benchmark spec): packed codes and optimal levels bit-exact; per-step
+gradients <= 1e-5 relative L2; model after one epoch with the same minibatch order <= 1e-4 relative
+L2; loss within 1e-3 relative (the kernels are far inside that: the tests use 1e-6).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1611_05402_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+GRAD_TOL, MODEL_TOL, LOSS_TOL = 1e-5, 1e-4, 1e-6
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_1611_05402_b200.build import build
+    build()
+    c = binding.Context("cuda:0")
+    yield c
+    c.close()
+
+
+def rel(a, b):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def to_dev(a, ctx):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(ctx.device)
+
+
+def dev_dataset(ods, ctx):
+    """Oracle dataset -> device dataset (so that SGD parity does not depend on quantize parity)."""
+    return binding.Dataset(to_dev(ods.plane1, ctx), to_dev(ods.plane2, ctx), ods.m, ods.n, ods.bits, ods.mode,
+                           to_dev(ods.feat_lo, ctx), to_dev(ods.feat_step, ctx) if ods.mode == oracle.UNIFORM else None,
+                           to_dev(ods.levels, ctx) if ods.levels is not None else None)
+
+
+def workload(key, m, n, seed=0):
+    w, A, b, xs = synth.make(key, m=m, n=n, seed=seed)
+    return w, A.numpy(), b.numpy(), xs.numpy()
+
+
+# ---------------------------------------------------------------------------------------------
+# quantize: bit-exact planes and scales
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("key,m,n,bits", [
+    ("c1", 300, 64, 4), ("c1", 257, 61, 4), ("c2", 500, 1000, 8), ("c2", 129, 1003, 8), ("c3", 200, 2048, 2),
+    ("c3", 77, 2050, 2), ("c3", 5, 1, 2), ("c4u", 333, 512, 3), ("c4u", 100, 37, 3), ("c5", 40, 4100, 4),
+    ("c1", 1, 5, 8), ("c2", 3000, 7, 2),
+])
+def test_quantize_bit_exact(ctx, key, m, n, bits):
+    _, A, _, _ = workload(key, m, n, seed=bits)
+    if m > 2:
+        A[:, n // 2] = 0.25                                        # a constant feature
+    ods = oracle.quantize(A, bits, seed=1234 + m)
+    gds = ctx.zipml_quantize(to_dev(A, ctx), bits, seed=1234 + m)
+    ctx.zipml_sync()
+    assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all()
+    assert (gds.feat_step.cpu().numpy() == ods.feat_step).all()
+    assert gds.row_bytes == ods.row_bytes
+    assert (gds.plane1.cpu().numpy() == ods.plane1).all()
+    assert (gds.plane2.cpu().numpy() == ods.plane2).all()
+
+
+def test_quantize_strided_and_unaligned_input(ctx):
+    _, A, _, _ = workload("c2", 200, 101, seed=3)
+    big = torch.zeros((200, 131), dtype=torch.float32, device=ctx.device)
+    big[:, 3:104] = to_dev(A, ctx)
+    view = big[:, 3:104]                                           # lda = 131, base not 16-byte aligned
+    ods = oracle.quantize(A, 4, seed=9)
+    gds = ctx.zipml_quantize(view, 4, seed=9, row_bytes=ods.row_bytes + 32)
+    ctx.zipml_sync()
+    assert (gds.plane1.cpu().numpy()[:, : ods.row_bytes] == ods.plane1).all()
+    assert (gds.plane2.cpu().numpy()[:, : ods.row_bytes] == ods.plane2).all()
+    assert not gds.plane1.cpu().numpy()[:, ods.row_bytes:].any()
+    assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all()
+
+
+def test_quantize_reports_bad_input(ctx):
+    A = torch.rand((64, 16), device=ctx.device)
+    A[5, 3] = float("nan")
+    ctx.zipml_quantize(A, 4, seed=0)
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sync()
+    assert e.value.code == binding.ERR_NONFINITE
+    ctx.zipml_sync()                                               # the error is reported once, then cleared
+    A[5, 3] = float("inf")
+    ctx.zipml_quantize(A, 4, seed=0)
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sync()
+    good = torch.rand((64, 16), device=ctx.device)
+    for bits in (1, 5, 16):
+        with pytest.raises(binding.ZipmlError) as e:
+            ctx.zipml_quantize(good, bits, seed=0)
+        assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_quantize(good, 4, seed=0, row_bytes=8)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_quantize(good, 8, seed=0, level_mode=binding.LEVELS_TABLE,
+                           levels=torch.zeros((16, 256), device=ctx.device))
+    assert e.value.code == binding.ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------------------------------------
+# optimal levels: bit-exact levels and objective; table quantization bit-exact
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("m,n,bits,bins", [(5000, 40, 3, 1024), (3000, 33, 2, 256), (2000, 16, 4, 1024), (700, 5, 3, 7),
+                                           (64, 3, 4, 1000)])
+def test_optimal_levels_bit_exact(ctx, m, n, bits, bins):
+    _, A, _, _ = workload("c4", m, n, seed=bins)
+    A[:, n - 1] = -0.5                                             # a constant feature
+    lev, obj = oracle.optimal_levels(A, bits, bins)
+    glev, gobj = ctx.zipml_optimal_levels(to_dev(A, ctx), bits, bins, want_objective=True)
+    ctx.zipml_sync()
+    assert (gobj.cpu().numpy().astype(np.uint64) == obj).all()
+    assert (glev.cpu().numpy() == lev).all()
+    ods = oracle.quantize(A, bits, seed=5, mode=oracle.TABLE, levels=lev)
+    gds = ctx.zipml_quantize(to_dev(A, ctx), bits, seed=5, level_mode=binding.LEVELS_TABLE, levels=glev)
+    ctx.zipml_sync()
+    assert (gds.plane1.cpu().numpy() == ods.plane1).all() and (gds.plane2.cpu().numpy() == ods.plane2).all()
+    assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# SGD: per-step gradient from identical x_t, model after an epoch, both engines, several grids
+# ---------------------------------------------------------------------------------------------
+SGD_CASES = [
+    # key, m, n, bits, batch, lr
+    ("c1", 1000, 64, 4, 16, 0.01),
+    ("c2", 2100, 1000, 8, 256, 1e-3),         # ragged tail: 2100 = 8*256 + 52
+    ("c3", 2500, 2048, 2, 1024, 5e-4),
+    ("c4u", 1500, 512, 3, 512, 1e-3),
+    ("c5", 300, 4099, 4, 128, 1e-4),          # n not a multiple of anything
+    ("c2", 100, 33, 8, 7, 1e-2),
+    ("c1", 50, 5, 2, 64, 0.05),               # batch larger than m
+]
+GRIDS = [(0, 0), (1, 1), (1, 5), (2, 3), (3, 1)]
+
+
+@pytest.mark.parametrize("case", SGD_CASES, ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
+@pytest.mark.parametrize("engine", [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT])
+def test_sgd_epoch_parity(ctx, case, engine):
+    key, m, n, bits, batch, lr = case
+    _, A, b, _ = workload(key, m, n, seed=1)
+    ods = oracle.quantize(A, bits, seed=7)
+    gds = dev_dataset(ods, ctx)
+    db = to_dev(b, ctx)
+    T = (m + batch - 1) // batch
+    order = np.random.default_rng(0).permutation(T).astype(np.int32)
+    x0 = (np.random.default_rng(1).standard_normal(n) * 0.1).astype(np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order)
+    # model just before the last step, for the per-step gradient check
+    x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order, num_steps=T - 1)
+    _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, batch_order=order, first_step=T - 1, num_steps=1,
+                                want_grad=True)
+    for fa, fb in GRIDS:
+        x = to_dev(x0, ctx)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, batch_order=order, engine=engine, grid_feature_parts=fa,
+                            grid_row_parts=fb)
+        ctx.zipml_sync()
+        assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL, (fa, fb)
+        xb = to_dev(x_before, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, batch_order=order, first_step=T - 1, num_steps=1, engine=engine,
+                            grid_feature_parts=fa, grid_row_parts=fb, grad_out=g)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL, (fa, fb)
+        assert (g[0] == g[1]).all()
+        assert rel(xb.cpu().numpy(), x_ref) <= MODEL_TOL
+
+
+def test_sgd_engines_and_grids_agree_bitwise_where_the_reduction_order_is_the_same(ctx):
+    _, A, b, _ = workload("c2", 1500, 300, seed=2)
+    ods = oracle.quantize(A, 8, seed=1)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    outs = []
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT):
+        x = torch.zeros(300, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, x, 128, 1e-3, engine=engine, grid_feature_parts=2, grid_row_parts=4)
+        ctx.zipml_sync()
+        outs.append(x.cpu().numpy())
+    assert (outs[0] == outs[1]).all()
+    # and a second run is bit-identical to the first: no atomics, fixed reduction order
+    x = torch.zeros(300, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, x, 128, 1e-3, engine=binding.ENGINE_PERSISTENT, grid_feature_parts=2, grid_row_parts=4)
+    ctx.zipml_sync()
+    assert (x.cpu().numpy() == outs[1]).all()
+
+
+def test_sgd_table_levels_parity(ctx):
+    _, A, b, _ = workload("c4", 3000, 100, seed=4)
+    lev, _ = oracle.optimal_levels(A, 3, 256)
+    ods = oracle.quantize(A, 3, seed=3, mode=oracle.TABLE, levels=lev)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = np.zeros(100, np.float32)
+    x_ref, g_ref = oracle.sgd_epoch(ods, b, x0, 512, 1e-2, want_grad=True)
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT):
+        for fa, fb in GRIDS:
+            x = to_dev(x0, ctx)
+            g = torch.zeros((2, 100), dtype=torch.float32, device=ctx.device)
+            ctx.zipml_sgd_epoch(gds, db, x, 512, 1e-2, engine=engine, grid_feature_parts=fa, grid_row_parts=fb,
+                                grad_out=g)
+            ctx.zipml_sync()
+            assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    # per-step gradient from the same x
+    _, g1 = oracle.sgd_epoch(ods, b, x_ref, 512, 1e-2, first_step=2, num_steps=1, want_grad=True)
+    x = to_dev(x_ref, ctx)
+    g = torch.zeros((2, 100), dtype=torch.float32, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, x, 512, 1e-2, first_step=2, num_steps=1, grad_out=g)
+    ctx.zipml_sync()
+    assert rel(g[0].cpu().numpy(), g1[0]) <= GRAD_TOL
+
+
+@pytest.mark.parametrize("model_bits,grad_bits", [(8, 0), (0, 8), (8, 8), (4, 4)])
+def test_sgd_end_to_end_quantization(ctx, model_bits, grad_bits):
+    _, A, b, _ = workload("c3", 3000, 512, seed=6)
+    ods = oracle.quantize(A, 2, seed=2)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = (np.random.default_rng(3).standard_normal(512) * 0.05).astype(np.float32)
+    # one step from identical x: the pre-Q4 gradient must agree to GRAD_TOL; the quantized
+    # quantities must agree exactly except where a stochastic rounding sits within 1e-4 of its
+    # threshold (a sub-ulp difference in the norm may flip those)
+    _, g_ref = oracle.sgd_epoch(ods, b, x0, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
+                                first_step=1, num_steps=1, want_grad=True)
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT):
+        x = to_dev(x0, ctx)
+        g = torch.zeros((2, 512), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
+                            first_step=1, num_steps=1, engine=engine, grad_out=g)
+        ctx.zipml_sync()
+        gg = g.cpu().numpy()
+        if model_bits == 0:
+            assert rel(gg[0], g_ref[0]) <= GRAD_TOL
+        else:
+            # a flipped model coordinate changes the gradient by about |a_j|*|step|: allow a few
+            assert rel(gg[0], g_ref[0]) <= 5e-3
+        if grad_bits:
+            sm = (1 << (grad_bits - 1)) - 1
+            unit = np.linalg.norm(g_ref[0]) / sm
+            flips = np.abs(gg[1] - g_ref[1]) > 0.5 * unit
+            assert flips.sum() <= 3
+            assert np.abs(gg[1] - g_ref[1])[~flips].max() <= 1e-5 * unit + 1e-12
+    # whole epoch: the trajectories stay together within the model tolerance
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2)
+    ctx.zipml_sync()
+    assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
+
+
+def test_sgd_split_calls_equal_one_call(ctx):
+    _, A, b, _ = workload("c1", 640, 64, seed=9)
+    ods = oracle.quantize(A, 4, seed=1)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x_all = torch.zeros(64, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, x_all, 16, 0.01)
+    x_two = torch.zeros(64, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, x_two, 16, 0.01, first_step=0, num_steps=13)
+    ctx.zipml_sgd_epoch(gds, db, x_two, 16, 0.01, first_step=13)
+    ctx.zipml_sync()
+    assert (x_all == x_two).all()
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, x_two, 16, 0.01, first_step=39, num_steps=5)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_epoch(gds, db, x_two, 0, 0.01)
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_epoch(gds, db, x_two, 16, 0.01, batch_order=np.full(40, 99, np.int32))
+
+
+# ---------------------------------------------------------------------------------------------
+# loss
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("key,m,n,bits", [("c1", 1000, 64, 4), ("c2", 700, 1001, 8), ("c3", 300, 2048, 2),
+                                          ("c5", 100, 5000, 4), ("c4u", 900, 77, 3)])
+def test_loss_parity(ctx, key, m, n, bits):
+    _, A, b, xs = workload(key, m, n, seed=2)
+    x = (xs * 0.9).astype(np.float32)
+    want = oracle.loss_dense(A, b, x)
+    got = ctx.zipml_loss(binding.LOSS_DENSE, to_dev(b, ctx), to_dev(x, ctx), A=to_dev(A, ctx))
+    ods = oracle.quantize(A, bits, seed=3)
+    want_c = oracle.loss_codes(ods, b, x)
+    got_c = ctx.zipml_loss(binding.LOSS_CODES, to_dev(b, ctx), to_dev(x, ctx), data=dev_dataset(ods, ctx))
+    ctx.zipml_sync()
+    assert abs(got.item() - want) <= LOSS_TOL * abs(want)
+    assert abs(got_c.item() - want_c) <= LOSS_TOL * max(abs(want_c), abs(want))
+
+
+def test_loss_codes_with_level_table_and_strided_dense(ctx):
+    _, A, b, xs = workload("c4", 2000, 60, seed=1)
+    lev, _ = oracle.optimal_levels(A, 3, 128)
+    ods = oracle.quantize(A, 3, seed=3, mode=oracle.TABLE, levels=lev)
+    want_c = oracle.loss_codes(ods, b, xs)
+    got_c = ctx.zipml_loss(binding.LOSS_CODES, to_dev(b, ctx), to_dev(xs, ctx), data=dev_dataset(ods, ctx))
+    big = torch.zeros((2000, 71), device=ctx.device)
+    big[:, 1:61] = to_dev(A, ctx)
+    got = ctx.zipml_loss(binding.LOSS_DENSE, to_dev(b, ctx), to_dev(xs, ctx), A=big[:, 1:61])
+    ctx.zipml_sync()
+    assert abs(got_c.item() - want_c) <= LOSS_TOL * abs(want_c)
+    assert abs(got.item() - oracle.loss_dense(A, b, xs)) <= LOSS_TOL * oracle.loss_dense(A, b, xs)
+
+
+# ---------------------------------------------------------------------------------------------
+# whole path from host buffers
+# ---------------------------------------------------------------------------------------------
+def test_train_host_matches_oracle_pipeline(ctx):
+    w, A, b, _ = workload("c1", 2048, 64, seed=0)
+    x = torch.zeros(64)
+    loss = ctx.zipml_train_host(torch.from_numpy(A), torch.from_numpy(b), x, bits=4, batch=16, lr=0.01, epochs=3,
+                                quantize_seed=5)
+    ods = oracle.quantize(A, 4, seed=5)
+    xr = np.zeros(64, np.float32)
+    for ep in range(3):
+        xr, _ = oracle.sgd_epoch(ods, b, xr, 16, 0.01, epoch=ep)
+    assert rel(x.numpy(), xr) <= MODEL_TOL
+    want = oracle.loss_dense(A, b, xr)
+    assert abs(loss - want) <= 1e-3 * want
+    # with optimal levels and the alpha/epoch schedule
+    w, A, b, _ = workload("c4", 3000, 48, seed=0)
+    x = torch.zeros(48)
+    loss = ctx.zipml_train_host(torch.from_numpy(A), torch.from_numpy(b), x, bits=3, batch=512, lr=0.05, epochs=2,
+                                optimal_levels=True, hist_bins=256, quantize_seed=8, lr_decay=True)
+    lev, _ = oracle.optimal_levels(A, 3, 256)
+    ods = oracle.quantize(A, 3, seed=8, mode=oracle.TABLE, levels=lev)
+    xr = np.zeros(48, np.float32)
+    for ep in range(2):
+        xr, _ = oracle.sgd_epoch(ods, b, xr, 512, np.float32(0.05) / np.float32(ep + 1), epoch=ep)
+    assert rel(x.numpy(), xr) <= MODEL_TOL
+    assert abs(loss - oracle.loss_dense(A, b, xr)) <= 1e-3 * oracle.loss_dense(A, b, xr)
