@@ -1,0 +1,301 @@
+#!/usr/bin/env python
+"""Benchmark of the double-sampled low-precision SGD path.
+
+A "step" is one pass of the whole path over one synthetic workload: quantize the dense fp32
+samples into two packed planes (after placing variance-optimal levels, if the workload asks for
+them), run the workload's SGD epochs over the planes, evaluate the dense training loss.
+
+  value         samples/s = (m * epochs) / step time, inputs already resident in device memory
+  e2e           the same through zipml_train_host with pinned HOST buffers (copies in the timed region)
+  roofline      packed-code bytes per SGD-epoch launch / its CUDA-event duration, against the
+                measured HBM copy rate
+  cpu_baseline  the CPU oracle as it stands, timed on this host (rank 0, N = 1 only)
+
+`--impl reference` times the oracle alone (the reference arm of this tier).
+With N > 1 ranks every rank runs its own replica of the workload (the path is single-GPU; there is
+no data-path collective), and value is the sum over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        mhz = sorted(int(r[0]) for r in self.rows if r and r[0].isdigit())
+        mx = [int(r[1]) for r in self.rows if len(r) > 1 and r[1].isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 2 + i and r[2 + i].lower().startswith("active")
+                                                         for r in self.rows)]
+        return {"sm_mhz": mhz[len(mhz) // 2] if mhz else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(mhz)}
+
+
+def run_oracle_pass(w, A, b, max_seconds=None):
+    """One pass of the whole path on the CPU oracle; returns (seconds, samples processed, x, loss)."""
+    import numpy as np
+    import oracle
+    t0 = time.perf_counter()
+    levels = None
+    if w.levels == "optimal":
+        levels, _ = oracle.optimal_levels(A, w.bits, w.hist_bins)
+    ds = oracle.quantize(A, w.bits, seed=w.seed, mode=oracle.TABLE if levels is not None else oracle.UNIFORM,
+                         levels=levels)
+    x = np.zeros(w.n, np.float32)
+    for ep in range(w.epochs):
+        x, _ = oracle.sgd_epoch(ds, b, x, w.batch, w.lr, model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed,
+                                epoch=ep)
+    loss = oracle.loss_dense(A, b, x)
+    return time.perf_counter() - t0, w.m * w.epochs, x, loss
+
+
+def oracle_sample_rows(w):
+    """Rows of the workload the oracle is timed on: about 10-30 s of single-core work."""
+    # measured cost on one core: ~75 ns per element to quantize, ~9 ns per element and epoch of SGD
+    per_row = w.n * (75e-9 + 9e-9 * w.epochs + 2e-9) + (w.n * 60e-9 if w.levels == "optimal" else 0)
+    rows = int(15.0 / per_row)
+    rows = max(w.batch * 4, min(w.m, rows))
+    return min(w.m, rows // w.batch * w.batch if rows >= w.batch else rows)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
+    ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
+    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent"])
+    ap.add_argument("--feature-parts", type=int, default=0)
+    ap.add_argument("--row-parts", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_1611_05402_b200 import synth
+    base = synth.WORKLOADS[args.workload]
+    metric, unit = "samples/sec over the whole path (quantize + SGD epochs + loss)", "samples/s"
+
+    # ------------------------------------------------------------------ reference arm: the oracle
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        import numpy as np
+        from oracle.build import build as build_oracle
+        build_oracle()
+        w0 = synth.Workload(**{**base.__dict__})
+        if args.m:
+            w0.m = args.m
+        rows = oracle_sample_rows(w0)
+        # spread the few-minute budget over warmup + steps
+        rows = max(w0.batch, int(rows / max(1, (args.steps + args.warmup) / 4)) // w0.batch * w0.batch)
+        rows = min(rows, w0.m)
+        w, A, b, _ = synth.make(args.workload, m=rows)
+        A, b = A.numpy(), b.numpy()
+        for _ in range(args.warmup):
+            run_oracle_pass(w, A, b)
+        t = 0.0
+        for _ in range(args.steps):
+            dt, samples, _, _ = run_oracle_pass(w, A, b)
+            t += dt
+        value = samples * args.steps / t
+        sample = f"first {rows} of {w0.m} rows of {args.workload}, all {w.epochs} epochs, single thread"
+        print(json.dumps({
+            "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w0.name, "m": w0.m, "n": w0.n, "bits": w0.bits, "batch": w0.batch, "epochs": w0.epochs},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0,
+        }))
+        return
+
+    # ------------------------------------------------------------------ our arm
+    import torch
+    import torch.distributed as dist
+    from paper_1611_05402_b200 import binding
+    from paper_1611_05402_b200.build import build as build_cuda
+    if rank == 0:
+        build_cuda()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT}[args.engine]
+
+    w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
+    ctx = binding.Context(dev)
+    loss_dev = torch.zeros(1, dtype=torch.float64, device=dev)
+    kw = dict(model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed, engine=engine,
+              grid_feature_parts=args.feature_parts, grid_row_parts=args.row_parts)
+    epoch_events = []
+
+    def one_pass(record):
+        levels = ctx.zipml_optimal_levels(A, w.bits, w.hist_bins) if w.levels == "optimal" else None
+        ds = ctx.zipml_quantize(A, w.bits, seed=w.seed, level_mode=binding.LEVELS_TABLE if levels is not None else
+                                binding.LEVELS_UNIFORM, levels=levels)
+        x = torch.zeros(w.n, dtype=torch.float32, device=dev)
+        for ep in range(w.epochs):
+            if record:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            ctx.zipml_sgd_epoch(ds, b, x, w.batch, w.lr, epoch=ep, **kw)
+            if record:
+                e1.record()
+                epoch_events.append((e0, e1))
+        ctx.zipml_loss(binding.LOSS_DENSE, b, x, A=A, out=loss_dev)
+        return ds, x
+
+    def fence():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 0)):
+        ds, x = one_pass(False)
+    ctx.zipml_sync()
+    sampler = ClockSampler(local_rank)
+    fence()
+    launches0 = ctx.zipml_kernel_launches()
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        ds, x = one_pass(True)
+    t1.record()
+    fence()
+    clocks = sampler.stop()
+    ctx.zipml_sync()
+    launches = ctx.zipml_kernel_launches() - launches0
+    ms = torch.tensor([t0.elapsed_time(t1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms_total = float(ms.item())
+    value = world * w.m * w.epochs * args.steps / (ms_total * 1e-3)
+    final_loss = float(loss_dev.item())
+
+    # dominant kernel: the SGD epoch launch
+    epoch_ms = sorted(a.elapsed_time(b_) for a, b_ in epoch_events)
+    epoch_avg_ms = sum(epoch_ms) / len(epoch_ms)
+    packed_bytes = ds.packed_bytes
+    peak, peak_kind = measured_peaks()
+    achieved = packed_bytes / (epoch_avg_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": f"of {peak_kind} copy rate", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "kernel": "sgd_kernel (one launch per epoch)", "algorithmic_bytes_per_launch": packed_bytes,
+                "launch_ms_avg": epoch_avg_ms, "launch_ms_min": epoch_ms[0],
+                "epoch_samples_per_s": w.m / (epoch_avg_ms * 1e-3)}
+
+    # ------------------------------------------------------------------ end to end from host buffers
+    e2e = None
+    if not args.no_e2e:
+        Ah = torch.empty(A.shape, dtype=torch.float32, pin_memory=True)
+        Ah.copy_(A)
+        bh = torch.empty(b.shape, dtype=torch.float32, pin_memory=True)
+        bh.copy_(b)
+        xh = torch.zeros(w.n, dtype=torch.float32, pin_memory=True)
+
+        def host_pass():
+            xh.zero_()
+            return ctx.zipml_train_host(Ah, bh, xh, w.bits, w.batch, w.lr, w.epochs, optimal_levels=w.levels == "optimal",
+                                        hist_bins=w.hist_bins, quantize_seed=w.seed, **kw)
+        host_pass()
+        fence()
+        h0 = time.perf_counter()
+        k_e2e = max(1, min(args.steps, 3))
+        for _ in range(k_e2e):
+            e2e_loss = host_pass()
+        torch.cuda.synchronize()
+        dt = torch.tensor([time.perf_counter() - h0], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(dt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * w.m * w.epochs * k_e2e / float(dt.item()), "unit": unit,
+               "h2d_bytes_per_step": int(Ah.numel() * 4 + bh.numel() * 4 + xh.numel() * 4),
+               "d2h_bytes_per_step": int(xh.numel() * 4 + 8), "steps": k_e2e, "loss": e2e_loss}
+        del Ah
+
+    # ------------------------------------------------------------------ the oracle beside it
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rows = oracle_sample_rows(w)
+        ws, As, bs, _ = synth.make(args.workload, m=rows)
+        dt, samples, _, _ = run_oracle_pass(ws, As.numpy(), bs.numpy())
+        cpu_baseline = {"value": samples / dt, "unit": unit, "cores": 1, "kind": "oracle",
+                        "sample": f"first {rows} of {w.m} rows of {args.workload}, whole path, all {w.epochs} epochs, "
+                                  f"{dt:.1f} s on one thread of {os.cpu_count()} host cores"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "m": w.m, "n": w.n, "bits": w.bits, "batch": w.batch, "epochs": w.epochs,
+                       "levels": w.levels, "model_bits": w.model_bits, "grad_bits": w.grad_bits, "engine": args.engine,
+                       "l2": "inputs larger than L2 (dense A and both planes are streamed every step)",
+                       "multi_gpu": "replicas only"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+            "cpu_baseline": cpu_baseline, "final_loss": final_loss,
+            "packed_gb_per_s_per_epoch": achieved,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

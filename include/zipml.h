@@ -94,6 +94,8 @@ int zipml_destroy(zipml_ctx* ctx);
  * (ZIPML_OK if none), clearing it. */
 int zipml_sync(zipml_ctx* ctx);
 const char* zipml_strerror(int status);
+/* Diagnostics: how many of the library's kernels this context has launched since zipml_create. */
+int64_t zipml_kernel_launches(const zipml_ctx* ctx);
 /* Smallest legal row stride for n features: ceil(n*cb/8) rounded up to 16; 0 if bits is unsupported. */
 int64_t zipml_row_bytes(int64_t n, int32_t bits);
 

@@ -16,7 +16,7 @@ LOSS_DENSE, LOSS_CODES = 0, 1
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT = 0, 1, 2
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host"]
 
 
@@ -58,6 +58,8 @@ def lib():
         L.zipml_create.argtypes = [C.POINTER(vp), C.c_int, vp]
         L.zipml_destroy.argtypes = [vp]
         L.zipml_sync.argtypes = [vp]
+        L.zipml_kernel_launches.argtypes = [vp]
+        L.zipml_kernel_launches.restype = i64
         L.zipml_strerror.argtypes = [C.c_int]
         L.zipml_strerror.restype = C.c_char_p
         L.zipml_row_bytes.argtypes = [i64, i32]
@@ -150,6 +152,9 @@ class Context:
     # --- the calls of include/zipml.h ----------------------------------------------------------
     def zipml_sync(self):
         _check(lib().zipml_sync(self._h), "zipml_sync")
+
+    def zipml_kernel_launches(self):
+        return int(lib().zipml_kernel_launches(self._h))
 
     def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None):
         m, n = A.shape

@@ -24,6 +24,7 @@ struct zipml_ctx {
     // staging buffers of zipml_train_host (grown on demand)
     unsigned char* stage = nullptr;
     size_t stage_bytes = 0;
+    int64_t launches = 0;           // kernels launched so far (diagnostics)
 };
 
 namespace zipml {

@@ -60,6 +60,7 @@ int launch_histogram(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64
     if (chunks > 65535) { rows_per_block = (m + 65534) / 65535; chunks = (m + rows_per_block - 1) / rows_per_block; }
     histogram_kernel<<<dim3((unsigned)col_tiles, (unsigned)chunks), dim3(32, 8), smem, ctx->stream>>>(
         A, m, n, lda, bins, rows_per_block, lo, inv, counts);
+    ctx->launches += 1;
     return cuda_status(cudaGetLastError());
 }
 
@@ -149,6 +150,7 @@ int launch_levels_dp(zipml_ctx* ctx, const uint32_t* counts, int64_t n, int bins
     if (n > 0x7fffffffLL) return ZIPML_ERR_WORKSPACE;
     levels_dp_kernel<<<(unsigned)n, kDpThreads, smem, ctx->stream>>>(
         counts, bins, s, lo, hi, levels_out, reinterpret_cast<unsigned long long*>(objective_out));
+    ctx->launches += 1;
     return cuda_status(cudaGetLastError());
 }
 

@@ -110,6 +110,7 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
     if (vec) range_scan_kernel<4><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key, hi_key, ctx->d_status);
     else range_scan_kernel<1><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key, hi_key, ctx->d_status);
     range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, lo_out, hi_out, inv_out, step_out);
+    ctx->launches += 3;
     return cuda_status(cudaGetLastError());
 }
 
@@ -200,6 +201,7 @@ int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_
     else if (cb == 4) { if (table) ZIPML_LAUNCH_Q(4, true); else ZIPML_LAUNCH_Q(4, false); }
     else { ZIPML_LAUNCH_Q(8, false); }
 #undef ZIPML_LAUNCH_Q
+    ctx->launches += 1;
     return cuda_status(cudaGetLastError());
 }
 

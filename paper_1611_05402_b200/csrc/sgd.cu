@@ -605,6 +605,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
             void* params[] = {&last_chunk_args};
             e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kSgdThreads), params, plan.smem, ctx->stream);
             if (e != cudaSuccess) return cuda_status(e);
+            ctx->launches += 1;
         }
         return ZIPML_OK;
     }
@@ -619,6 +620,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
             void* params[] = {&step_args};
             e = cudaLaunchKernel(kernel, dim3((unsigned)G), dim3(kSgdThreads), params, plan.smem, ctx->stream);
             if (e != cudaSuccess) return cuda_status(e);
+            ctx->launches += 1;
         }
     }
     return ZIPML_OK;
@@ -737,6 +739,7 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
     else { ZIPML_LAUNCH_L(8, false); }
 #undef ZIPML_LAUNCH_L
     loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)d->m), loss_out);
+    ctx->launches += 3;
     return cuda_status(cudaGetLastError());
 }
 
@@ -802,6 +805,7 @@ int launch_loss_dense(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int6
     if (vec) loss_dense_kernel<true><<<blocks, 256, 0, ctx->stream>>>(A, m, n, lda, b, x, partials);
     else loss_dense_kernel<false><<<blocks, 256, 0, ctx->stream>>>(A, m, n, lda, b, x, partials);
     loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)m), loss_out);
+    ctx->launches += 2;
     return cuda_status(cudaGetLastError());
 }
 
