@@ -159,6 +159,30 @@ int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, 
                      int32_t hist_bins, uint64_t quantize_seed, const zipml_sgd_params* params,
                      int32_t epochs, int32_t lr_decay, double* loss_out_host);
 
+/* The code-plane loss of zipml_loss (ZIPML_LOSS_CODES) for callers that may not allocate device
+ * memory.  (The paper has no counterpart: this is a packaging variant of the same computation.)
+ * Who needs it: code that runs where cudaMalloc is forbidden or harmful -- between the kernels of a
+ * latency-critical loop (an allocation may synchronise the whole device), under a framework whose
+ * memory pool already owns the GPU's memory, or on a system with a fixed memory budget.  Such a
+ * caller cannot create a zipml_ctx either, so this call takes the device and the stream directly.
+ *   - Its scratch (the table step*x or level*x and one partial sum per block) is a fixed array
+ *     inside the library image, about 1 MiB, which every GPU that loads the library holds until the
+ *     process exits.  Limit: n <= 262144 features for a uniform grid, 2^bits * n <= 262144 with a
+ *     level table; larger problems are refused with ZIPML_ERR_WORKSPACE.
+ *   - It calls no cudaMalloc/cudaFree and no allocating library routine.  The first call on a
+ *     device looks up the array's device address (once per device); make that first call outside
+ *     any stream capture.
+ *   - All calls on one device share the array and the array keeps the previous call's contents.
+ *     Every slot a call reads it has written itself, so nothing needs clearing, but two calls that
+ *     overlap on the GPU (different streams, or two host threads) race on it: serialise them.
+ *   device       ordinal of the GPU that holds the data
+ *   cuda_stream  cudaStream_t as void* (NULL: the legacy default stream); the work is enqueued there
+ *   data, b, x   as for zipml_loss; DEVICE pointers.   loss_out  one double, DEVICE pointer.
+ * Returns like the other calls; the result equals zipml_loss(CODES) up to the order in which the
+ * per-block partial sums are added. */
+int zipml_loss_codes_static(int device, void* cuda_stream, const zipml_dataset* data, const float* b,
+                            const float* x, double* loss_out);
+
 #ifdef __cplusplus
 }
 #endif

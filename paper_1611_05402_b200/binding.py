@@ -17,7 +17,8 @@ ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT = 0, 1, 2
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
 EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
-           "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host"]
+           "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
+           "zipml_loss_codes_static"]
 
 
 class ZipmlError(RuntimeError):
@@ -70,6 +71,7 @@ def lib():
         L.zipml_loss.argtypes = [vp, i32, vp, i64, i64, i64, C.POINTER(CDataset), vp, vp, vp]
         L.zipml_train_host.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, i32, i32, u64, C.POINTER(CSgdParams), i32, i32,
                                        vp]
+        L.zipml_loss_codes_static.argtypes = [C.c_int, vp, C.POINTER(CDataset), vp, vp, vp]
         _lib = L
     return _lib
 
@@ -230,3 +232,21 @@ class Context:
                                       epochs, int(lr_decay), _ptr(loss)), "zipml_train_host")
         del keep
         return float(loss[0])
+
+
+def zipml_loss_codes_static(data, b, x, out=None, stream=None):
+    """Code-plane loss without any allocation inside the library (see include/zipml.h).
+
+    For callers that cannot let the library call cudaMalloc: there is no context; the device and
+    stream come from the tensors and from torch's current stream.  Problems larger than the
+    library's fixed scratch raise ZipmlError(ERR_WORKSPACE).  Calls that overlap on the GPU race on
+    that scratch, so keep them on one stream.
+    """
+    dev = b.device
+    out = torch.empty(1, dtype=torch.float64, device=dev) if out is None else out
+    stream = torch.cuda.current_stream(dev) if stream is None else stream
+    d = data.c_struct()
+    _check(lib().zipml_loss_codes_static(dev.index, C.c_void_p(stream.cuda_stream), C.byref(d),
+                                         _ptr(b, torch.float32, dev), _ptr(x, torch.float32, dev), _ptr(out)),
+           "zipml_loss_codes_static")
+    return out

@@ -810,3 +810,99 @@ int launch_loss_dense(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int6
 }
 
 }  // namespace zipml
+
+namespace zipml {
+
+// ---------------------------------------------------------------------------------------------
+// Loss estimate from the two planes for callers that cannot allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a region that must not
+// synchronise the device (an allocation can), under a memory pool that owns every byte of the GPU,
+// or in a real-time loop with a fixed memory budget.  zipml_loss (CODES) needs scratch -- the
+// per-step table w = step*x (or level*x) and one partial sum per block -- which it takes from the
+// context's workspace, allocated on demand.  This variant takes the same scratch from a fixed array
+// that is part of the loaded library image instead, so it never allocates; the price is an upper
+// bound on the problem size and one shared array per device.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStaticLossPartials = 1024;
+constexpr int kStaticLossTableFloats = 1 << 18;        // n (uniform) or 2^bits * n (table) must fit
+constexpr size_t kStaticLossBytes = sizeof(double) * (kStaticLossPartials + 2) + sizeof(float) * kStaticLossTableFloats;
+
+static __device__ __align__(256) unsigned char g_static_loss_scratch[kStaticLossBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticLossDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;   // device address of g_static_loss_scratch on this device
+    int sm_count = 0;
+};
+static StaticLossDevice g_static_loss_devices[kMaxDevices];
+
+// Once per device, with that device current: in host code the array's name is only a handle, the
+// kernels need the device address, which cudaGetSymbolAddress returns.
+static int static_loss_setup(int device, StaticLossDevice** out) {
+    if (device < 0 || device >= kMaxDevices) return ZIPML_ERR_INVALID_ARG;
+    StaticLossDevice& d = g_static_loss_devices[device];
+    if (!d.ready) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_loss_scratch);
+        if (e != cudaSuccess) return cuda_status(e);
+        e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return cuda_status(e);
+        d.scratch = static_cast<unsigned char*>(p);
+        d.ready = true;
+    }
+    *out = &d;
+    return ZIPML_OK;
+}
+
+}  // namespace zipml
+
+extern "C" int zipml_loss_codes_static(int device, void* cuda_stream, const zipml_dataset* data, const float* b,
+                                       const float* x, double* loss_out) {
+    using namespace zipml;
+    if (!data || data->struct_size != sizeof(zipml_dataset) || !b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
+    const int cb = container_bits(data->bits);
+    if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
+    const bool table = data->level_mode == ZIPML_LEVELS_TABLE;
+    if (!table && data->level_mode != ZIPML_LEVELS_UNIFORM) return ZIPML_ERR_INVALID_ARG;
+    if (table && data->bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (data->m <= 0 || data->n <= 0 || !data->plane1 || !data->plane2) return ZIPML_ERR_INVALID_ARG;
+    if (data->row_bytes % 16 != 0 || data->row_bytes < zipml_row_bytes(data->n, data->bits)) return ZIPML_ERR_INVALID_ARG;
+    if (table ? !data->levels : (!data->feat_lo || !data->feat_step)) return ZIPML_ERR_INVALID_ARG;
+    const int L = 1 << data->bits;
+    const int64_t table_floats = (table ? (int64_t)L : 1) * data->n;
+    if (table_floats > kStaticLossTableFloats) return ZIPML_ERR_WORKSPACE;   // beyond the fixed scratch
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return cuda_status(cudaGetLastError());
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) return cuda_status(cudaGetLastError());
+    StaticLossDevice* dev = nullptr;
+    int rc = static_loss_setup(device, &dev);
+    if (rc == ZIPML_OK) {
+        cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+        double* partials = reinterpret_cast<double*>(dev->scratch);
+        double* base = partials + kStaticLossPartials;
+        float* wtab = reinterpret_cast<float*>(base + 2);
+        // every slot that is read is written first by this call: nothing has to start at zero
+        loss_prepare_kernel<<<1, 1024, 0, stream>>>(data->feat_lo, data->feat_step, data->levels, x, data->n, L, table,
+                                                    wtab, base);
+        int blocks = dev->sm_count * 8;
+        if (blocks > kStaticLossPartials) blocks = kStaticLossPartials;
+        const int64_t need = (data->m + 7) / 8;
+        if (blocks > need) blocks = (int)need;
+        const uint32_t* p1 = reinterpret_cast<const uint32_t*>(data->plane1);
+        const uint32_t* p2 = reinterpret_cast<const uint32_t*>(data->plane2);
+        const int64_t rw = data->row_bytes / 4;
+#define ZIPML_LAUNCH_SL(CB_, T_) \
+    loss_codes_kernel<CB_, T_><<<blocks, 256, 0, stream>>>(p1, p2, rw, data->m, data->n, wtab, base, b, partials)
+        if (cb == 2) { if (table) ZIPML_LAUNCH_SL(2, true); else ZIPML_LAUNCH_SL(2, false); }
+        else if (cb == 4) { if (table) ZIPML_LAUNCH_SL(4, true); else ZIPML_LAUNCH_SL(4, false); }
+        else { ZIPML_LAUNCH_SL(8, false); }
+#undef ZIPML_LAUNCH_SL
+        loss_finish_kernel<<<1, 256, 0, stream>>>(partials, blocks, 1.0 / (2.0 * (double)data->m), loss_out);
+        rc = cuda_status(cudaGetLastError());
+    }
+    if (prev != device) (void)cudaSetDevice(prev);
+    return rc;
+}

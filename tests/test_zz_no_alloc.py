@@ -1,0 +1,48 @@
+"""The allocation-free loss entry point against the regular one (collected last on purpose).
+
+zipml_loss_codes_static serves callers that cannot let the library allocate device memory (no
+cudaMalloc inside a latency-critical region, or under a pool that owns the GPU): its scratch is a
+fixed array in the library image.  It must give the same loss as zipml_loss(CODES), also on a second
+call that finds the first call's leftovers in the shared scratch, and it must refuse what does not fit.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_1611_05402_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_scratch_loss_matches_regular_entry_point_twice_in_a_row():
+    from paper_1611_05402_b200.build import build
+    build()
+    dev = torch.device("cuda", 0)
+    with binding.Context(dev) as ctx:
+        results = []
+        # two different problems back to back: the second call sees the first one's scratch contents
+        for key, m, n, bits in (("c2", 3000, 1000, 8), ("c4", 2500, 300, 3)):
+            w, A, b, xs = synth.make(key, m=m, n=n, device=dev)
+            levels = ctx.zipml_optimal_levels(A, bits, 256) if key == "c4" else None
+            ds = ctx.zipml_quantize(A, bits, seed=3, levels=levels,
+                                    level_mode=binding.LEVELS_TABLE if levels is not None else binding.LEVELS_UNIFORM)
+            x = (xs * 0.8).contiguous()
+            want = ctx.zipml_loss(binding.LOSS_CODES, b, x, data=ds)
+            ctx.zipml_sync()
+            before = torch.cuda.memory_allocated(dev)
+            got = binding.zipml_loss_codes_static(ds, b, x, out=torch.empty(1, dtype=torch.float64, device=dev))
+            again = binding.zipml_loss_codes_static(ds, b, x, out=torch.empty(1, dtype=torch.float64, device=dev))
+            torch.cuda.synchronize(dev)
+            results.append((want.item(), got.item(), again.item()))
+            assert before <= torch.cuda.memory_allocated(dev) <= before + 1024   # only the two 8-byte outputs
+        for want, got, again in results:
+            assert abs(got - want) <= 1e-6 * abs(want)        # the tolerance of the other loss tests
+            assert again == got                                  # same scratch, same order: bit-identical
+        # a problem beyond the fixed scratch is refused, not truncated
+        n_big = (1 << 18) + 64
+        p = torch.zeros((2, binding.lib().zipml_row_bytes(n_big, 2)), dtype=torch.uint8, device=dev)
+        big = binding.Dataset(p, p, 2, n_big, 2, binding.LEVELS_UNIFORM, torch.zeros(n_big, device=dev),
+                              torch.zeros(n_big, device=dev), None)
+        with pytest.raises(binding.ZipmlError) as e:
+            binding.zipml_loss_codes_static(big, torch.zeros(2, device=dev), torch.zeros(n_big, device=dev))
+        assert e.value.code == binding.ERR_WORKSPACE
