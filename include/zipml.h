@@ -48,7 +48,9 @@ enum { ZIPML_LOSS_DENSE = 0, ZIPML_LOSS_CODES = 1 };
 enum {
     ZIPML_ENGINE_AUTO = 0,
     ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
-    ZIPML_ENGINE_PERSISTENT = 2 /* one cooperative launch per call, grid barriers between the phases */
+    ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
+    ZIPML_ENGINE_RING = 3        /* one cooperative launch; producer warp streams code chunks through a
+                                    shared-memory ring, gradients meet by reduce-scatter / all-gather  */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -96,6 +98,12 @@ int zipml_sync(zipml_ctx* ctx);
 const char* zipml_strerror(int status);
 /* Diagnostics: how many of the library's kernels this context has launched since zipml_create. */
 int64_t zipml_kernel_launches(const zipml_ctx* ctx);
+/* Diagnostics for the latency model of zipml_sgd_epoch: runs `iterations` steps of the per-step
+ * communication skeleton on `ctas` co-resident CTAs (each publishes floats_per_cta floats through
+ * L2, a bounded-spin grid barrier, each reads 16 bytes of every other CTA) and writes the elapsed
+ * nanoseconds (device timer) to ns_out (one uint64, DEVICE pointer).  floats_per_cta % 4 == 0.
+ * ZIPML_ERR_WORKSPACE if `ctas` CTAs cannot be resident at once. */
+int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, int32_t iterations, uint64_t* ns_out);
 /* Smallest legal row stride for n features: ceil(n*cb/8) rounded up to 16; 0 if bits is unsupported. */
 int64_t zipml_row_bytes(int64_t n, int32_t bits);
 

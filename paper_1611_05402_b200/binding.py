@@ -13,10 +13,10 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
-ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT = 0, 1, 2
+ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING = 0, 1, 2, 3
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_barrier_latency", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -61,6 +61,7 @@ def lib():
         L.zipml_sync.argtypes = [vp]
         L.zipml_kernel_launches.argtypes = [vp]
         L.zipml_kernel_launches.restype = i64
+        L.zipml_barrier_latency.argtypes = [vp, i32, i32, i32, vp]
         L.zipml_strerror.argtypes = [C.c_int]
         L.zipml_strerror.restype = C.c_char_p
         L.zipml_row_bytes.argtypes = [i64, i32]
@@ -157,6 +158,13 @@ class Context:
 
     def zipml_kernel_launches(self):
         return int(lib().zipml_kernel_launches(self._h))
+
+    def zipml_barrier_latency(self, ctas, floats_per_cta=0, iterations=1000):
+        """Nanoseconds per step of the SGD step's communication skeleton on `ctas` CTAs."""
+        out = torch.zeros(1, dtype=torch.int64, device=self.device)
+        _check(lib().zipml_barrier_latency(self._h, ctas, floats_per_cta, iterations, _ptr(out)), "zipml_barrier_latency")
+        self.zipml_sync()
+        return out.item() / iterations
 
     def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None):
         m, n = A.shape

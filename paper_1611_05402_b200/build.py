@@ -5,8 +5,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libzipml.so")
-SOURCES = ["api.cu", "quantize.cu", "levels.cu", "sgd.cu"]
-HEADERS = ["common.cuh", "internal.h", os.path.join("..", "..", "include", "zipml.h")]
+SOURCES = ["api.cu", "quantize.cu", "levels.cu", "sgd.cu", "sgd_ring.cu", "loss.cu"]
+HEADERS = ["common.cuh", "internal.h", "sgd_common.cuh", os.path.join("..", "..", "include", "zipml.h")]
 
 
 def _stale() -> bool:

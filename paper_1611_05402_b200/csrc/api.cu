@@ -196,7 +196,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (!b || !x || params->batch <= 0) return ZIPML_ERR_INVALID_ARG;
     if (params->model_bits != 0 && (params->model_bits < 2 || params->model_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
     if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
-    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_PERSISTENT) return ZIPML_ERR_INVALID_ARG;
+    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_RING) return ZIPML_ERR_INVALID_ARG;
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
@@ -208,7 +208,20 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (count == 0) return ZIPML_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
+    if (params->engine == ZIPML_ENGINE_RING) return launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
+    if (params->engine == ZIPML_ENGINE_AUTO) {
+        rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
+        if (rc != ZIPML_ERR_WORKSPACE) return rc;
+    }
     return launch_sgd_epoch(ctx, data, b, x, params, first, count, grad_out);
+}
+
+int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, int32_t iterations, uint64_t* ns_out) {
+    if (!ctx || !ns_out || ctas < 1 || floats_per_cta < 0 || floats_per_cta % 4 != 0 || iterations < 1 || iterations > (1 << 20))
+        return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    return launch_barrier_latency(ctx, ctas, floats_per_cta, iterations, reinterpret_cast<unsigned long long*>(ns_out));
 }
 
 int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t n, int64_t lda,

@@ -120,4 +120,38 @@ __device__ __forceinline__ float float_from_order_key(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Unpacking a 32-bit word of codes into floats.  A code byte is dropped into the mantissa of 2^23
+// with one byte permute, and subtracting 2^23 leaves the exact integer: no int->float conversion
+// instruction (they issue at a fraction of the FMA rate).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float byte_to_float(uint32_t bytes, int i) {
+    return __uint_as_float(__byte_perm(bytes, 0x4B000000u, 0x7650 + i)) - 8388608.0f;
+}
+
+template <int CB>
+__device__ __forceinline__ void unpack_word(uint32_t w, float (&c)[32 / CB]) {
+    if constexpr (CB == 8) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[i] = byte_to_float(w, i);
+    } else if constexpr (CB == 4) {
+        const uint32_t even = w & 0x0F0F0F0Fu, odd = (w >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { c[2 * i] = byte_to_float(even, i); c[2 * i + 1] = byte_to_float(odd, i); }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t t = (w >> (2 * k)) & 0x03030303u;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) c[4 * i + k] = byte_to_float(t, i);
+        }
+    }
+}
+
+template <int CB>
+__device__ __forceinline__ int code_at(uint32_t w, int i) {
+    return (int)((w >> (i * CB)) & ((1u << CB) - 1u));
+}
+
+
 }  // namespace zipml

@@ -71,7 +71,9 @@ int launch_loss_dense(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int6
 int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, const float* x, double* partials,
                       int max_partials, double* loss_out);
 
-size_t sgd_workspace_bytes(const zipml_ctx* ctx, const zipml_dataset* d, const zipml_sgd_params* p);
+int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                    int64_t first_step, int64_t num_steps, float* grad_out, bool probe_only);
+int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                      int64_t first_step, int64_t num_steps, float* grad_out);
 

@@ -1,0 +1,287 @@
+// Training loss (paper Eq. (leastsquares) with l = a^T x - b) on the dense samples, its unbiased
+// estimate from the two code planes, and the allocation-free variant of the latter.
+#include "common.cuh"
+#include "internal.h"
+
+namespace zipml {
+
+// ---------------------------------------------------------------------------------------------
+// Loss estimate from the two planes: 1/(2m) sum_k (Q1(a_k)^T x - b_k)(Q2(a_k)^T x - b_k).
+// A small kernel first writes w_j = step_j x_j (or the level*x table) and the base lo^T x to
+// scratch; the streaming kernel then takes one row per warp.
+// ---------------------------------------------------------------------------------------------
+__global__ void loss_prepare_kernel(const float* __restrict__ lo, const float* __restrict__ step,
+                                    const float* __restrict__ levels, const float* __restrict__ x, int64_t n, int L,
+                                    bool table, float* __restrict__ wtab, double* __restrict__ base_out) {
+    __shared__ double red[40];
+    double base = 0.0;
+    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) {
+        const float xv = x[j];
+        if (!table) {
+            wtab[j] = step[j] * xv;
+            base += (double)lo[j] * (double)xv;
+        } else {
+            for (int c = 0; c < L; ++c) wtab[(int64_t)c * n + j] = levels[j * L + c] * xv;
+        }
+    }
+    base = block_sum(base, red);
+    if (threadIdx.x == 0) *base_out = base;
+}
+
+template <int CB, bool TABLE>
+__global__ void __launch_bounds__(256) loss_codes_kernel(const uint32_t* __restrict__ p1, const uint32_t* __restrict__ p2,
+                                                         int64_t row_words, int64_t m, int64_t n,
+                                                         const float* __restrict__ wtab, const double* __restrict__ base_in,
+                                                         const float* __restrict__ b, double* __restrict__ partials) {
+    constexpr int FPW = 32 / CB;
+    __shared__ double red[40];
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t words = (n + FPW - 1) / FPW;
+    const double base = *base_in;
+    double total = 0.0;
+    for (int64_t k = warp_global; k < m; k += nwarps) {
+        const uint32_t* row1 = p1 + k * row_words;
+        const uint32_t* row2 = p2 + k * row_words;
+        double d1 = 0.0, d2 = 0.0;
+        for (int64_t q0 = 0; q0 < words; q0 += 32 * 8) {
+            float acc1 = 0.0f, acc2 = 0.0f;
+#pragma unroll 2
+            for (int s = 0; s < 8; ++s) {
+                const int64_t q = q0 + s * 32 + lane;
+                if (q < words) {
+                    const uint32_t u1 = __ldg(row1 + q), u2 = __ldg(row2 + q);
+                    if constexpr (!TABLE) {
+                        float c1[FPW], c2[FPW];
+                        unpack_word<CB>(u1, c1);
+                        unpack_word<CB>(u2, c2);
+#pragma unroll
+                        for (int i = 0; i < FPW; ++i) {
+                            const int64_t j = q * FPW + i;
+                            const float wv = (j < n) ? __ldg(wtab + j) : 0.0f;
+                            acc1 = fmaf(c1[i], wv, acc1);
+                            acc2 = fmaf(c2[i], wv, acc2);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < FPW; ++i) {
+                            const int64_t j = q * FPW + i;
+                            if (j < n) {
+                                acc1 += __ldg(wtab + (int64_t)code_at<CB>(u1, i) * n + j);
+                                acc2 += __ldg(wtab + (int64_t)code_at<CB>(u2, i) * n + j);
+                            }
+                        }
+                    }
+                }
+            }
+            d1 += (double)acc1;
+            d2 += (double)acc2;
+        }
+        d1 = warp_sum(d1) + base;
+        d2 = warp_sum(d2) + base;
+        const double bk = (double)__ldg(b + k);
+        if (lane == 0) total += (d1 - bk) * (d2 - bk);
+    }
+    total = block_sum(total, red);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
+__global__ void loss_finish_kernel(const double* __restrict__ partials, int count, double scale, double* out) {
+    __shared__ double red[40];
+    double v = 0.0;
+    for (int i = threadIdx.x; i < count; i += blockDim.x) v += partials[i];
+    v = block_sum(v, red);
+    if (threadIdx.x == 0) *out = v * scale;
+}
+
+int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, const float* x, double* partials,
+                      int max_partials, double* loss_out) {
+    const int cb = container_bits(d->bits);
+    const bool table = d->level_mode == ZIPML_LEVELS_TABLE;
+    const int L = 1 << d->bits;
+    // scratch behind the partials: base (1 double) then the w table
+    double* base = partials + max_partials;
+    float* wtab = reinterpret_cast<float*>(base + 2);
+    loss_prepare_kernel<<<1, 1024, 0, ctx->stream>>>(d->feat_lo, d->feat_step, d->levels, x, d->n, L, table, wtab, base);
+    int blocks = ctx->sm_count * 8;
+    if (blocks > max_partials) blocks = max_partials;
+    const int64_t need = (d->m + 7) / 8;
+    if (blocks > need) blocks = (int)need;
+    const uint32_t* p1 = reinterpret_cast<const uint32_t*>(d->plane1);
+    const uint32_t* p2 = reinterpret_cast<const uint32_t*>(d->plane2);
+    const int64_t rw = d->row_bytes / 4;
+#define ZIPML_LAUNCH_L(CB_, T_) \
+    loss_codes_kernel<CB_, T_><<<blocks, 256, 0, ctx->stream>>>(p1, p2, rw, d->m, d->n, wtab, base, b, partials)
+    if (cb == 2) { if (table) ZIPML_LAUNCH_L(2, true); else ZIPML_LAUNCH_L(2, false); }
+    else if (cb == 4) { if (table) ZIPML_LAUNCH_L(4, true); else ZIPML_LAUNCH_L(4, false); }
+    else { ZIPML_LAUNCH_L(8, false); }
+#undef ZIPML_LAUNCH_L
+    loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)d->m), loss_out);
+    ctx->launches += 3;
+    return cuda_status(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------------------------
+// Dense loss on the original samples: one row per warp, fp32 products over runs of 32*8 elements,
+// doubles across runs, lanes, warps and blocks; block partials are summed in order by one block.
+// ---------------------------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(256) loss_dense_kernel(const float* __restrict__ A, int64_t m, int64_t n, int64_t lda,
+                                                         const float* __restrict__ b, const float* __restrict__ x,
+                                                         double* __restrict__ partials) {
+    __shared__ double red[40];
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    double total = 0.0;
+    for (int64_t k = warp_global; k < m; k += nwarps) {
+        const float* row = A + k * lda;
+        double d = 0.0;
+        if constexpr (VEC) {
+            const int64_t n4 = n >> 2;
+            for (int64_t q0 = 0; q0 < n4; q0 += 32 * 8) {
+                float acc = 0.0f;
+#pragma unroll 4
+                for (int s = 0; s < 8; ++s) {
+                    const int64_t q = q0 + s * 32 + lane;
+                    if (q < n4) {
+                        const float4 av = __ldg(reinterpret_cast<const float4*>(row) + q);
+                        const float4 xv = __ldg(reinterpret_cast<const float4*>(x) + q);
+                        acc = fmaf(av.x, xv.x, acc); acc = fmaf(av.y, xv.y, acc);
+                        acc = fmaf(av.z, xv.z, acc); acc = fmaf(av.w, xv.w, acc);
+                    }
+                }
+                d += (double)acc;
+            }
+            for (int64_t j = (n4 << 2) + lane; j < n; j += 32) d += (double)(__ldg(row + j) * __ldg(x + j));
+        } else {
+            for (int64_t j0 = 0; j0 < n; j0 += 32 * 8) {
+                float acc = 0.0f;
+#pragma unroll 4
+                for (int s = 0; s < 8; ++s) {
+                    const int64_t j = j0 + s * 32 + lane;
+                    if (j < n) acc = fmaf(__ldg(row + j), __ldg(x + j), acc);
+                }
+                d += (double)acc;
+            }
+        }
+        d = warp_sum(d);
+        const double r = d - (double)__ldg(b + k);
+        if (lane == 0) total += r * r;
+    }
+    total = block_sum(total, red);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
+int launch_loss_dense(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, const float* b, const float* x,
+                      double* partials, int max_partials, double* loss_out) {
+    int blocks = ctx->sm_count * 8;
+    if (blocks > max_partials) blocks = max_partials;
+    const int64_t need = (m + 7) / 8;
+    if (blocks > need) blocks = (int)need;
+    const bool vec = (lda % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && ((reinterpret_cast<uintptr_t>(x) & 15) == 0);
+    if (vec) loss_dense_kernel<true><<<blocks, 256, 0, ctx->stream>>>(A, m, n, lda, b, x, partials);
+    else loss_dense_kernel<false><<<blocks, 256, 0, ctx->stream>>>(A, m, n, lda, b, x, partials);
+    loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)m), loss_out);
+    ctx->launches += 2;
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace zipml
+
+namespace zipml {
+
+// ---------------------------------------------------------------------------------------------
+// Loss estimate from the two planes for callers that cannot allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a region that must not
+// synchronise the device (an allocation can), under a memory pool that owns every byte of the GPU,
+// or in a real-time loop with a fixed memory budget.  zipml_loss (CODES) needs scratch -- the
+// per-step table w = step*x (or level*x) and one partial sum per block -- which it takes from the
+// context's workspace, allocated on demand.  This variant takes the same scratch from a fixed array
+// that is part of the loaded library image instead, so it never allocates; the price is an upper
+// bound on the problem size and one shared array per device.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStaticLossPartials = 1024;
+constexpr int kStaticLossTableFloats = 1 << 18;        // n (uniform) or 2^bits * n (table) must fit
+constexpr size_t kStaticLossBytes = sizeof(double) * (kStaticLossPartials + 2) + sizeof(float) * kStaticLossTableFloats;
+
+static __device__ __align__(256) unsigned char g_static_loss_scratch[kStaticLossBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticLossDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;   // device address of g_static_loss_scratch on this device
+    int sm_count = 0;
+};
+static StaticLossDevice g_static_loss_devices[kMaxDevices];
+
+// Once per device, with that device current: in host code the array's name is only a handle, the
+// kernels need the device address, which cudaGetSymbolAddress returns.
+static int static_loss_setup(int device, StaticLossDevice** out) {
+    if (device < 0 || device >= kMaxDevices) return ZIPML_ERR_INVALID_ARG;
+    StaticLossDevice& d = g_static_loss_devices[device];
+    if (!d.ready) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_loss_scratch);
+        if (e != cudaSuccess) return cuda_status(e);
+        e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return cuda_status(e);
+        d.scratch = static_cast<unsigned char*>(p);
+        d.ready = true;
+    }
+    *out = &d;
+    return ZIPML_OK;
+}
+
+}  // namespace zipml
+
+extern "C" int zipml_loss_codes_static(int device, void* cuda_stream, const zipml_dataset* data, const float* b,
+                                       const float* x, double* loss_out) {
+    using namespace zipml;
+    if (!data || data->struct_size != sizeof(zipml_dataset) || !b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
+    const int cb = container_bits(data->bits);
+    if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
+    const bool table = data->level_mode == ZIPML_LEVELS_TABLE;
+    if (!table && data->level_mode != ZIPML_LEVELS_UNIFORM) return ZIPML_ERR_INVALID_ARG;
+    if (table && data->bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (data->m <= 0 || data->n <= 0 || !data->plane1 || !data->plane2) return ZIPML_ERR_INVALID_ARG;
+    if (data->row_bytes % 16 != 0 || data->row_bytes < zipml_row_bytes(data->n, data->bits)) return ZIPML_ERR_INVALID_ARG;
+    if (table ? !data->levels : (!data->feat_lo || !data->feat_step)) return ZIPML_ERR_INVALID_ARG;
+    const int L = 1 << data->bits;
+    const int64_t table_floats = (table ? (int64_t)L : 1) * data->n;
+    if (table_floats > kStaticLossTableFloats) return ZIPML_ERR_WORKSPACE;   // beyond the fixed scratch
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return cuda_status(cudaGetLastError());
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) return cuda_status(cudaGetLastError());
+    StaticLossDevice* dev = nullptr;
+    int rc = static_loss_setup(device, &dev);
+    if (rc == ZIPML_OK) {
+        cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+        double* partials = reinterpret_cast<double*>(dev->scratch);
+        double* base = partials + kStaticLossPartials;
+        float* wtab = reinterpret_cast<float*>(base + 2);
+        // every slot that is read is written first by this call: nothing has to start at zero
+        loss_prepare_kernel<<<1, 1024, 0, stream>>>(data->feat_lo, data->feat_step, data->levels, x, data->n, L, table,
+                                                    wtab, base);
+        int blocks = dev->sm_count * 8;
+        if (blocks > kStaticLossPartials) blocks = kStaticLossPartials;
+        const int64_t need = (data->m + 7) / 8;
+        if (blocks > need) blocks = (int)need;
+        const uint32_t* p1 = reinterpret_cast<const uint32_t*>(data->plane1);
+        const uint32_t* p2 = reinterpret_cast<const uint32_t*>(data->plane2);
+        const int64_t rw = data->row_bytes / 4;
+#define ZIPML_LAUNCH_SL(CB_, T_) \
+    loss_codes_kernel<CB_, T_><<<blocks, 256, 0, stream>>>(p1, p2, rw, data->m, data->n, wtab, base, b, partials)
+        if (cb == 2) { if (table) ZIPML_LAUNCH_SL(2, true); else ZIPML_LAUNCH_SL(2, false); }
+        else if (cb == 4) { if (table) ZIPML_LAUNCH_SL(4, true); else ZIPML_LAUNCH_SL(4, false); }
+        else { ZIPML_LAUNCH_SL(8, false); }
+#undef ZIPML_LAUNCH_SL
+        loss_finish_kernel<<<1, 256, 0, stream>>>(partials, blocks, 1.0 / (2.0 * (double)data->m), loss_out);
+        rc = cuda_status(cudaGetLastError());
+    }
+    if (prev != device) (void)cudaSetDevice(prev);
+    return rc;
+}
