@@ -39,8 +39,11 @@ struct SgdArgs {
     int stages;             // shared-memory stages of the code ring (STAGED kernels)
     int cr;                 // ring engine: rows per chunk (one ring slot holds cr rows of both planes)
     int sub;                // ring engine: features of a part that one row-part CTA reduces and updates
-    float* xg;              // ring engine: [na*wc*FPW] model published by the owners of each sub-slice
-    double* gn;             // ring engine: [2][G] partial squared norms (gradient, model)
+    // ring engine: exchange buffers of 8-byte packets {fp32 value, step tag}, zeroed before a launch
+    unsigned long long* ll_pd;   // [2][nb][na][rc][4]   partial dots (hi, lo of two doubles); only na > 1
+    unsigned long long* ll_rs;   // [na][nb][nb][sub+2]  partial gradients per (owner, writer) + residual sum
+    unsigned long long* ll_gn;   // [2][G][2]            partial squared gradient norms (hi, lo)
+    unsigned long long* ll_ag;   // [na*wc*FPW] new model, then [G][2] partial squared model norms
     double* pd;             // [2][na][batch][2]   partial dots
     float* pg;              // [2][nb][na*wc*FPW]  partial code gradients (table mode: value gradients)
     double* ps;             // [2][nb]             partial sums of r1 + r2

@@ -11,14 +11,21 @@
 //     the model, so the producer runs ahead across phases and steps as far as the ring allows and
 //     HBM latency never sits on the step-to-step dependency chain;
 //   * consumers wait for a slot, compute on it and hand it back (one arrival per consumer warp).
-// Per step:  phase A dots -> residuals (through pd and a grid barrier if na > 1);
-//            phase B partial gradients of the CTA's rows -> pg, ps; grid barrier;
-//            reduce-scatter: CTA (ai, bi) sums the nb row parts of its own sub-slice of feature
-//            part ai in a fixed order, applies the optional gradient quantizer (one more barrier
-//            for the norm) and the update, and publishes the new sub-slice; grid barrier;
-//            all-gather: every CTA reads the new model of its feature part.
+// Per step:  phase A dots -> residuals (with na > 1 the partial dots of a row meet first);
+//            phase B partial gradients of the CTA's rows;
+//            reduce-scatter: CTA (ai, bi) collects the nb row parts of its own sub-slice of feature
+//            part ai, sums them in a fixed order, applies the optional gradient quantizer (one more
+//            exchange for the norm) and the update, and publishes the new sub-slice;
+//            all-gather: every CTA collects the new model of its feature part.
+// Exchange.  Nothing here uses a grid barrier.  Every exchanged number travels as an 8-byte packet
+// {fp32 value, step tag} written with one 64-bit store; a reader polls the packet until the tag is
+// the current step's, so the data announces itself and one L2 round trip replaces "write, fence,
+// count arrivals, poll the counter, read".  Buffers are zeroed before a launch and tags start at 1.
+// A packet of step t is overwritten only by a CTA that has already collected everything of step t
+// that depends on its readers, so single buffers suffice; the two exchanges that couple CTAs of
+// different feature parts (dots, gradient norm) alternate between two buffers by step parity.
 // Every wait is bounded: when one gives up it records ZIPML_ERR_TIMEOUT, later waits of that CTA
-// are skipped and the CTA still arrives at every barrier, so the launch always ends.
+// are skipped and the CTA still publishes everything, so the launch always ends.
 #include "sgd_common.cuh"
 
 namespace zipml {
@@ -62,38 +69,60 @@ __device__ __forceinline__ void ring_wait(unsigned long long* bar, uint32_t pari
     set_status(status, ZIPML_ERR_TIMEOUT, where);
 }
 
-// Grid barrier among the consumers of all CTAs (the producer warps do not take part).
-__device__ __forceinline__ void ring_grid_barrier(unsigned* counter, unsigned target, RingShared* sh, DeviceStatus* status,
-                                                  int where) {
-    consumer_sync();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(counter, 1u);
-        if (!sh->abort_flag) {
-            bool ok = false;
-            for (long long it = 0; it < kBarrierSpinLimit; ++it) {
-                unsigned v;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-                if (v >= target) { ok = true; break; }
-                if ((it & 1023) == 1023) {
-                    if (*reinterpret_cast<volatile int*>(&status->code) != 0) break;
-                    __nanosleep(200);
+// ---- packets ---------------------------------------------------------------------------------
+__device__ __forceinline__ void ll_store(unsigned long long* p, float v, uint32_t tag) {
+    __stcg(p, ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(v));
+}
+__device__ __forceinline__ void ll_store_double(unsigned long long* p, double v, uint32_t tag) {
+    const float hi = (float)v;
+    ll_store(p, hi, tag);
+    ll_store(p + 1, (float)(v - (double)hi), tag);
+}
+__device__ __forceinline__ unsigned long long ll_load(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+constexpr long long kPacketSpinLimit = 1ll << 22;
+
+// Collects `count` contiguous packets of the current step into dst (shared memory), the consumer
+// threads taking them four at a time so that their loads are in flight together.
+__device__ __forceinline__ void ll_gather(const unsigned long long* src, int count, uint32_t tag, float* dst,
+                                          RingShared* sh, DeviceStatus* status, int where) {
+    for (int i0 = threadIdx.x; i0 < count; i0 += 4 * kRingConsumers) {
+        unsigned long long v[4];
+        bool ok = false;
+        if (!*reinterpret_cast<volatile int*>(&sh->abort_flag)) {
+            for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
+                ok = true;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * kRingConsumers;
+                    if (i < count) { v[u] = ll_load(src + i); ok = ok && ((uint32_t)(v[u] >> 32) == tag); }
                 }
             }
             if (!ok) { sh->abort_flag = 1; set_status(status, ZIPML_ERR_TIMEOUT, where); }
         }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * kRingConsumers;
+            if (i < count) dst[i] = ok ? __uint_as_float((uint32_t)v[u]) : 0.0f;
+        }
     }
-    consumer_sync();
 }
 
 // Shared memory plan, F = wc * FPW features per CTA:
 //   RingShared
-//   xs[F] float                model of the CTA's feature part
-//   tab float                  uniform: w[F] ([u][word][4]); table: WL[L*F] then LV[L*F] ([code][slot][word])
-//   gsub[sub] float            gradient of the CTA's own sub-slice
-//   gred[kRingConsumers*FPW]   cross-group reduction of phase B
-//   res[2*rc] float            residuals
-//   ring[slots][2][cr][wc] u32 code chunks
+//   xs[F] float                 model of the CTA's feature part
+//   tab float                   uniform: w[F] ([u][word][4]); table: WL[L*F] then LV[L*F] ([code][slot][word])
+//   gsub[sub] float             gradient of the CTA's own sub-slice
+//   gbuf[nb*(sub+2)] float      collected row parts of the own sub-slice (+ residual sums)
+//   dsum[sub+2] double          their sums
+//   nbuf[4*G] float             collected partial norms
+//   gred[kRingConsumers*FPW]    cross-group reduction of phase B
+//   res[2*rc] float             residuals
+//   bsm[2][rc] float            labels of the current and the next step's rows
+//   ring[slots][2][cr][wc] u32  code chunks
 template <int CB, bool TABLE>
 __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a) {
     constexpr int FPW = 32 / CB;
@@ -101,16 +130,21 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     RingShared* sh = reinterpret_cast<RingShared*>(s_raw);
     const int L = 1 << a.bits;
     const int F = a.wc * FPW;
+    const int G = a.na * a.nb;
+    const int subp = a.sub + 2;                                  // packets per (owner, writer)
     float* xs = reinterpret_cast<float*>(s_raw + ((sizeof(RingShared) + 15) & ~(size_t)15));
     float* tab = xs + F;
     float* gsub = tab + (TABLE ? 2 * L * F : F);
-    float* gred = gsub + a.sub;
+    float* gbuf = gsub + a.sub;
+    double* dsum = reinterpret_cast<double*>(gbuf + ((a.nb * subp + 3) & ~3));
+    float* nbuf = reinterpret_cast<float*>(dsum + ((subp + 1) & ~1));
+    float* gred = nbuf + 4 * G;
     float* res = gred + kRingConsumers * FPW;
-    uint32_t* ring = reinterpret_cast<uint32_t*>(res + ((2 * a.rc + 3) & ~3));
+    float* bsm = res + ((2 * a.rc + 3) & ~3);
+    uint32_t* ring = reinterpret_cast<uint32_t*>(bsm + ((2 * a.rc + 3) & ~3));
     const size_t slot_words = (size_t)2 * a.cr * a.wc;
 
     const int ai = blockIdx.x % a.na, bi = blockIdx.x / a.na;
-    const int G = a.na * a.nb;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t words_needed = (a.n + FPW - 1) / FPW;
     const int64_t w0 = (int64_t)ai * a.wc;
@@ -197,6 +231,12 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         for (int64_t j = threadIdx.x; j < a.n; j += kRingConsumers) { const double v = (double)a.x[j]; ss += v * v; }
         xnorm2 = consumer_sum(ss, sh->red);
     }
+    {   // labels of the first step's rows
+        int64_t r0; int bt, rcnt;
+        step_rows(a.first_step, r0, bt, rcnt);
+        float* bcur = bsm + (size_t)(a.first_step & 1) * a.rc;
+        for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) bcur[r] = __ldg(a.b + r0 + k0 + r);
+    }
     consumer_sync();
 
     // step-invariant thread roles
@@ -204,19 +244,25 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     const int ngroups = kRingConsumers / lanes_q;
     const int group = threadIdx.x / lanes_q;
     const int ql = threadIdx.x % lanes_q;
-    const int qpasses = (wcnt + lanes_q - 1) / lanes_q;                      // > 1 only for parts wider than the CTA
     const int sub0 = min(F, bi * a.sub), sub1 = min(F, sub0 + a.sub);        // own sub-slice of the feature part
     const float* LV = tab + L * F;
     const int chunks_w = (wcnt + 31) / 32;
-    unsigned barriers_done = 0;
     int slot = 0;
     uint32_t phase = 0;
+    // where this CTA's packets go and come from
+    unsigned long long* rs_mine = a.ll_rs + (size_t)ai * a.nb * a.nb * subp;                 // + (owner*nb + writer)*subp
+    const unsigned long long* rs_own = rs_mine + (size_t)bi * a.nb * subp;                   // collected by this owner
+    unsigned long long* ag_part = a.ll_ag + j0;
+    unsigned long long* ag_norm = a.ll_ag + npad;
 
     for (int64_t it = a.first_step; it < step_end; ++it) {
         int64_t r0; int bt, rcnt;
         step_rows(it, r0, bt, rcnt);
         const int C = (rcnt + a.cr - 1) / a.cr;
         const bool last = (it == step_end - 1);
+        const uint32_t tag = (uint32_t)(it - a.first_step) + 1u;
+        const int par = (int)(it & 1);
+        const float* bcur = bsm + (size_t)par * a.rc;
 
         // -------------------------------------------------------------- model seen by the step
         VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 3u};
@@ -248,6 +294,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
 
         // -------------------------------------------------------------- phase A: dots
         const bool dots_local = (a.na == 1);
+        unsigned long long* pd_mine = a.ll_pd + (((size_t)par * a.nb + bi) * a.na + ai) * a.rc * 4;
         const int slot_a = slot;                 // slot of the single chunk when C == 1
         for (int chunk = 0; chunk < C; ++chunk) {
             const int rows = min(a.cr, rcnt - chunk * a.cr);
@@ -270,14 +317,14 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
 #pragma unroll
                             for (int u = 0; u < FPW / 4; ++u) {
                                 const float4 wv = *reinterpret_cast<const float4*>(tab + (u * a.wc + q) * 4);
-                                acc1[u & 1] = fmaf(c1[4 * u + 0], wv.x, acc1[u & 1]);
-                                acc1[u & 1] = fmaf(c1[4 * u + 1], wv.y, acc1[u & 1]);
-                                acc1[u & 1] = fmaf(c1[4 * u + 2], wv.z, acc1[u & 1]);
-                                acc1[u & 1] = fmaf(c1[4 * u + 3], wv.w, acc1[u & 1]);
-                                acc2[u & 1] = fmaf(c2[4 * u + 0], wv.x, acc2[u & 1]);
-                                acc2[u & 1] = fmaf(c2[4 * u + 1], wv.y, acc2[u & 1]);
-                                acc2[u & 1] = fmaf(c2[4 * u + 2], wv.z, acc2[u & 1]);
-                                acc2[u & 1] = fmaf(c2[4 * u + 3], wv.w, acc2[u & 1]);
+                                acc1[0] = fmaf(c1[4 * u + 0], wv.x, acc1[0]);
+                                acc1[1] = fmaf(c1[4 * u + 1], wv.y, acc1[1]);
+                                acc1[0] = fmaf(c1[4 * u + 2], wv.z, acc1[0]);
+                                acc1[1] = fmaf(c1[4 * u + 3], wv.w, acc1[1]);
+                                acc2[0] = fmaf(c2[4 * u + 0], wv.x, acc2[0]);
+                                acc2[1] = fmaf(c2[4 * u + 1], wv.y, acc2[1]);
+                                acc2[0] = fmaf(c2[4 * u + 2], wv.z, acc2[0]);
+                                acc2[1] = fmaf(c2[4 * u + 3], wv.w, acc2[1]);
                             }
                         } else {
 #pragma unroll
@@ -293,12 +340,12 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 if (lane == 0) {
                     const int r = chunk * a.cr + lr;
                     if (dots_local) {
-                        const double bk = (double)__ldg(a.b + r0 + k0 + r);
+                        const double bk = (double)bcur[r];
                         res[2 * r] = (float)(d1 - bk);
                         res[2 * r + 1] = (float)(d2 - bk);
                     } else {
-                        __stcg(a.pd + ((size_t)ai * a.batch + k0 + r) * 2 + 0, d1);
-                        __stcg(a.pd + ((size_t)ai * a.batch + k0 + r) * 2 + 1, d2);
+                        ll_store_double(pd_mine + (size_t)r * 4, d1, tag);
+                        ll_store_double(pd_mine + (size_t)r * 4 + 2, d2, tag);
                     }
                 }
             }
@@ -308,37 +355,38 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 if (++slot == slots) { slot = 0; phase ^= 1u; }
             }
         }
-        if (!dots_local) ring_grid_barrier(a.barrier, (unsigned)G * ++barriers_done, sh, a.status, 1);
-        else consumer_sync();
+        if (!dots_local) {
+            // every row's dot is the sum, in part order, of the na partial dots published for it
+            const unsigned long long* pd_row = a.ll_pd + ((size_t)par * a.nb + bi) * a.na * a.rc * 4;
+            for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) {
+                double d1 = 0.0, d2 = 0.0;
+                bool good = !*reinterpret_cast<volatile int*>(&sh->abort_flag);
+                for (int p = 0; p < a.na && good; ++p) {
+                    const unsigned long long* src = pd_row + ((size_t)p * a.rc + r) * 4;
+                    unsigned long long v[4];
+                    bool ok = false;
+                    for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
+                        ok = true;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) { v[u] = ll_load(src + u); ok = ok && ((uint32_t)(v[u] >> 32) == tag); }
+                    }
+                    if (!ok) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 1); good = false; break; }
+                    d1 += (double)__uint_as_float((uint32_t)v[0]) + (double)__uint_as_float((uint32_t)v[1]);
+                    d2 += (double)__uint_as_float((uint32_t)v[2]) + (double)__uint_as_float((uint32_t)v[3]);
+                }
+                const double bk = (double)bcur[r];
+                res[2 * r] = good ? (float)(d1 - bk) : 0.0f;
+                res[2 * r + 1] = good ? (float)(d2 - bk) : 0.0f;
+            }
+        }
+        consumer_sync();                         // residuals are complete
 
         // -------------------------------------------------------------- phase B: gradient
         double ssum = 0.0;
-        for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) {
-            float r1, r2;
-            if (dots_local) {
-                r1 = res[2 * r];
-                r2 = res[2 * r + 1];
-            } else {
-                double d1 = 0.0, d2 = 0.0;
-                for (int p = 0; p < a.na; ++p) {
-                    d1 += __ldcg(a.pd + ((size_t)p * a.batch + k0 + r) * 2 + 0);
-                    d2 += __ldcg(a.pd + ((size_t)p * a.batch + k0 + r) * 2 + 1);
-                }
-                const double bk = (double)__ldg(a.b + r0 + k0 + r);
-                r1 = (float)(d1 - bk);
-                r2 = (float)(d2 - bk);
-                res[2 * r] = r1;
-                res[2 * r + 1] = r2;
-            }
-            ssum += (double)r1 + (double)r2;
-        }
-        ssum = consumer_sum(ssum, sh->red);      // residuals are complete after its barriers
-        if (threadIdx.x == 0 && ai == 0) __stcg(a.ps + bi, ssum);
-
-        // parts wider than the consumer count (qpasses > 1) are planned as one retained chunk (C <= 1),
-        // so the chunk sequence below is walked exactly once whenever chunks are fetched again
-        for (int qp = 0; qp < qpasses; ++qp) {
-            const int q = qp * lanes_q + ql;
+        for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) ssum += (double)res[2 * r] + (double)res[2 * r + 1];
+        ssum = consumer_sum(ssum, sh->red);
+        {
+            const int q = ql;
             const bool active = (group < ngroups) && (q < wcnt);
             float acc[FPW];
 #pragma unroll
@@ -399,9 +447,13 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 }
             }
             if (active && group == 0) {
-                float4* dst = reinterpret_cast<float4*>(a.pg + (size_t)bi * npad + (size_t)(w0 + q) * FPW);
+                // feature f of the part belongs to owner f / sub; its packet sits in that owner's block for this writer
 #pragma unroll
-                for (int u = 0; u < FPW / 4; ++u) __stcg(dst + u, make_float4(acc[4 * u], acc[4 * u + 1], acc[4 * u + 2], acc[4 * u + 3]));
+                for (int i = 0; i < FPW; ++i) {
+                    const int f = q * FPW + i;
+                    const int owner = f / a.sub;
+                    ll_store(rs_mine + ((size_t)owner * a.nb + bi) * subp + (f - owner * a.sub), acc[i], tag);
+                }
             }
         }
         if (C == 1) {                            // the retained single chunk goes back now
@@ -409,86 +461,101 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
             if (++slot == slots) { slot = 0; phase ^= 1u; }
         }
-        ring_grid_barrier(a.barrier, (unsigned)G * ++barriers_done, sh, a.status, 2);
+        // owners also wait for the slots of features past the part's last code word and of their
+        // sub-slice's unused tail: those carry zeros
+        for (int f = wcnt * FPW + threadIdx.x; f < a.nb * a.sub; f += kRingConsumers) {
+            const int owner = f / a.sub;
+            ll_store(rs_mine + ((size_t)owner * a.nb + bi) * subp + (f - owner * a.sub), 0.0f, tag);
+        }
+        // the residual sum goes to every owner of the part, behind the gradient packets
+        for (int o = threadIdx.x; o < a.nb; o += kRingConsumers)
+            ll_store_double(rs_mine + ((size_t)o * a.nb + bi) * subp + a.sub, ssum, tag);
+        // labels of the next step's rows, fetched while the packets travel
+        if (!last) {
+            int64_t r0n; int btn, rcntn;
+            step_rows(it + 1, r0n, btn, rcntn);
+            float* bnext = bsm + (size_t)(par ^ 1) * a.rc;
+            for (int r = threadIdx.x; r < rcntn; r += kRingConsumers) bnext[r] = __ldg(a.b + r0n + k0 + r);
+        }
 
         // -------------------------------------------------------------- reduce-scatter: own sub-slice
-        double stot = 0.0;
-        if constexpr (!TABLE) {
-            double part = 0.0;
-            if (warp == 0) {
-                for (int p = lane; p < a.nb; p += 32) part += __ldcg(a.ps + p);
-                part = warp_sum(part);
+        const int nsub = sub1 - sub0;            // features this CTA owns (may be 0 for the last owners)
+        ll_gather(rs_own, a.nb * subp, tag, gbuf, sh, a.status, 2);
+        consumer_sync();
+        if (a.nb <= 32) {
+            for (int k = threadIdx.x; k < subp; k += kRingConsumers) {
+                double t = 0.0;
+                for (int w = 0; w < a.nb; ++w) t += (double)gbuf[w * subp + k];
+                dsum[k] = t;
             }
-            if (threadIdx.x == 0) sh->misc[0] = part;
-            consumer_sync();
-            stot = sh->misc[0];
+        } else {
+            for (int k = warp; k < subp; k += kRingWarps) {
+                double t = 0.0;
+                for (int w = lane; w < a.nb; w += 32) t += (double)gbuf[w * subp + k];
+                t = warp_sum(t);
+                if (lane == 0) dsum[k] = t;
+            }
         }
+        consumer_sync();
+        const double stot = dsum[a.sub] + dsum[a.sub + 1];
         const double scale = 1.0 / (2.0 * (double)bt);
         double gsq = 0.0;
-        for (int f = sub0 + 4 * threadIdx.x; f < sub1; f += 4 * kRingConsumers) {
-            double acc[4] = {0.0, 0.0, 0.0, 0.0};
-            const float4* src = reinterpret_cast<const float4*>(a.pg + j0 + f);
-#pragma unroll 8
-            for (int p = 0; p < a.nb; ++p) {
-                const float4 v = __ldcg(src + (size_t)p * (npad / 4));
-                acc[0] += (double)v.x; acc[1] += (double)v.y; acc[2] += (double)v.z; acc[3] += (double)v.w;
+        for (int k = threadIdx.x; k < nsub; k += kRingConsumers) {
+            const int f = sub0 + k;
+            float g = 0.0f;
+            if (f < fcnt) {
+                double v = dsum[k];
+                if constexpr (!TABLE) v = (double)__ldg(a.lo + j0 + f) * stot + (double)__ldg(a.step + j0 + f) * v;
+                g = (float)(v * scale);
+                if (last && a.grad_out) a.grad_out[j0 + f] = g;
             }
-            float g[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                g[e] = 0.0f;
-                if (f + e < fcnt) {
-                    double v = acc[e];
-                    if constexpr (!TABLE) v = (double)__ldg(a.lo + j0 + f + e) * stot + (double)__ldg(a.step + j0 + f + e) * v;
-                    g[e] = (float)(v * scale);
-                    if (last && a.grad_out) a.grad_out[j0 + f + e] = g[e];
-                }
-                gsq += (double)g[e] * (double)g[e];
-            }
-            *reinterpret_cast<float4*>(gsub + (f - sub0)) = make_float4(g[0], g[1], g[2], g[3]);
+            gsub[k] = g;
+            gsq += (double)g * (double)g;
         }
         VecQuant q4{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 4u};
         if (a.grad_bits > 0) {
             gsq = consumer_sum(gsq, sh->red);
-            if (threadIdx.x == 0) __stcg(a.gn + blockIdx.x, gsq);
-            ring_grid_barrier(a.barrier, (unsigned)G * ++barriers_done, sh, a.status, 3);
+            unsigned long long* gn = a.ll_gn + (size_t)par * G * 2;
+            if (threadIdx.x == 0) ll_store_double(gn + (size_t)blockIdx.x * 2, gsq, tag);
+            ll_gather(gn, 2 * G, tag, nbuf, sh, a.status, 3);
+            consumer_sync();
             double part = 0.0;
             if (warp == 0) {
-                for (int p = lane; p < G; p += 32) part += __ldcg(a.gn + p);
+                for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * p] + (double)nbuf[2 * p + 1];
                 part = warp_sum(part);
             }
             if (threadIdx.x == 0) sh->misc[1] = part;
             consumer_sync();
             q4.M = (float)sqrt(sh->misc[1]);
             q4.sm = (1 << (a.grad_bits - 1)) - 1;
-        } else {
-            consumer_sync();                     // gsub is complete
         }
         double xsq = 0.0;
-        for (int f = sub0 + threadIdx.x; f < sub1; f += kRingConsumers) {
+        for (int k = threadIdx.x; k < nsub; k += kRingConsumers) {
+            const int f = sub0 + k;
             float xn = 0.0f;
             if (f < fcnt) {
-                float g = gsub[f - sub0];
+                float g = gsub[k];
                 if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
                 if (last && a.grad_out) a.grad_out[a.n + j0 + f] = g;
                 xn = fmaf(-a.lr, g, xs[f]);
                 xsq += (double)xn * (double)xn;
             }
-            __stcg(a.xg + j0 + f, xn);
+            ll_store(ag_part + f, xn, tag);
         }
         if (a.model_bits > 0) {
             xsq = consumer_sum(xsq, sh->red);
-            if (threadIdx.x == 0) __stcg(a.gn + G + blockIdx.x, xsq);
+            if (threadIdx.x == 0) ll_store_double(ag_norm + (size_t)blockIdx.x * 2, xsq, tag);
         }
-        ring_grid_barrier(a.barrier, (unsigned)G * ++barriers_done, sh, a.status, 4);
 
         // -------------------------------------------------------------- all-gather: new model of the part
-        for (int f = 4 * threadIdx.x; f < F; f += 4 * kRingConsumers)
-            *reinterpret_cast<float4*>(xs + f) = __ldcg(reinterpret_cast<const float4*>(a.xg + j0 + f));
+        consumer_sync();                         // everybody is done with xs of this step
+        ll_gather(ag_part, F, tag, xs, sh, a.status, 4);
         if (a.model_bits > 0) {
+            ll_gather(ag_norm, 2 * G, tag, nbuf + 2 * G, sh, a.status, 8);
+            consumer_sync();
             double part = 0.0;
             if (warp == 0) {
-                for (int p = lane; p < G; p += 32) part += __ldcg(a.gn + G + p);
+                for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * G + 2 * p] + (double)nbuf[2 * G + 2 * p + 1];
                 part = warp_sum(part);
             }
             if (threadIdx.x == 0) sh->misc[2] = part;
@@ -510,11 +577,14 @@ struct RingPlan {
     size_t smem;
 };
 
-static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int sub, int cr, int slots) {
+static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int sub, int cr, int slots, int nb, int G) {
     const int fpw = 32 / cb;
     const size_t F = (size_t)wc * fpw, L = (size_t)1 << bits;
+    const size_t subp = (size_t)sub + 2;
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
-    bytes += sizeof(float) * (F + (table ? 2 * L * F : F) + (size_t)sub + (size_t)kRingConsumers * fpw + (size_t)((2 * rc + 3) & ~3));
+    bytes += sizeof(float) * (F + (table ? 2 * L * F : F) + (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
+    bytes += sizeof(double) * ((subp + 1) & ~(size_t)1);
+    bytes += sizeof(float) * (4 * (size_t)G + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
     bytes += sizeof(uint32_t) * (size_t)slots * 2 * cr * wc;
     return bytes;
 }
@@ -554,25 +624,27 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         r.cr = cr;
         if (sizeof(uint32_t) * 2 * (size_t)cr * r.wc >= (1u << 20)) return false;   // mbarrier tx-count range
         int slots = kRingMaxSlots;
-        while (slots >= 2 && ring_smem_bytes(cb, table, r.wc, r.rc, d->bits, r.sub, cr, slots) > cap) --slots;
+        while (slots >= 2 && ring_smem_bytes(cb, table, r.wc, r.rc, d->bits, r.sub, cr, slots, r.nb, r.na * r.nb) > cap) --slots;
         if (slots < 2) return false;
         r.slots = slots;
-        r.smem = ring_smem_bytes(cb, table, r.wc, r.rc, d->bits, r.sub, cr, slots);
+        r.smem = ring_smem_bytes(cb, table, r.wc, r.rc, d->bits, r.sub, cr, slots, r.nb, r.na * r.nb);
         *out = r;
         return true;
     };
 
+    const int na_min = (int)((words + kRingConsumers - 1) / kRingConsumers);
     if (p->grid_feature_parts > 0 || p->grid_row_parts > 0) {
         int na = p->grid_feature_parts > 0 ? p->grid_feature_parts : 1;
         int nb = p->grid_row_parts > 0 ? p->grid_row_parts : 1;
         if ((int64_t)na * 32 > ring_round_up((int)words, 32)) na = (int)((words + 31) / 32);
+        if (na < na_min) na = na_min;          // the request is a hint: parts never exceed one word column per thread
         if (nb > B) nb = (int)B;
         return shape(na, nb, plan) ? ZIPML_OK : ZIPML_ERR_WORKSPACE;
     }
     bool found = false;
     double best_cost = 0.0;
     const int na_max = (int)((words + 31) / 32);
-    for (int na = 1; na <= na_max && na <= sms; ++na) {
+    for (int na = na_min; na <= na_max && na <= sms; ++na) {
         int nb = sms / na;
         if (nb > B) nb = (int)B;
         if (nb < 1) nb = 1;
@@ -613,12 +685,13 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     const size_t npad = (size_t)plan.na * plan.wc * fpw;
     size_t off = 0;
     auto piece = [&](size_t bytes) { const size_t o = off; off += carve_size(bytes); return o; };
-    const size_t o_pd = piece(sizeof(double) * (size_t)plan.na * (size_t)B * 2);
-    const size_t o_pg = piece(sizeof(float) * (size_t)plan.nb * npad);
-    const size_t o_ps = piece(sizeof(double) * (size_t)plan.nb);
-    const size_t o_xg = piece(sizeof(float) * npad);
-    const size_t o_gn = piece(sizeof(double) * 2 * (size_t)G);
-    const size_t o_bar = piece(sizeof(unsigned) * 4);
+    const size_t subp = (size_t)plan.sub + 2;
+    const size_t n_pd = plan.na > 1 ? 2 * (size_t)plan.nb * plan.na * plan.rc * 4 : 0;
+    const size_t n_rs = (size_t)G * plan.nb * subp;
+    const size_t n_gn = 2 * (size_t)G * 2;
+    const size_t n_ag = npad + 2 * (size_t)G;
+    const size_t o_ll = piece(sizeof(unsigned long long) * (n_pd + n_rs + n_gn + n_ag));
+    const size_t ll_bytes = off - o_ll;
     const size_t o_ord = piece(sizeof(int32_t) * (size_t)(p->batch_order ? T : 0));
     rc = ws_reserve(ctx, off);
     if (rc != ZIPML_OK) return rc;
@@ -636,12 +709,11 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.seed = p->seed; a.epoch = (uint32_t)p->epoch;
     a.na = plan.na; a.nb = plan.nb; a.wc = plan.wc; a.rc = plan.rc; a.stages = plan.slots;
     a.cr = plan.cr; a.sub = plan.sub;
-    a.pd = reinterpret_cast<double*>(ctx->ws + o_pd);
-    a.pg = reinterpret_cast<float*>(ctx->ws + o_pg);
-    a.ps = reinterpret_cast<double*>(ctx->ws + o_ps);
-    a.xg = reinterpret_cast<float*>(ctx->ws + o_xg);
-    a.gn = reinterpret_cast<double*>(ctx->ws + o_gn);
-    a.barrier = reinterpret_cast<unsigned*>(ctx->ws + o_bar);
+    a.pd = nullptr; a.pg = nullptr; a.ps = nullptr; a.barrier = nullptr;
+    a.ll_pd = reinterpret_cast<unsigned long long*>(ctx->ws + o_ll);
+    a.ll_rs = a.ll_pd + n_pd;
+    a.ll_gn = a.ll_rs + n_rs;
+    a.ll_ag = a.ll_gn + n_gn;
     a.status = ctx->d_status;
     a.order = nullptr;
     a.phases = kPhaseAll; a.persistent = 1;
@@ -651,10 +723,10 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         if (e != cudaSuccess) return cuda_status(e);
         a.order = dev_order;
     }
-    // barrier targets are 32-bit: at most 4 barriers per step and G arrivals per barrier
-    const int64_t max_steps = (int64_t)(0x7fffffffLL / (4LL * G));
+    // packet tags are 32-bit step counters starting at 1
+    const int64_t max_steps = 0x7fffffffLL;
     for (int64_t s0 = first_step; s0 < first_step + num_steps; s0 += max_steps) {
-        e = cudaMemsetAsync(a.barrier, 0, sizeof(unsigned) * 4, ctx->stream);
+        e = cudaMemsetAsync(ctx->ws + o_ll, 0, ll_bytes, ctx->stream);
         if (e != cudaSuccess) return cuda_status(e);
         SgdArgs chunk = a;
         chunk.first_step = s0;
