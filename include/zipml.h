@@ -85,7 +85,10 @@ typedef struct zipml_sgd_params {
     float lr;                   /* step length gamma, constant within the call                       */
     int32_t grid_feature_parts; /* tuning, 0 = automatic: CTAs along the features                    */
     int32_t grid_row_parts;     /* tuning, 0 = automatic: CTAs along the rows of a minibatch         */
-    int32_t reserved;
+    int32_t trace_steps;        /* profiling: number of steps to trace (0 = none)                    */
+    uint64_t* trace;            /* profiling, DEVICE pointer or NULL: 8 uint64 per traced step; CTA 0
+                                   stores the device nanosecond timer at the step's phase boundaries
+                                   (ring engine only)                                                */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

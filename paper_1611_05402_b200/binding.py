@@ -42,7 +42,8 @@ class CSgdParams(C.Structure):
     _fields_ = [("struct_size", C.c_uint32), ("model_bits", C.c_int32), ("grad_bits", C.c_int32), ("engine", C.c_int32),
                 ("batch", C.c_int64), ("epoch", C.c_int64), ("first_step", C.c_int64), ("num_steps", C.c_int64),
                 ("seed", C.c_uint64), ("batch_order", C.c_void_p), ("lr", C.c_float),
-                ("grid_feature_parts", C.c_int32), ("grid_row_parts", C.c_int32), ("reserved", C.c_int32)]
+                ("grid_feature_parts", C.c_int32), ("grid_row_parts", C.c_int32), ("trace_steps", C.c_int32),
+                ("trace", C.c_void_p)]
 
 
 _lib = None
@@ -191,12 +192,15 @@ class Context:
         return (lev, obj) if want_objective else lev
 
     def sgd_params(self, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=-1,
-                   batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0):
+                   batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0, trace=None):
         p = CSgdParams()
         p.struct_size = C.sizeof(CSgdParams)
         p.model_bits, p.grad_bits, p.engine = model_bits, grad_bits, engine
         p.batch, p.epoch, p.first_step, p.num_steps, p.seed, p.lr = batch, epoch, first_step, num_steps, seed, lr
         p.grid_feature_parts, p.grid_row_parts = grid_feature_parts, grid_row_parts
+        if trace is not None:      # (steps, 8) int64 device tensor
+            assert trace.dtype == torch.int64 and trace.is_contiguous() and trace.shape[1] == 8
+            p.trace, p.trace_steps = trace.data_ptr(), trace.shape[0]
         keep = None
         if batch_order is not None:
             keep = torch.as_tensor(batch_order, dtype=torch.int32, device="cpu").contiguous()

@@ -43,12 +43,14 @@ struct SgdArgs {
     unsigned long long* ll_pd;   // [2][nb][na][rc][4]   partial dots (hi, lo of two doubles); only na > 1
     unsigned long long* ll_rs;   // [na][nb][nb][sub+2]  partial gradients per (owner, writer) + residual sum
     unsigned long long* ll_gn;   // [2][G][2]            partial squared gradient norms (hi, lo)
-    unsigned long long* ll_ag;   // [na*wc*FPW] new model, then [G][2] partial squared model norms
+    unsigned long long* ll_ag;   // [na*wc*FPW] model the next step sees, then [2][G][2] partial squared model norms
     double* pd;             // [2][na][batch][2]   partial dots
     float* pg;              // [2][nb][na*wc*FPW]  partial code gradients (table mode: value gradients)
     double* ps;             // [2][nb]             partial sums of r1 + r2
     unsigned* barrier;      // grid barrier counter (zeroed before a persistent launch)
     DeviceStatus* status;
+    unsigned long long* trace;   // ring engine: optional timestamps, 8 per step for the first trace_steps steps
+    int trace_steps;
     int phases;             // mask of kPhase*
     int persistent;
 };

@@ -16,7 +16,9 @@
 //            reduce-scatter: CTA (ai, bi) collects the nb row parts of its own sub-slice of feature
 //            part ai, sums them in a fixed order, applies the optional gradient quantizer (one more
 //            exchange for the norm) and the update, and publishes the new sub-slice;
-//            all-gather: every CTA collects the new model of its feature part.
+//            all-gather: every CTA collects, word by word, the model its feature part will see in
+//            the next step (the owners keep the fp32 master of their sub-slice to themselves and
+//            publish Q3 of it when the model quantizer is on) and turns it into w = step * x~.
 // Exchange.  Nothing here uses a grid barrier.  Every exchanged number travels as an 8-byte packet
 // {fp32 value, step tag} written with one 64-bit store; a reader polls the packet until the tag is
 // the current step's, so the data announces itself and one L2 round trip replaces "write, fence,
@@ -52,6 +54,7 @@ __device__ __forceinline__ double consumer_sum(double v, double* scratch) {
 
 struct RingShared {
     double red[16];
+    double dpart[16];
     double misc[8];
     unsigned long long full[kRingMaxSlots];
     unsigned long long empty[kRingMaxSlots];
@@ -67,6 +70,14 @@ __device__ __forceinline__ void ring_wait(unsigned long long* bar, uint32_t pari
         if (mbar_try_wait(reinterpret_cast<uint64_t*>(bar), parity)) return;
     *abort_flag = 1;
     set_status(status, ZIPML_ERR_TIMEOUT, where);
+}
+
+__device__ __forceinline__ void trace_mark(const SgdArgs& a, int64_t it, int slot_id) {
+    if (a.trace && blockIdx.x == 0 && threadIdx.x == 0 && it - a.first_step < a.trace_steps) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        a.trace[(it - a.first_step) * 8 + slot_id] = t;
+    }
 }
 
 // ---- packets ---------------------------------------------------------------------------------
@@ -113,12 +124,12 @@ __device__ __forceinline__ void ll_gather(const unsigned long long* src, int cou
 
 // Shared memory plan, F = wc * FPW features per CTA:
 //   RingShared
-//   xs[F] float                 model of the CTA's feature part
 //   tab float                   uniform: w[F] ([u][word][4]); table: WL[L*F] then LV[L*F] ([code][slot][word])
-//   gsub[sub] float             gradient of the CTA's own sub-slice
+//   lw[wc] float                uniform: sum over a word's features of lo * x~ (its share of lo^T x~)
+//   xown[sub] float             master model of the CTA's own sub-slice
+//   gsub[sub] float             gradient of the own sub-slice
 //   gbuf[nb*(sub+2)] float      collected row parts of the own sub-slice (+ residual sums)
-//   dsum[sub+2] double          their sums
-//   nbuf[4*G] float             collected partial norms
+//   nbuf[2*G] float             collected partial norms
 //   gred[kRingConsumers*FPW]    cross-group reduction of phase B
 //   res[2*rc] float             residuals
 //   bsm[2][rc] float            labels of the current and the next step's rows
@@ -132,13 +143,13 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     const int F = a.wc * FPW;
     const int G = a.na * a.nb;
     const int subp = a.sub + 2;                                  // packets per (owner, writer)
-    float* xs = reinterpret_cast<float*>(s_raw + ((sizeof(RingShared) + 15) & ~(size_t)15));
-    float* tab = xs + F;
-    float* gsub = tab + (TABLE ? 2 * L * F : F);
+    float* tab = reinterpret_cast<float*>(s_raw + ((sizeof(RingShared) + 15) & ~(size_t)15));
+    float* lw = tab + (TABLE ? 2 * L * F : F);
+    float* xown = lw + a.wc;
+    float* gsub = xown + a.sub;
     float* gbuf = gsub + a.sub;
-    double* dsum = reinterpret_cast<double*>(gbuf + ((a.nb * subp + 3) & ~3));
-    float* nbuf = reinterpret_cast<float*>(dsum + ((subp + 1) & ~1));
-    float* gred = nbuf + 4 * G;
+    float* nbuf = gbuf + ((a.nb * subp + 3) & ~3);
+    float* gred = nbuf + ((2 * G + 3) & ~3);
     float* res = gred + kRingConsumers * FPW;
     float* bsm = res + ((2 * a.rc + 3) & ~3);
     uint32_t* ring = reinterpret_cast<uint32_t*>(bsm + ((2 * a.rc + 3) & ~3));
@@ -215,7 +226,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     }
 
     // ================================================================== consumers
-    for (int f = threadIdx.x; f < F; f += kRingConsumers) xs[f] = (f < fcnt) ? a.x[j0 + f] : 0.0f;
+    const float* LV = tab + L * F;
     if constexpr (TABLE) {
         float* LVw = tab + L * F;
         for (int idx = threadIdx.x; idx < L * F; idx += kRingConsumers) {
@@ -223,15 +234,60 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             const int f = q * FPW + i;
             LVw[idx] = (f < fcnt) ? __ldg(a.levels + (j0 + f) * L + c) : 0.0f;
         }
+        consumer_sync();
     }
-    // squared norm of the whole model for the first step's model quantizer
-    double xnorm2 = 0.0;
-    if (a.model_bits > 0) {
-        double ss = 0.0;
-        for (int64_t j = threadIdx.x; j < a.n; j += kRingConsumers) { const double v = (double)a.x[j]; ss += v * v; }
-        xnorm2 = consumer_sum(ss, sh->red);
-    }
-    {   // labels of the first step's rows
+    // Turns the model values of word q (as the gradient will see them) into what phase A reads.
+    auto build_word = [&](int q, const float (&xt)[FPW]) {
+        if constexpr (!TABLE) {
+            float wv[FPW];
+            float lsum = 0.0f;
+#pragma unroll
+            for (int i = 0; i < FPW; ++i) {
+                const int f = q * FPW + i;
+                float sv = 0.0f, lv = 0.0f;
+                if (f < fcnt) { sv = __ldg(a.step + j0 + f); lv = __ldg(a.lo + j0 + f); }
+                wv[i] = sv * xt[i];
+                lsum = fmaf(lv, xt[i], lsum);
+            }
+#pragma unroll
+            for (int u = 0; u < FPW / 4; ++u)
+                *reinterpret_cast<float4*>(tab + (u * a.wc + q) * 4) = make_float4(wv[4 * u], wv[4 * u + 1], wv[4 * u + 2], wv[4 * u + 3]);
+            lw[q] = lsum;
+        } else {
+#pragma unroll
+            for (int i = 0; i < FPW; ++i)
+                for (int c = 0; c < L; ++c) tab[(c * FPW + i) * a.wc + q] = LV[(c * FPW + i) * a.wc + q] * xt[i];
+        }
+    };
+
+    // own sub-slice of the feature part, and who acts for feature k of it: a thread when few CTAs
+    // contribute, lane 0 of a warp (whose lanes split the contributors) when many do
+    const int sub0 = min(F, bi * a.sub), sub1 = min(F, sub0 + a.sub);
+    const int nsub = sub1 - sub0;
+    const bool warp_path = a.nb > 32;
+    const int kstart = warp_path ? warp : threadIdx.x, kstride = warp_path ? kRingWarps : kRingConsumers;
+    const bool actor = !warp_path || lane == 0;
+
+    // first step: model from the caller's vector
+    {
+        VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)a.first_step, 3u};
+        if (a.model_bits > 0) {
+            double ss = 0.0;
+            for (int64_t j = threadIdx.x; j < a.n; j += kRingConsumers) { const double v = (double)a.x[j]; ss += v * v; }
+            q3.M = (float)sqrt(consumer_sum(ss, sh->red));
+            q3.sm = (1 << (a.model_bits - 1)) - 1;
+        }
+        for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
+            float xt[FPW];
+#pragma unroll
+            for (int i = 0; i < FPW; ++i) {
+                const int f = q * FPW + i;
+                xt[i] = (f < fcnt) ? a.x[j0 + f] : 0.0f;
+                if (a.model_bits > 0) xt[i] = q3.apply(xt[i], (uint32_t)(j0 + f));
+            }
+            build_word(q, xt);
+        }
+        for (int k = threadIdx.x; k < nsub; k += kRingConsumers) xown[k] = (sub0 + k < fcnt) ? a.x[j0 + sub0 + k] : 0.0f;
         int64_t r0; int bt, rcnt;
         step_rows(a.first_step, r0, bt, rcnt);
         float* bcur = bsm + (size_t)(a.first_step & 1) * a.rc;
@@ -239,21 +295,24 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     }
     consumer_sync();
 
-    // step-invariant thread roles
+    // step-invariant thread roles of phase B and where this CTA's packets go and come from
     const int lanes_q = min(kRingConsumers, ((wcnt + 31) / 32) * 32);
     const int ngroups = kRingConsumers / lanes_q;
     const int group = threadIdx.x / lanes_q;
     const int ql = threadIdx.x % lanes_q;
-    const int sub0 = min(F, bi * a.sub), sub1 = min(F, sub0 + a.sub);        // own sub-slice of the feature part
-    const float* LV = tab + L * F;
     const int chunks_w = (wcnt + 31) / 32;
-    int slot = 0;
-    uint32_t phase = 0;
-    // where this CTA's packets go and come from
     unsigned long long* rs_mine = a.ll_rs + (size_t)ai * a.nb * a.nb * subp;                 // + (owner*nb + writer)*subp
     const unsigned long long* rs_own = rs_mine + (size_t)bi * a.nb * subp;                   // collected by this owner
     unsigned long long* ag_part = a.ll_ag + j0;
-    unsigned long long* ag_norm = a.ll_ag + npad;
+    int rs_off[FPW];                             // packet of feature i of this thread's word, for the writer bi
+#pragma unroll
+    for (int i = 0; i < FPW; ++i) {
+        const int f = ql * FPW + i;
+        const int owner = min(f / a.sub, a.nb - 1);
+        rs_off[i] = (owner * a.nb + bi) * subp + (f - owner * a.sub);
+    }
+    int slot = 0;
+    uint32_t phase = 0;
 
     for (int64_t it = a.first_step; it < step_end; ++it) {
         int64_t r0; int bt, rcnt;
@@ -263,50 +322,41 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         const uint32_t tag = (uint32_t)(it - a.first_step) + 1u;
         const int par = (int)(it & 1);
         const float* bcur = bsm + (size_t)par * a.rc;
+        trace_mark(a, it, 0);
 
-        // -------------------------------------------------------------- model seen by the step
-        VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 3u};
-        if (a.model_bits > 0) { q3.M = (float)sqrt(xnorm2); q3.sm = (1 << (a.model_bits - 1)) - 1; }
-        double base = 0.0;
-        if constexpr (!TABLE) {
-            for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
-#pragma unroll
-                for (int i = 0; i < FPW; ++i) {
-                    const int f = q * FPW + i;
-                    float xv = xs[f];
-                    if (a.model_bits > 0) xv = q3.apply(xv, (uint32_t)(j0 + f));
-                    float sv = 0.0f, lv = 0.0f;
-                    if (f < fcnt) { sv = __ldg(a.step + j0 + f); lv = __ldg(a.lo + j0 + f); }
-                    tab[((i >> 2) * a.wc + q) * 4 + (i & 3)] = sv * xv;
-                    base += (double)lv * (double)xv;
-                }
-            }
-            base = consumer_sum(base, sh->red);
-        } else {
-            for (int f = threadIdx.x; f < F; f += kRingConsumers) {
-                float xv = xs[f];
-                if (a.model_bits > 0) xv = q3.apply(xv, (uint32_t)(j0 + f));
-                const int q = f / FPW, i = f % FPW;
-                for (int c = 0; c < L; ++c) tab[(c * FPW + i) * a.wc + q] = LV[(c * FPW + i) * a.wc + q] * xv;
-            }
-            consumer_sync();
+        // labels of the next step's rows: requested now, parked in shared memory at the end of the step
+        float breg = 0.0f;
+        int rcnt_next = 0;
+        int64_t r0_next = 0;
+        if (!last) {
+            int btn;
+            step_rows(it + 1, r0_next, btn, rcnt_next);
+            if ((int)threadIdx.x < rcnt_next) breg = __ldg(a.b + r0_next + k0 + threadIdx.x);
         }
 
         // -------------------------------------------------------------- phase A: dots
         const bool dots_local = (a.na == 1);
         unsigned long long* pd_mine = a.ll_pd + (((size_t)par * a.nb + bi) * a.na + ai) * a.rc * 4;
         const int slot_a = slot;                 // slot of the single chunk when C == 1
+        // with fewer rows than warps (single-chunk tiles only) a row is split over S warps
+        int S = 1;
+        if (C == 1 && rcnt < kRingWarps) S = max(1, min(chunks_w, kRingWarps / rcnt));
+        const int cps = (chunks_w + S - 1) / S;
+        double wsum = 0.0;                       // lane 0: r1 + r2 over the rows this warp finished
         for (int chunk = 0; chunk < C; ++chunk) {
             const int rows = min(a.cr, rcnt - chunk * a.cr);
             ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 6);
             const uint32_t* t1 = ring + (size_t)slot * slot_words;
             const uint32_t* t2 = t1 + (size_t)a.cr * a.wc;
-            for (int lr = warp; lr < rows; lr += kRingWarps) {
+            for (int task = warp; task < rows * S; task += kRingWarps) {
+                const int lr = task / S, seg = task - lr * S;
                 const uint32_t* row1 = t1 + (size_t)lr * a.wc;
                 const uint32_t* row2 = t2 + (size_t)lr * a.wc;
                 float acc1[2] = {0.0f, 0.0f}, acc2[2] = {0.0f, 0.0f};
+                float lsum = 0.0f;
+                const int c_end = min(chunks_w, (seg + 1) * cps);
 #pragma unroll 4
-                for (int c = 0; c < chunks_w; ++c) {
+                for (int c = seg * cps; c < c_end; ++c) {
                     const int q = c * 32 + lane;
                     if (q < wcnt) {
                         const uint32_t u1 = row1[q], u2 = row2[q];
@@ -314,6 +364,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                             float c1[FPW], c2[FPW];
                             unpack_word<CB>(u1, c1);
                             unpack_word<CB>(u2, c2);
+                            lsum += lw[q];
 #pragma unroll
                             for (int u = 0; u < FPW / 4; ++u) {
                                 const float4 wv = *reinterpret_cast<const float4*>(tab + (u * a.wc + q) * 4);
@@ -335,14 +386,19 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                         }
                     }
                 }
-                const double d1 = warp_sum((double)acc1[0] + (double)acc1[1]) + base;
-                const double d2 = warp_sum((double)acc2[0] + (double)acc2[1]) + base;
+                const double d1 = warp_sum((double)acc1[0] + (double)acc1[1] + (double)lsum);
+                const double d2 = warp_sum((double)acc2[0] + (double)acc2[1] + (double)lsum);
                 if (lane == 0) {
                     const int r = chunk * a.cr + lr;
-                    if (dots_local) {
+                    if (S > 1) {
+                        sh->dpart[2 * task] = d1;
+                        sh->dpart[2 * task + 1] = d2;
+                    } else if (dots_local) {
                         const double bk = (double)bcur[r];
-                        res[2 * r] = (float)(d1 - bk);
-                        res[2 * r + 1] = (float)(d2 - bk);
+                        const float r1 = (float)(d1 - bk), r2 = (float)(d2 - bk);
+                        res[2 * r] = r1;
+                        res[2 * r + 1] = r2;
+                        wsum += (double)r1 + (double)r2;
                     } else {
                         ll_store_double(pd_mine + (size_t)r * 4, d1, tag);
                         ll_store_double(pd_mine + (size_t)r * 4 + 2, d2, tag);
@@ -355,9 +411,35 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 if (++slot == slots) { slot = 0; phase ^= 1u; }
             }
         }
-        if (!dots_local) {
+        if (S > 1) {
+            consumer_sync();
+            if (warp == 0) {                     // rcnt < 8 rows: one lane per row, in segment order
+                double v = 0.0;
+                if (lane < rcnt) {
+                    double d1 = 0.0, d2 = 0.0;
+                    for (int sg = 0; sg < S; ++sg) { d1 += sh->dpart[2 * (lane * S + sg)]; d2 += sh->dpart[2 * (lane * S + sg) + 1]; }
+                    if (dots_local) {
+                        const double bk = (double)bcur[lane];
+                        const float r1 = (float)(d1 - bk), r2 = (float)(d2 - bk);
+                        res[2 * lane] = r1;
+                        res[2 * lane + 1] = r2;
+                        v = (double)r1 + (double)r2;
+                    } else {
+                        ll_store_double(pd_mine + (size_t)lane * 4, d1, tag);
+                        ll_store_double(pd_mine + (size_t)lane * 4 + 2, d2, tag);
+                    }
+                }
+                wsum = warp_sum(v);
+            } else {
+                wsum = 0.0;
+            }
+        }
+        if (dots_local) {
+            if (lane == 0) sh->red[warp] = wsum;
+        } else {
             // every row's dot is the sum, in part order, of the na partial dots published for it
             const unsigned long long* pd_row = a.ll_pd + ((size_t)par * a.nb + bi) * a.na * a.rc * 4;
+            double part = 0.0;
             for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) {
                 double d1 = 0.0, d2 = 0.0;
                 bool good = !*reinterpret_cast<volatile int*>(&sh->abort_flag);
@@ -375,16 +457,18 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                     d2 += (double)__uint_as_float((uint32_t)v[2]) + (double)__uint_as_float((uint32_t)v[3]);
                 }
                 const double bk = (double)bcur[r];
-                res[2 * r] = good ? (float)(d1 - bk) : 0.0f;
-                res[2 * r + 1] = good ? (float)(d2 - bk) : 0.0f;
+                const float r1 = good ? (float)(d1 - bk) : 0.0f, r2 = good ? (float)(d2 - bk) : 0.0f;
+                res[2 * r] = r1;
+                res[2 * r + 1] = r2;
+                part += (double)r1 + (double)r2;
             }
+            part = warp_sum(part);
+            if (lane == 0) sh->red[warp] = part;
         }
-        consumer_sync();                         // residuals are complete
+        consumer_sync();                         // residuals and the per-warp residual sums are complete
+        trace_mark(a, it, 1);
 
         // -------------------------------------------------------------- phase B: gradient
-        double ssum = 0.0;
-        for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) ssum += (double)res[2 * r] + (double)res[2 * r + 1];
-        ssum = consumer_sum(ssum, sh->red);
         {
             const int q = ql;
             const bool active = (group < ngroups) && (q < wcnt);
@@ -407,7 +491,8 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                     for (int lr = group; lr < rows; lr += ngroups) {
                         const uint32_t u1 = col1[(size_t)lr * a.wc];
                         const uint32_t u2 = col2[(size_t)lr * a.wc];
-                        const float r1 = rr[2 * lr], r2 = rr[2 * lr + 1];
+                        const float2 rv = *reinterpret_cast<const float2*>(rr + 2 * lr);
+                        const float r1 = rv.x, r2 = rv.y;
                         if constexpr (!TABLE) {
                             float c1[FPW], c2[FPW];
                             unpack_word<CB>(u1, c1);
@@ -447,13 +532,8 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 }
             }
             if (active && group == 0) {
-                // feature f of the part belongs to owner f / sub; its packet sits in that owner's block for this writer
 #pragma unroll
-                for (int i = 0; i < FPW; ++i) {
-                    const int f = q * FPW + i;
-                    const int owner = f / a.sub;
-                    ll_store(rs_mine + ((size_t)owner * a.nb + bi) * subp + (f - owner * a.sub), acc[i], tag);
-                }
+                for (int i = 0; i < FPW; ++i) ll_store(rs_mine + rs_off[i], acc[i], tag);
             }
         }
         if (C == 1) {                            // the retained single chunk goes back now
@@ -468,49 +548,48 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             ll_store(rs_mine + ((size_t)owner * a.nb + bi) * subp + (f - owner * a.sub), 0.0f, tag);
         }
         // the residual sum goes to every owner of the part, behind the gradient packets
-        for (int o = threadIdx.x; o < a.nb; o += kRingConsumers)
-            ll_store_double(rs_mine + ((size_t)o * a.nb + bi) * subp + a.sub, ssum, tag);
-        // labels of the next step's rows, fetched while the packets travel
-        if (!last) {
-            int64_t r0n; int btn, rcntn;
-            step_rows(it + 1, r0n, btn, rcntn);
-            float* bnext = bsm + (size_t)(par ^ 1) * a.rc;
-            for (int r = threadIdx.x; r < rcntn; r += kRingConsumers) bnext[r] = __ldg(a.b + r0n + k0 + r);
+        if ((int)threadIdx.x < a.nb) {
+            double ssum = 0.0;
+#pragma unroll
+            for (int w = 0; w < kRingWarps; ++w) ssum += sh->red[w];
+            for (int o = threadIdx.x; o < a.nb; o += kRingConsumers)
+                ll_store_double(rs_mine + ((size_t)o * a.nb + bi) * subp + a.sub, ssum, tag);
         }
+        trace_mark(a, it, 2);
 
         // -------------------------------------------------------------- reduce-scatter: own sub-slice
-        const int nsub = sub1 - sub0;            // features this CTA owns (may be 0 for the last owners)
         ll_gather(rs_own, a.nb * subp, tag, gbuf, sh, a.status, 2);
         consumer_sync();
-        if (a.nb <= 32) {
-            for (int k = threadIdx.x; k < subp; k += kRingConsumers) {
-                double t = 0.0;
-                for (int w = 0; w < a.nb; ++w) t += (double)gbuf[w * subp + k];
-                dsum[k] = t;
-            }
+        trace_mark(a, it, 3);
+        double stot = 0.0;
+        if (warp_path) {
+            double t = 0.0;
+            for (int w = lane; w < a.nb; w += 32) t += (double)gbuf[w * subp + a.sub] + (double)gbuf[w * subp + a.sub + 1];
+            stot = warp_sum(t);
         } else {
-            for (int k = warp; k < subp; k += kRingWarps) {
-                double t = 0.0;
-                for (int w = lane; w < a.nb; w += 32) t += (double)gbuf[w * subp + k];
-                t = warp_sum(t);
-                if (lane == 0) dsum[k] = t;
-            }
+            for (int w = 0; w < a.nb; ++w) stot += (double)gbuf[w * subp + a.sub] + (double)gbuf[w * subp + a.sub + 1];
         }
-        consumer_sync();
-        const double stot = dsum[a.sub] + dsum[a.sub + 1];
         const double scale = 1.0 / (2.0 * (double)bt);
         double gsq = 0.0;
-        for (int k = threadIdx.x; k < nsub; k += kRingConsumers) {
-            const int f = sub0 + k;
-            float g = 0.0f;
-            if (f < fcnt) {
-                double v = dsum[k];
-                if constexpr (!TABLE) v = (double)__ldg(a.lo + j0 + f) * stot + (double)__ldg(a.step + j0 + f) * v;
-                g = (float)(v * scale);
-                if (last && a.grad_out) a.grad_out[j0 + f] = g;
+        for (int k = kstart; k < nsub; k += kstride) {
+            double t = 0.0;
+            if (warp_path) {
+                for (int w = lane; w < a.nb; w += 32) t += (double)gbuf[w * subp + k];
+                t = warp_sum(t);
+            } else {
+                for (int w = 0; w < a.nb; ++w) t += (double)gbuf[w * subp + k];
             }
-            gsub[k] = g;
-            gsq += (double)g * (double)g;
+            if (actor) {
+                const int f = sub0 + k;
+                float g = 0.0f;
+                if (f < fcnt) {
+                    if constexpr (!TABLE) t = (double)__ldg(a.lo + j0 + f) * stot + (double)__ldg(a.step + j0 + f) * t;
+                    g = (float)(t * scale);
+                    if (last && a.grad_out) a.grad_out[j0 + f] = g;
+                }
+                gsub[k] = g;
+                gsq += (double)g * (double)g;
+            }
         }
         VecQuant q4{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 4u};
         if (a.grad_bits > 0) {
@@ -520,53 +599,81 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             ll_gather(gn, 2 * G, tag, nbuf, sh, a.status, 3);
             consumer_sync();
             double part = 0.0;
-            if (warp == 0) {
-                for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * p] + (double)nbuf[2 * p + 1];
-                part = warp_sum(part);
-            }
-            if (threadIdx.x == 0) sh->misc[1] = part;
-            consumer_sync();
-            q4.M = (float)sqrt(sh->misc[1]);
+            for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * p] + (double)nbuf[2 * p + 1];
+            q4.M = (float)sqrt(warp_sum(part));  // every warp adds the same numbers in the same order
             q4.sm = (1 << (a.grad_bits - 1)) - 1;
         }
         double xsq = 0.0;
-        for (int k = threadIdx.x; k < nsub; k += kRingConsumers) {
-            const int f = sub0 + k;
-            float xn = 0.0f;
-            if (f < fcnt) {
-                float g = gsub[k];
-                if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
-                if (last && a.grad_out) a.grad_out[a.n + j0 + f] = g;
-                xn = fmaf(-a.lr, g, xs[f]);
+        for (int k = kstart; k < nsub; k += kstride) {
+            if (actor) {
+                const int f = sub0 + k;
+                float xn = 0.0f;
+                if (f < fcnt) {
+                    float g = gsub[k];
+                    if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
+                    if (last && a.grad_out) a.grad_out[a.n + j0 + f] = g;
+                    xn = fmaf(-a.lr, g, xown[k]);
+                }
+                xown[k] = xn;
                 xsq += (double)xn * (double)xn;
             }
-            ll_store(ag_part + f, xn, tag);
         }
+        trace_mark(a, it, 4);
+        if (last) break;
+
+        // what the next step's gradient will see: Q3 of the new model, or the model itself
+        VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)(it + 1), 3u};
         if (a.model_bits > 0) {
             xsq = consumer_sum(xsq, sh->red);
-            if (threadIdx.x == 0) ll_store_double(ag_norm + (size_t)blockIdx.x * 2, xsq, tag);
-        }
-
-        // -------------------------------------------------------------- all-gather: new model of the part
-        consumer_sync();                         // everybody is done with xs of this step
-        ll_gather(ag_part, F, tag, xs, sh, a.status, 4);
-        if (a.model_bits > 0) {
-            ll_gather(ag_norm, 2 * G, tag, nbuf + 2 * G, sh, a.status, 8);
+            unsigned long long* xnp = a.ll_ag + npad + (size_t)par * G * 2;
+            if (threadIdx.x == 0) ll_store_double(xnp + (size_t)blockIdx.x * 2, xsq, tag);
+            ll_gather(xnp, 2 * G, tag, nbuf, sh, a.status, 8);
             consumer_sync();
             double part = 0.0;
-            if (warp == 0) {
-                for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * G + 2 * p] + (double)nbuf[2 * G + 2 * p + 1];
-                part = warp_sum(part);
-            }
-            if (threadIdx.x == 0) sh->misc[2] = part;
-            consumer_sync();
-            xnorm2 = sh->misc[2];
-        } else {
-            consumer_sync();
+            for (int p = lane; p < G; p += 32) part += (double)nbuf[2 * p] + (double)nbuf[2 * p + 1];
+            q3.M = (float)sqrt(warp_sum(part));
+            q3.sm = (1 << (a.model_bits - 1)) - 1;
         }
+        for (int k = kstart; k < nsub; k += kstride) {
+            if (actor) {
+                const int f = sub0 + k;
+                float xt = xown[k];
+                if (a.model_bits > 0 && f < fcnt) xt = q3.apply(xt, (uint32_t)(j0 + f));
+                ll_store(ag_part + f, xt, tag);
+            }
+        }
+        trace_mark(a, it, 5);
+
+        // -------------------------------------------------------------- all-gather: the part's model, word by word
+        for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
+            const unsigned long long* src = ag_part + (size_t)q * FPW;
+            unsigned long long v[FPW];
+            bool ok = false;
+            if (!*reinterpret_cast<volatile int*>(&sh->abort_flag)) {
+                for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
+                    ok = true;
+#pragma unroll
+                    for (int i = 0; i < FPW; ++i) { v[i] = ll_load(src + i); ok = ok && ((uint32_t)(v[i] >> 32) == tag); }
+                }
+                if (!ok) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 4); }
+            }
+            float xt[FPW];
+#pragma unroll
+            for (int i = 0; i < FPW; ++i) xt[i] = ok ? __uint_as_float((uint32_t)v[i]) : 0.0f;
+            build_word(q, xt);
+        }
+        {
+            float* bnext = bsm + (size_t)(par ^ 1) * a.rc;
+            if ((int)threadIdx.x < rcnt_next) bnext[threadIdx.x] = breg;
+            for (int r = threadIdx.x + kRingConsumers; r < rcnt_next; r += kRingConsumers) bnext[r] = __ldg(a.b + r0_next + k0 + r);
+        }
+        consumer_sync();
+        trace_mark(a, it, 6);
     }
-    if (bi == 0)
-        for (int f = threadIdx.x; f < fcnt; f += kRingConsumers) a.x[j0 + f] = xs[f];
+    consumer_sync();
+    // every owner returns its sub-slice of the master model
+    for (int k = threadIdx.x; k < nsub; k += kRingConsumers)
+        if (sub0 + k < fcnt) a.x[j0 + sub0 + k] = xown[k];
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -582,9 +689,8 @@ static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int 
     const size_t F = (size_t)wc * fpw, L = (size_t)1 << bits;
     const size_t subp = (size_t)sub + 2;
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
-    bytes += sizeof(float) * (F + (table ? 2 * L * F : F) + (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
-    bytes += sizeof(double) * ((subp + 1) & ~(size_t)1);
-    bytes += sizeof(float) * (4 * (size_t)G + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
+    bytes += sizeof(float) * ((table ? 2 * L * F : F) + (size_t)wc + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
+    bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
     bytes += sizeof(uint32_t) * (size_t)slots * 2 * cr * wc;
     return bytes;
 }
@@ -689,7 +795,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     const size_t n_pd = plan.na > 1 ? 2 * (size_t)plan.nb * plan.na * plan.rc * 4 : 0;
     const size_t n_rs = (size_t)G * plan.nb * subp;
     const size_t n_gn = 2 * (size_t)G * 2;
-    const size_t n_ag = npad + 2 * (size_t)G;
+    const size_t n_ag = npad + 4 * (size_t)G;
     const size_t o_ll = piece(sizeof(unsigned long long) * (n_pd + n_rs + n_gn + n_ag));
     const size_t ll_bytes = off - o_ll;
     const size_t o_ord = piece(sizeof(int32_t) * (size_t)(p->batch_order ? T : 0));
@@ -717,6 +823,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.status = ctx->d_status;
     a.order = nullptr;
     a.phases = kPhaseAll; a.persistent = 1;
+    a.trace = reinterpret_cast<unsigned long long*>(p->trace); a.trace_steps = p->trace ? p->trace_steps : 0;
     if (p->batch_order) {
         int32_t* dev_order = reinterpret_cast<int32_t*>(ctx->ws + o_ord);
         e = cudaMemcpyAsync(dev_order, p->batch_order, sizeof(int32_t) * (size_t)T, cudaMemcpyHostToDevice, ctx->stream);
