@@ -87,7 +87,7 @@ typedef struct zipml_sgd_params {
     int32_t grid_row_parts;     /* tuning, 0 = automatic: CTAs along the rows of a minibatch         */
     int32_t trace_steps;        /* profiling: number of steps to trace (0 = none)                    */
     uint64_t* trace;            /* profiling, DEVICE pointer or NULL: 8 uint64 per traced step; CTA 0
-                                   stores the device nanosecond timer at the step's phase boundaries
+                                   stores its SM's cycle counter at the step's phase boundaries
                                    (ring engine only)                                                */
 } zipml_sgd_params;
 

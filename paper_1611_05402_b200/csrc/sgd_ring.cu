@@ -75,7 +75,7 @@ __device__ __forceinline__ void ring_wait(unsigned long long* bar, uint32_t pari
 __device__ __forceinline__ void trace_mark(const SgdArgs& a, int64_t it, int slot_id) {
     if (a.trace && blockIdx.x == 0 && threadIdx.x == 0 && it - a.first_step < a.trace_steps) {
         unsigned long long t;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        asm volatile("mov.u64 %0, %clock64;" : "=l"(t));
         a.trace[(it - a.first_step) * 8 + slot_id] = t;
     }
 }
@@ -95,6 +95,23 @@ __device__ __forceinline__ unsigned long long ll_load(const unsigned long long* 
     return v;
 }
 constexpr long long kPacketSpinLimit = 1ll << 22;
+
+// Waits, with back-off, until `count` sentinel packets (src[i * stride], one per contributor) carry the
+// current step's tag.  Only `count` threads poll, so the wait costs L2 little; the full collection that
+// follows then finds (almost) every packet in place and still checks each tag itself.
+__device__ __forceinline__ void ll_wait_sentinels(const unsigned long long* src, int stride, int count, uint32_t tag,
+                                                  RingShared* sh, DeviceStatus* status, int where) {
+    for (int i = threadIdx.x; i < count; i += kRingConsumers) {
+        if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) break;
+        bool ok = false;
+        for (long long spin = 0; spin < kPacketSpinLimit; ++spin) {
+            if ((uint32_t)(ll_load(src + (size_t)i * stride) >> 32) == tag) { ok = true; break; }
+            __nanosleep(spin < 64 ? 32 : 256);
+        }
+        if (!ok) { sh->abort_flag = 1; set_status(status, ZIPML_ERR_TIMEOUT, where); }
+    }
+    consumer_sync();
+}
 
 // Collects `count` contiguous packets of the current step into dst (shared memory), the consumer
 // threads taking them four at a time so that their loads are in flight together.
@@ -558,6 +575,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         trace_mark(a, it, 2);
 
         // -------------------------------------------------------------- reduce-scatter: own sub-slice
+        ll_wait_sentinels(rs_own + a.sub, subp, a.nb, tag, sh, a.status, 2);      // each contributor's residual sum
         ll_gather(rs_own, a.nb * subp, tag, gbuf, sh, a.status, 2);
         consumer_sync();
         trace_mark(a, it, 3);
@@ -645,6 +663,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         trace_mark(a, it, 5);
 
         // -------------------------------------------------------------- all-gather: the part's model, word by word
+        ll_wait_sentinels(ag_part, a.sub, (F + a.sub - 1) / a.sub, tag, sh, a.status, 4);  // each owner's first feature
         for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
             const unsigned long long* src = ag_part + (size_t)q * FPW;
             unsigned long long v[FPW];
