@@ -56,6 +56,7 @@ struct RingShared {
     double red[16];
     double dpart[16];
     double misc[8];
+    float fmax[16];                // per-warp maxima: [0..7] |w| of the word stage, [8..15] |residual|
     unsigned long long full[kRingMaxSlots];
     unsigned long long empty[kRingMaxSlots];
     int abort_flag;
@@ -139,9 +140,87 @@ __device__ __forceinline__ void ll_gather(const unsigned long long* src, int cou
     }
 }
 
+// ---- integer contraction (uniform grids) ---------------------------------------------------------
+// Both phases contract small unsigned codes with an fp32 vector that is constant for many rows (w in
+// phase A, the residuals in phase B).  That vector is turned, once per step, into fixed point:
+// value ~ delta * W with |W| <= QMAX, and W into NS balanced base-128 digits in [-64, 63], each an
+// int8.  Four codes times four digits are then one dp4a into an int32, the digit sums are combined
+// exactly in 64 bits, and the only rounding is the one quantization of the vector (2^-20 of its
+// largest entry with three digits, 2^-27 with four; 8-bit codes use four because their large code
+// values amplify it).
+template <int CB>
+struct IntPath {
+    static constexpr int NS = (CB == 8) ? 4 : 3;
+    static constexpr int QMAX = (NS == 4) ? 133000000 : 1040000;   // below 63 * (128^NS - 1) / 127
+    static constexpr int NG = 8 / CB;                              // groups of four codes in a 32-bit word
+};
+
+__device__ __forceinline__ int dp4a_us(uint32_t codes, uint32_t digits, int acc) {
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(digits), "r"(acc));
+    return d;
+}
+
+// The four codes of group g of a word, one per byte: byte b holds feature b * NG + g of the word.
+template <int CB>
+__device__ __forceinline__ uint32_t group_bytes(uint32_t u, int g) {
+    if constexpr (CB == 8) return u;
+    else if constexpr (CB == 4) return (u >> (4 * g)) & 0x0F0F0F0Fu;
+    else return (u >> (2 * g)) & 0x03030303u;
+}
+
+template <int NS>
+__device__ __forceinline__ void balanced_digits(int W, int (&d)[NS]) {
+#pragma unroll
+    for (int s = 0; s < NS - 1; ++s) {
+        d[s] = ((W + 64) & 127) - 64;
+        W = (W - d[s]) >> 7;
+    }
+    d[NS - 1] = W;
+}
+
+__device__ __forceinline__ uint32_t pack_bytes(int b0, int b1, int b2, int b3) {
+    return (uint32_t)(b0 & 255) | ((uint32_t)(b1 & 255) << 8) | ((uint32_t)(b2 & 255) << 16) | ((uint32_t)(b3 & 255) << 24);
+}
+
+// Digit words of four values: out.x/.y/.z/.w = digit 0..3 of (v0, v1, v2, v3), one value per byte.
+template <int NS>
+__device__ __forceinline__ uint4 digit_words(const float (&v)[4], float inv_delta) {
+    int d[4][NS];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) balanced_digits<NS>(__float2int_rn(v[b] * inv_delta), d[b]);
+    uint4 o;
+    o.x = pack_bytes(d[0][0], d[1][0], d[2][0], d[3][0]);
+    o.y = pack_bytes(d[0][1], d[1][1], d[2][1], d[3][1]);
+    o.z = pack_bytes(d[0][2], d[1][2], d[2][2], d[3][2]);
+    o.w = (NS == 4) ? pack_bytes(d[0][NS - 1], d[1][NS - 1], d[2][NS - 1], d[3][NS - 1]) : 0u;
+    return o;
+}
+
+template <int NS>
+__device__ __forceinline__ long long combine_digits(const int (&acc)[NS]) {
+    long long t = 0;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) t += (long long)acc[s] << (7 * s);
+    return t;
+}
+
+// Maximum over the consumer threads (values >= 0); `slot` = 0 or 8 picks the half of sh->fmax.
+__device__ __forceinline__ float consumer_max(float v, RingShared* sh, int slot) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) sh->fmax[slot + (threadIdx.x >> 5)] = v;
+    consumer_sync();
+    float m = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kRingWarps; ++w) m = fmaxf(m, sh->fmax[slot + w]);
+    return m;
+}
+
 // Shared memory plan, F = wc * FPW features per CTA:
 //   RingShared
-//   tab float                   uniform: w[F] ([u][word][4]); table: WL[L*F] then LV[L*F] ([code][slot][word])
+//   tab                         uniform: digit words of w, uint4 [group][word]; table: WL[L*F] then LV[L*F] floats
+//                               ([code][slot][word])
 //   lw[wc] float                uniform: sum over a word's features of lo * x~ (its share of lo^T x~)
 //   xown[sub] float             master model of the CTA's own sub-slice
 //   gsub[sub] float             gradient of the own sub-slice
@@ -149,11 +228,14 @@ __device__ __forceinline__ void ll_gather(const unsigned long long* src, int cou
 //   nbuf[2*G] float             collected partial norms
 //   gred[kRingConsumers*FPW]    cross-group reduction of phase B
 //   res[2*rc] float             residuals
+//   rqs[2*ceil(rc/4)] uint4     uniform: digit words of the residuals, four rows each (r1 then r2)
 //   bsm[2][rc] float            labels of the current and the next step's rows
 //   ring[slots][2][cr][wc] u32  code chunks
 template <int CB, bool TABLE>
-__global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a) {
+__global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs a) {
     constexpr int FPW = 32 / CB;
+    constexpr int NS = IntPath<CB>::NS, NG = IntPath<CB>::NG;
+    constexpr float QMAXF = (float)IntPath<CB>::QMAX;
     extern __shared__ __align__(16) unsigned char s_raw[];
     RingShared* sh = reinterpret_cast<RingShared*>(s_raw);
     const int L = 1 << a.bits;
@@ -168,7 +250,8 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     float* nbuf = gbuf + ((a.nb * subp + 3) & ~3);
     float* gred = nbuf + ((2 * G + 3) & ~3);
     float* res = gred + kRingConsumers * FPW;
-    float* bsm = res + ((2 * a.rc + 3) & ~3);
+    uint4* rqs = reinterpret_cast<uint4*>(res + ((2 * a.rc + 3) & ~3));
+    float* bsm = reinterpret_cast<float*>(rqs + 2 * ((a.rc + 3) / 4));
     uint32_t* ring = reinterpret_cast<uint32_t*>(bsm + ((2 * a.rc + 3) & ~3));
     const size_t slot_words = (size_t)2 * a.cr * a.wc;
 
@@ -253,27 +336,41 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         }
         consumer_sync();
     }
-    // Turns the model values of word q (as the gradient will see them) into what phase A reads.
-    auto build_word = [&](int q, const float (&xt)[FPW]) {
+    // Turns the model values of this thread's word (as the gradient will see them) into what phase A
+    // reads; every consumer calls it, `have` says whether the thread holds a word (parts are at most
+    // one word per consumer wide).  Returns delta_w, the value of one fixed-point unit of w.
+    uint4* tabq = reinterpret_cast<uint4*>(tab);
+    auto word_stage = [&](bool have, int q, const float (&xt)[FPW]) -> double {
         if constexpr (!TABLE) {
             float wv[FPW];
-            float lsum = 0.0f;
+            float lsum = 0.0f, m = 0.0f;
 #pragma unroll
             for (int i = 0; i < FPW; ++i) {
                 const int f = q * FPW + i;
                 float sv = 0.0f, lv = 0.0f;
-                if (f < fcnt) { sv = __ldg(a.step + j0 + f); lv = __ldg(a.lo + j0 + f); }
+                if (have && f < fcnt) { sv = __ldg(a.step + j0 + f); lv = __ldg(a.lo + j0 + f); }
                 wv[i] = sv * xt[i];
                 lsum = fmaf(lv, xt[i], lsum);
+                m = fmaxf(m, fabsf(wv[i]));
             }
+            const float wmax = consumer_max(m, sh, 0);
+            const float inv = wmax > 0.0f ? QMAXF / wmax : 0.0f;
+            if (have) {
 #pragma unroll
-            for (int u = 0; u < FPW / 4; ++u)
-                *reinterpret_cast<float4*>(tab + (u * a.wc + q) * 4) = make_float4(wv[4 * u], wv[4 * u + 1], wv[4 * u + 2], wv[4 * u + 3]);
-            lw[q] = lsum;
+                for (int g = 0; g < NG; ++g) {
+                    const float v4[4] = {wv[0 * NG + g], wv[1 * NG + g], wv[2 * NG + g], wv[3 * NG + g]};
+                    tabq[g * a.wc + q] = digit_words<NS>(v4, inv);
+                }
+                lw[q] = lsum;
+            }
+            return (double)wmax / (double)QMAXF;
         } else {
+            if (have) {
 #pragma unroll
-            for (int i = 0; i < FPW; ++i)
-                for (int c = 0; c < L; ++c) tab[(c * FPW + i) * a.wc + q] = LV[(c * FPW + i) * a.wc + q] * xt[i];
+                for (int i = 0; i < FPW; ++i)
+                    for (int c = 0; c < L; ++c) tab[(c * FPW + i) * a.wc + q] = LV[(c * FPW + i) * a.wc + q] * xt[i];
+            }
+            return 0.0;
         }
     };
 
@@ -286,6 +383,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
     const bool actor = !warp_path || lane == 0;
 
     // first step: model from the caller's vector
+    double delta_w = 0.0;                        // one fixed-point unit of w, renewed with the model every step
     {
         VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)a.first_step, 3u};
         if (a.model_bits > 0) {
@@ -294,15 +392,17 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             q3.M = (float)sqrt(consumer_sum(ss, sh->red));
             q3.sm = (1 << (a.model_bits - 1)) - 1;
         }
-        for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
+        {
+            const int q = threadIdx.x;
+            const bool have = q < a.wc;
             float xt[FPW];
 #pragma unroll
             for (int i = 0; i < FPW; ++i) {
                 const int f = q * FPW + i;
-                xt[i] = (f < fcnt) ? a.x[j0 + f] : 0.0f;
-                if (a.model_bits > 0) xt[i] = q3.apply(xt[i], (uint32_t)(j0 + f));
+                xt[i] = (have && f < fcnt) ? a.x[j0 + f] : 0.0f;
+                if (a.model_bits > 0 && have) xt[i] = q3.apply(xt[i], (uint32_t)(j0 + f));
             }
-            build_word(q, xt);
+            delta_w = word_stage(have, q, xt);
         }
         for (int k = threadIdx.x; k < nsub; k += kRingConsumers) xown[k] = (sub0 + k < fcnt) ? a.x[j0 + sub0 + k] : 0.0f;
         int64_t r0; int bt, rcnt;
@@ -360,6 +460,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
         if (C == 1 && rcnt < kRingWarps) S = max(1, min(chunks_w, kRingWarps / rcnt));
         const int cps = (chunks_w + S - 1) / S;
         double wsum = 0.0;                       // lane 0: r1 + r2 over the rows this warp finished
+        float rmax = 0.0f;                       // and the largest |residual| this thread produced
         for (int chunk = 0; chunk < C; ++chunk) {
             const int rows = min(a.cr, rcnt - chunk * a.cr);
             ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 6);
@@ -370,6 +471,9 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 const uint32_t* row1 = t1 + (size_t)lr * a.wc;
                 const uint32_t* row2 = t2 + (size_t)lr * a.wc;
                 float acc1[2] = {0.0f, 0.0f}, acc2[2] = {0.0f, 0.0f};
+                int ia1[NS], ia2[NS];
+#pragma unroll
+                for (int sidx = 0; sidx < NS; ++sidx) { ia1[sidx] = 0; ia2[sidx] = 0; }
                 float lsum = 0.0f;
                 const int c_end = min(chunks_w, (seg + 1) * cps);
 #pragma unroll 4
@@ -378,21 +482,15 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                     if (q < wcnt) {
                         const uint32_t u1 = row1[q], u2 = row2[q];
                         if constexpr (!TABLE) {
-                            float c1[FPW], c2[FPW];
-                            unpack_word<CB>(u1, c1);
-                            unpack_word<CB>(u2, c2);
                             lsum += lw[q];
 #pragma unroll
-                            for (int u = 0; u < FPW / 4; ++u) {
-                                const float4 wv = *reinterpret_cast<const float4*>(tab + (u * a.wc + q) * 4);
-                                acc1[0] = fmaf(c1[4 * u + 0], wv.x, acc1[0]);
-                                acc1[1] = fmaf(c1[4 * u + 1], wv.y, acc1[1]);
-                                acc1[0] = fmaf(c1[4 * u + 2], wv.z, acc1[0]);
-                                acc1[1] = fmaf(c1[4 * u + 3], wv.w, acc1[1]);
-                                acc2[0] = fmaf(c2[4 * u + 0], wv.x, acc2[0]);
-                                acc2[1] = fmaf(c2[4 * u + 1], wv.y, acc2[1]);
-                                acc2[0] = fmaf(c2[4 * u + 2], wv.z, acc2[0]);
-                                acc2[1] = fmaf(c2[4 * u + 3], wv.w, acc2[1]);
+                            for (int g = 0; g < NG; ++g) {
+                                const uint4 dq = tabq[g * a.wc + q];
+                                const uint32_t b1 = group_bytes<CB>(u1, g), b2 = group_bytes<CB>(u2, g);
+                                ia1[0] = dp4a_us(b1, dq.x, ia1[0]); ia2[0] = dp4a_us(b2, dq.x, ia2[0]);
+                                ia1[1] = dp4a_us(b1, dq.y, ia1[1]); ia2[1] = dp4a_us(b2, dq.y, ia2[1]);
+                                ia1[2] = dp4a_us(b1, dq.z, ia1[2]); ia2[2] = dp4a_us(b2, dq.z, ia2[2]);
+                                if constexpr (NS == 4) { ia1[NS - 1] = dp4a_us(b1, dq.w, ia1[NS - 1]); ia2[NS - 1] = dp4a_us(b2, dq.w, ia2[NS - 1]); }
                             }
                         } else {
 #pragma unroll
@@ -403,8 +501,16 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                         }
                     }
                 }
-                const double d1 = warp_sum((double)acc1[0] + (double)acc1[1] + (double)lsum);
-                const double d2 = warp_sum((double)acc2[0] + (double)acc2[1] + (double)lsum);
+                double p1, p2;
+                if constexpr (!TABLE) {
+                    p1 = (double)combine_digits<NS>(ia1) * delta_w + (double)lsum;
+                    p2 = (double)combine_digits<NS>(ia2) * delta_w + (double)lsum;
+                } else {
+                    p1 = (double)acc1[0] + (double)acc1[1];
+                    p2 = (double)acc2[0] + (double)acc2[1];
+                }
+                const double d1 = warp_sum(p1);
+                const double d2 = warp_sum(p2);
                 if (lane == 0) {
                     const int r = chunk * a.cr + lr;
                     if (S > 1) {
@@ -416,6 +522,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                         res[2 * r] = r1;
                         res[2 * r + 1] = r2;
                         wsum += (double)r1 + (double)r2;
+                        rmax = fmaxf(rmax, fmaxf(fabsf(r1), fabsf(r2)));
                     } else {
                         ll_store_double(pd_mine + (size_t)r * 4, d1, tag);
                         ll_store_double(pd_mine + (size_t)r * 4 + 2, d2, tag);
@@ -441,6 +548,7 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                         res[2 * lane] = r1;
                         res[2 * lane + 1] = r2;
                         v = (double)r1 + (double)r2;
+                        rmax = fmaxf(fabsf(r1), fabsf(r2));
                     } else {
                         ll_store_double(pd_mine + (size_t)lane * 4, d1, tag);
                         ll_store_double(pd_mine + (size_t)lane * 4 + 2, d2, tag);
@@ -478,11 +586,36 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 res[2 * r] = r1;
                 res[2 * r + 1] = r2;
                 part += (double)r1 + (double)r2;
+                rmax = fmaxf(rmax, fmaxf(fabsf(r1), fabsf(r2)));
             }
             part = warp_sum(part);
             if (lane == 0) sh->red[warp] = part;
         }
-        consumer_sync();                         // residuals and the per-warp residual sums are complete
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+        if (lane == 0) sh->fmax[8 + warp] = rmax;
+        consumer_sync();                         // residuals, their per-warp sums and maxima are complete
+        double delta_r = 0.0;                    // one fixed-point unit of the residuals of this step
+        if constexpr (!TABLE) {
+            float rho = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kRingWarps; ++w) rho = fmaxf(rho, sh->fmax[8 + w]);
+            const float inv = rho > 0.0f ? QMAXF / rho : 0.0f;
+            delta_r = (double)rho / (double)QMAXF;
+            // digit words of the residuals, four rows at a time (rows past the batch count as zero)
+            for (int k4 = threadIdx.x; k4 < (rcnt + 3) / 4; k4 += kRingConsumers) {
+                float v1[4], v2[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int k = 4 * k4 + r;
+                    v1[r] = k < rcnt ? res[2 * k] : 0.0f;
+                    v2[r] = k < rcnt ? res[2 * k + 1] : 0.0f;
+                }
+                rqs[2 * k4] = digit_words<NS>(v1, inv);
+                rqs[2 * k4 + 1] = digit_words<NS>(v2, inv);
+            }
+            consumer_sync();
+        }
         trace_mark(a, it, 1);
 
         // -------------------------------------------------------------- phase B: gradient
@@ -492,6 +625,11 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
             float acc[FPW];
 #pragma unroll
             for (int i = 0; i < FPW; ++i) acc[i] = 0.0f;
+            int ib[TABLE ? 1 : FPW][NS];         // uniform: digit sums per feature of the word
+#pragma unroll
+            for (int i = 0; i < (TABLE ? 1 : FPW); ++i)
+#pragma unroll
+                for (int sidx = 0; sidx < NS; ++sidx) ib[i][sidx] = 0;
             for (int ci = 0; ci < C; ++ci) {
                 const int chunk = C - 1 - ci;
                 const int rows = min(a.cr, rcnt - chunk * a.cr);
@@ -503,20 +641,50 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                 if (active) {
                     const uint32_t* col1 = ring + (size_t)use_slot * slot_words + q;
                     const uint32_t* col2 = col1 + (size_t)a.cr * a.wc;
-                    const float* rr = res + 2 * chunk * a.cr;
-#pragma unroll 4
-                    for (int lr = group; lr < rows; lr += ngroups) {
-                        const uint32_t u1 = col1[(size_t)lr * a.wc];
-                        const uint32_t u2 = col2[(size_t)lr * a.wc];
-                        const float2 rv = *reinterpret_cast<const float2*>(rr + 2 * lr);
-                        const float r1 = rv.x, r2 = rv.y;
-                        if constexpr (!TABLE) {
-                            float c1[FPW], c2[FPW];
-                            unpack_word<CB>(u1, c1);
-                            unpack_word<CB>(u2, c2);
+                    if constexpr (!TABLE) {
+                        // four rows at a time: transpose their codes so that a register holds one feature of
+                        // the four rows, then one dp4a per residual digit (slots hold a multiple of four rows;
+                        // rows past the chunk meet zero digits)
+                        const uint4* rq = rqs + 2 * (chunk * a.cr / 4);
+#pragma unroll 2
+                        for (int l4 = group; l4 < (rows + 3) / 4; l4 += ngroups) {
+                            uint32_t u1[4], u2[4];
 #pragma unroll
-                            for (int i = 0; i < FPW; ++i) acc[i] = fmaf(c1[i], r2, fmaf(c2[i], r1, acc[i]));
-                        } else {
+                            for (int r = 0; r < 4; ++r) {
+                                u1[r] = col1[(size_t)(4 * l4 + r) * a.wc];
+                                u2[r] = col2[(size_t)(4 * l4 + r) * a.wc];
+                            }
+                            const uint4 d1 = rq[2 * l4], d2 = rq[2 * l4 + 1];     // digits of r1, of r2
+#pragma unroll
+                            for (int g = 0; g < NG; ++g) {
+#pragma unroll
+                                for (int pl = 0; pl < 2; ++pl) {
+                                    const uint32_t x0 = group_bytes<CB>(pl ? u2[0] : u1[0], g), x1 = group_bytes<CB>(pl ? u2[1] : u1[1], g);
+                                    const uint32_t x2 = group_bytes<CB>(pl ? u2[2] : u1[2], g), x3 = group_bytes<CB>(pl ? u2[3] : u1[3], g);
+                                    const uint32_t lo01 = __byte_perm(x0, x1, 0x5140), hi01 = __byte_perm(x0, x1, 0x7362);
+                                    const uint32_t lo23 = __byte_perm(x2, x3, 0x5140), hi23 = __byte_perm(x2, x3, 0x7362);
+                                    const uint32_t t[4] = {__byte_perm(lo01, lo23, 0x5410), __byte_perm(lo01, lo23, 0x7632),
+                                                           __byte_perm(hi01, hi23, 0x5410), __byte_perm(hi01, hi23, 0x7632)};
+                                    const uint4 dr = pl ? d1 : d2;             // plane 1 meets r2, plane 2 meets r1
+#pragma unroll
+                                    for (int b = 0; b < 4; ++b) {
+                                        const int f = b * NG + g;
+                                        ib[f][0] = dp4a_us(t[b], dr.x, ib[f][0]);
+                                        ib[f][1] = dp4a_us(t[b], dr.y, ib[f][1]);
+                                        ib[f][2] = dp4a_us(t[b], dr.z, ib[f][2]);
+                                        if constexpr (NS == 4) ib[f][NS - 1] = dp4a_us(t[b], dr.w, ib[f][NS - 1]);
+                                    }
+                                }
+                            }
+                        }
+                    } else {
+                        const float* rr = res + 2 * chunk * a.cr;
+#pragma unroll 4
+                        for (int lr = group; lr < rows; lr += ngroups) {
+                            const uint32_t u1 = col1[(size_t)lr * a.wc];
+                            const uint32_t u2 = col2[(size_t)lr * a.wc];
+                            const float2 rv = *reinterpret_cast<const float2*>(rr + 2 * lr);
+                            const float r1 = rv.x, r2 = rv.y;
 #pragma unroll
                             for (int i = 0; i < FPW; ++i) {
                                 const float l1 = LV[(code_at<CB>(u1, i) * FPW + i) * a.wc + q];
@@ -531,6 +699,10 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
                     if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
                     if (++slot == slots) { slot = 0; phase ^= 1u; }
                 }
+            }
+            if constexpr (!TABLE) {
+#pragma unroll
+                for (int i = 0; i < FPW; ++i) acc[i] = (float)((double)combine_digits<NS>(ib[i]) * delta_r);
             }
             if (ngroups > 1) {
                 consumer_sync();
@@ -664,22 +836,28 @@ __global__ void __launch_bounds__(kRingThreads) sgd_ring_kernel(const SgdArgs a)
 
         // -------------------------------------------------------------- all-gather: the part's model, word by word
         ll_wait_sentinels(ag_part, a.sub, (F + a.sub - 1) / a.sub, tag, sh, a.status, 4);  // each owner's first feature
-        for (int q = threadIdx.x; q < a.wc; q += kRingConsumers) {
-            const unsigned long long* src = ag_part + (size_t)q * FPW;
-            unsigned long long v[FPW];
-            bool ok = false;
-            if (!*reinterpret_cast<volatile int*>(&sh->abort_flag)) {
-                for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
-                    ok = true;
-#pragma unroll
-                    for (int i = 0; i < FPW; ++i) { v[i] = ll_load(src + i); ok = ok && ((uint32_t)(v[i] >> 32) == tag); }
-                }
-                if (!ok) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 4); }
-            }
+        {
+            const int q = threadIdx.x;
+            const bool have = q < a.wc;
             float xt[FPW];
 #pragma unroll
-            for (int i = 0; i < FPW; ++i) xt[i] = ok ? __uint_as_float((uint32_t)v[i]) : 0.0f;
-            build_word(q, xt);
+            for (int i = 0; i < FPW; ++i) xt[i] = 0.0f;
+            if (have) {
+                const unsigned long long* src = ag_part + (size_t)q * FPW;
+                unsigned long long v[FPW];
+                bool ok = false;
+                if (!*reinterpret_cast<volatile int*>(&sh->abort_flag)) {
+                    for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
+                        ok = true;
+#pragma unroll
+                        for (int i = 0; i < FPW; ++i) { v[i] = ll_load(src + i); ok = ok && ((uint32_t)(v[i] >> 32) == tag); }
+                    }
+                    if (!ok) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 4); }
+                }
+#pragma unroll
+                for (int i = 0; i < FPW; ++i) xt[i] = ok ? __uint_as_float((uint32_t)v[i]) : 0.0f;
+            }
+            delta_w = word_stage(have, q, xt);
         }
         {
             float* bnext = bsm + (size_t)(par ^ 1) * a.rc;
@@ -710,6 +888,7 @@ static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int 
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
     bytes += sizeof(float) * ((table ? 2 * L * F : F) + (size_t)wc + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
     bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
+    bytes += 16 * 2 * (size_t)((rc + 3) / 4);
     bytes += sizeof(uint32_t) * (size_t)slots * 2 * cr * wc;
     return bytes;
 }
@@ -743,9 +922,9 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         const bool wide = r.wc > kRingConsumers;
         // chunk: about 32 KiB of codes, at least one row, at most the CTA's rows
         int cr = (int)(32768 / (2 * (size_t)r.wc * 4));
-        cr = cr < 1 ? 1 : cr;
-        cr = cr > r.rc ? r.rc : cr;
-        if (wide) cr = r.rc;
+        cr = (cr + 3) & ~3;                                   // phase B walks a slot four rows at a time
+        cr = cr < 4 ? 4 : cr;
+        if (cr > ((r.rc + 3) & ~3) || wide) cr = (r.rc + 3) & ~3;
         r.cr = cr;
         if (sizeof(uint32_t) * 2 * (size_t)cr * r.wc >= (1u << 20)) return false;   // mbarrier tx-count range
         int slots = kRingMaxSlots;
