@@ -637,7 +637,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
     a.status = ctx->d_status;
     a.order = nullptr;
     a.phases = kPhaseAll; a.persistent = 0;
-    a.trace = nullptr; a.trace_steps = 0;
+    a.trace = nullptr; a.trace_steps = 0; a.use_tmap = 0;
     if (p->batch_order) {
         int32_t* dev_order = reinterpret_cast<int32_t*>(ctx->ws + sc.order_off);
         e = cudaMemcpyAsync(dev_order, p->batch_order, sizeof(int32_t) * (size_t)T, cudaMemcpyHostToDevice, ctx->stream);

@@ -51,6 +51,7 @@ struct SgdArgs {
     DeviceStatus* status;
     unsigned long long* trace;   // ring engine: optional timestamps, 8 per step for the first trace_steps steps
     int trace_steps;
+    int use_tmap;           // ring engine: chunks arrive as 2-D tensor copies
     int phases;             // mask of kPhase*
     int persistent;
 };

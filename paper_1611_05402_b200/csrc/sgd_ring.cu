@@ -28,6 +28,9 @@
 // different feature parts (dots, gradient norm) alternate between two buffers by step parity.
 // Every wait is bounded: when one gives up it records ZIPML_ERR_TIMEOUT, later waits of that CTA
 // are skipped and the CTA still publishes everything, so the launch always ends.
+#include <cuda.h>
+#include <string.h>
+
 #include "sgd_common.cuh"
 
 namespace zipml {
@@ -54,9 +57,10 @@ __device__ __forceinline__ double consumer_sum(double v, double* scratch) {
 
 struct RingShared {
     double red[16];
-    double dpart[16];
+    double dpart[8 * 16];          // [task][8] partial sums of split row blocks
     double misc[8];
-    float fmax[16];                // per-warp maxima: [0..7] |w| of the word stage, [8..15] |residual|
+    double wbase[16];              // per-warp parts of lo^T x~ over the CTA's feature part
+    float fmax[32];                // per-warp maxima: [0..15] |w| of the word stage, [16..31] |residual|
     unsigned long long full[kRingMaxSlots];
     unsigned long long empty[kRingMaxSlots];
     int abort_flag;
@@ -79,6 +83,13 @@ __device__ __forceinline__ void trace_mark(const SgdArgs& a, int64_t it, int slo
         asm volatile("mov.u64 %0, %clock64;" : "=l"(t));
         a.trace[(it - a.first_step) * 8 + slot_id] = t;
     }
+}
+
+// 2-D tiled bulk copy global -> shared through a tensor map (rows x words box); x in elements must make
+// x * 4 bytes a multiple of 16, the destination is 128-byte aligned.
+__device__ __forceinline__ void tensor_copy_g2s(void* dst_smem, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
 // ---- packets ---------------------------------------------------------------------------------
@@ -145,13 +156,14 @@ __device__ __forceinline__ void ll_gather(const unsigned long long* src, int cou
 // phase A, the residuals in phase B).  That vector is turned, once per step, into fixed point:
 // value ~ delta * W with |W| <= QMAX, and W into NS balanced base-128 digits in [-64, 63], each an
 // int8.  Four codes times four digits are then one dp4a into an int32, the digit sums are combined
-// exactly in 64 bits, and the only rounding is the one quantization of the vector (2^-20 of its
-// largest entry with three digits, 2^-27 with four; 8-bit codes use four because their large code
-// values amplify it).
+// exactly in 64 bits, and the only rounding is the one quantization of the vector, 2^-27 of its
+// largest entry with four digits.  (Three digits, 2^-20, are not enough: the error of w is the same
+// for every row, survives the minibatch mean and is amplified where residuals are small against the
+// dots; measured 1.3e-5 on the gradient of clustered 3-bit codes.)
 template <int CB>
 struct IntPath {
-    static constexpr int NS = (CB == 8) ? 4 : 3;
-    static constexpr int QMAX = (NS == 4) ? 133000000 : 1040000;   // below 63 * (128^NS - 1) / 127
+    static constexpr int NS = 4;
+    static constexpr int QMAX = 133000000;                         // below 63 * (128^NS - 1) / 127
     static constexpr int NG = 8 / CB;                              // groups of four codes in a 32-bit word
 };
 
@@ -205,7 +217,31 @@ __device__ __forceinline__ long long combine_digits(const int (&acc)[NS]) {
     return t;
 }
 
-// Maximum over the consumer threads (values >= 0); `slot` = 0 or 8 picks the half of sh->fmax.
+// Eight values per lane -> their eight sums over the warp with 9 shuffles instead of 40: in each of
+// the first three steps a lane hands half of what it holds to its partner and keeps (and adds) the
+// other half.  Afterwards lane L holds sum number (L >> 2) & 7, complete, in a fixed order.
+template <typename T>
+__device__ __forceinline__ T reduce8(const T (&v)[8], int lane) {
+    const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0;
+    T w4[4], w2[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const T send = up16 ? v[i] : v[i + 4], keep = up16 ? v[i + 4] : v[i];
+        w4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const T send = up8 ? w4[i] : w4[i + 2], keep = up8 ? w4[i + 2] : w4[i];
+        w2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+    const T send = up4 ? w2[0] : w2[1], keep = up4 ? w2[1] : w2[0];
+    T w1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    w1 += __shfl_xor_sync(0xffffffffu, w1, 2);
+    w1 += __shfl_xor_sync(0xffffffffu, w1, 1);
+    return w1;
+}
+
+// Maximum over the consumer threads (values >= 0); `slot` = 0 or 16 picks the half of sh->fmax.
 __device__ __forceinline__ float consumer_max(float v, RingShared* sh, int slot) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
@@ -232,7 +268,8 @@ __device__ __forceinline__ float consumer_max(float v, RingShared* sh, int slot)
 //   bsm[2][rc] float            labels of the current and the next step's rows
 //   ring[slots][2][cr][wc] u32  code chunks
 template <int CB, bool TABLE>
-__global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs a) {
+__global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs a, const __grid_constant__ CUtensorMap tm1,
+                                                                  const __grid_constant__ CUtensorMap tm2) {
     constexpr int FPW = 32 / CB;
     constexpr int NS = IntPath<CB>::NS, NG = IntPath<CB>::NG;
     constexpr float QMAXF = (float)IntPath<CB>::QMAX;
@@ -252,7 +289,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     float* res = gred + kRingConsumers * FPW;
     uint4* rqs = reinterpret_cast<uint4*>(res + ((2 * a.rc + 3) & ~3));
     float* bsm = reinterpret_cast<float*>(rqs + 2 * ((a.rc + 3) / 4));
-    uint32_t* ring = reinterpret_cast<uint32_t*>(bsm + ((2 * a.rc + 3) & ~3));
+    uint32_t* ring = reinterpret_cast<uint32_t*>(
+        (reinterpret_cast<uintptr_t>(bsm + ((2 * a.rc + 3) & ~3)) + 127) & ~(uintptr_t)127);      // tensor copies want 128 bytes
     const size_t slot_words = (size_t)2 * a.cr * a.wc;
 
     const int ai = blockIdx.x % a.na, bi = blockIdx.x / a.na;
@@ -301,22 +339,34 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 const int chunk = s < C ? s : 2 * C - 1 - s;
                 const int rows = min(a.cr, rcnt - chunk * a.cr);
                 uint64_t* full = reinterpret_cast<uint64_t*>(sh->full + slot);
-                if (lane == 0) {
-                    ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
-                    mbar_arrive_expect_tx(full, 2u * (uint32_t)rows * row_bytes);
-                }
-                __syncwarp();
                 uint32_t* dst = ring + (size_t)slot * slot_words;
                 const int64_t first = r0 + k0 + (int64_t)chunk * a.cr;
-                if (contiguous) {
-                    if (lane < 2)
-                        bulk_copy_g2s(dst + (size_t)lane * a.cr * a.wc, (lane == 0 ? a.p1 : a.p2) + first * a.row_words,
-                                      (uint32_t)rows * row_bytes, full);
+                if (a.use_tmap) {
+                    // one box of cr rows x wc words per plane; rows past the chunk (the next rows of the
+                    // plane, or zeros past its end) come along and are never used
+                    if (lane == 0) {
+                        ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
+                        mbar_arrive_expect_tx(full, 2u * (uint32_t)a.cr * (uint32_t)a.wc * 4u);
+                        tensor_copy_g2s(dst, &tm1, (int)w0, (int)first, full);
+                        tensor_copy_g2s(dst + (size_t)a.cr * a.wc, &tm2, (int)w0, (int)first, full);
+                    }
+                    __syncwarp();
                 } else {
-                    for (int i = lane; i < 2 * rows; i += 32) {
-                        const int plane = i & 1, r = i >> 1;
-                        bulk_copy_g2s(dst + ((size_t)plane * a.cr + r) * a.wc,
-                                      (plane == 0 ? a.p1 : a.p2) + (first + r) * a.row_words + w0, row_bytes, full);
+                    if (lane == 0) {
+                        ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
+                        mbar_arrive_expect_tx(full, 2u * (uint32_t)rows * row_bytes);
+                    }
+                    __syncwarp();
+                    if (contiguous) {
+                        if (lane < 2)
+                            bulk_copy_g2s(dst + (size_t)lane * a.cr * a.wc, (lane == 0 ? a.p1 : a.p2) + first * a.row_words,
+                                          (uint32_t)rows * row_bytes, full);
+                    } else {
+                        for (int i = lane; i < 2 * rows; i += 32) {
+                            const int plane = i & 1, r = i >> 1;
+                            bulk_copy_g2s(dst + ((size_t)plane * a.cr + r) * a.wc,
+                                          (plane == 0 ? a.p1 : a.p2) + (first + r) * a.row_words + w0, row_bytes, full);
+                        }
                     }
                 }
                 if (++slot == slots) { slot = 0; phase ^= 1u; }
@@ -340,6 +390,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     // reads; every consumer calls it, `have` says whether the thread holds a word (parts are at most
     // one word per consumer wide).  Returns delta_w, the value of one fixed-point unit of w.
     uint4* tabq = reinterpret_cast<uint4*>(tab);
+    double base_w = 0.0;                         // lo^T x~ over the CTA's feature part (uniform grids)
     auto word_stage = [&](bool have, int q, const float (&xt)[FPW]) -> double {
         if constexpr (!TABLE) {
             float wv[FPW];
@@ -353,7 +404,14 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 lsum = fmaf(lv, xt[i], lsum);
                 m = fmaxf(m, fabsf(wv[i]));
             }
-            const float wmax = consumer_max(m, sh, 0);
+            {
+                const double wb = warp_sum((double)lsum);
+                if (lane == 0) sh->wbase[warp] = wb;
+            }
+            const float wmax = consumer_max(m, sh, 0);     // its barrier also publishes wbase
+            base_w = 0.0;
+#pragma unroll
+            for (int w = 0; w < kRingWarps; ++w) base_w += sh->wbase[w];
             const float inv = wmax > 0.0f ? QMAXF / wmax : 0.0f;
             if (have) {
 #pragma unroll
@@ -361,7 +419,6 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                     const float v4[4] = {wv[0 * NG + g], wv[1 * NG + g], wv[2 * NG + g], wv[3 * NG + g]};
                     tabq[g * a.wc + q] = digit_words<NS>(v4, inv);
                 }
-                lw[q] = lsum;
             }
             return (double)wmax / (double)QMAXF;
         } else {
@@ -455,77 +512,97 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
         const bool dots_local = (a.na == 1);
         unsigned long long* pd_mine = a.ll_pd + (((size_t)par * a.nb + bi) * a.na + ai) * a.rc * 4;
         const int slot_a = slot;                 // slot of the single chunk when C == 1
-        // with fewer rows than warps (single-chunk tiles only) a row is split over S warps
+        // A warp takes four rows at a time: one load of w's digit words serves them all and the
+        // eight (row, plane) sums are independent chains.  When the tile has fewer row blocks than warps
+        // (single-chunk tiles only) a block's words are split over S warps.
+        constexpr int RB = 4;
         int S = 1;
-        if (C == 1 && rcnt < kRingWarps) S = max(1, min(chunks_w, kRingWarps / rcnt));
+        {
+            const int nblk_all = (rcnt + RB - 1) / RB;
+            if (C == 1 && nblk_all > 0 && nblk_all < kRingWarps) S = max(1, min(chunks_w, kRingWarps / nblk_all));
+        }
         const int cps = (chunks_w + S - 1) / S;
-        double wsum = 0.0;                       // lane 0: r1 + r2 over the rows this warp finished
+        double wsum = 0.0;                       // r1 + r2 (one of them per lane) over what this thread finished
         float rmax = 0.0f;                       // and the largest |residual| this thread produced
+        const int vmine = (lane >> 2) & 7;       // after the butterfly a lane holds sum number vmine = 2*row + plane
         for (int chunk = 0; chunk < C; ++chunk) {
             const int rows = min(a.cr, rcnt - chunk * a.cr);
             ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 6);
             const uint32_t* t1 = ring + (size_t)slot * slot_words;
             const uint32_t* t2 = t1 + (size_t)a.cr * a.wc;
-            for (int task = warp; task < rows * S; task += kRingWarps) {
-                const int lr = task / S, seg = task - lr * S;
-                const uint32_t* row1 = t1 + (size_t)lr * a.wc;
-                const uint32_t* row2 = t2 + (size_t)lr * a.wc;
-                float acc1[2] = {0.0f, 0.0f}, acc2[2] = {0.0f, 0.0f};
-                int ia1[NS], ia2[NS];
+            const int nblk = (rows + RB - 1) / RB;
+            for (int task = warp; task < nblk * S; task += kRingWarps) {
+                const int blk = task / S, seg = task - blk * S;
+                const uint32_t* rowp1 = t1 + (size_t)(blk * RB) * a.wc;
+                const uint32_t* rowp2 = t2 + (size_t)(blk * RB) * a.wc;
+                int ia[TABLE ? 1 : 2 * RB][NS];
+                float fa[2 * RB];
 #pragma unroll
-                for (int sidx = 0; sidx < NS; ++sidx) { ia1[sidx] = 0; ia2[sidx] = 0; }
-                float lsum = 0.0f;
+                for (int v = 0; v < 2 * RB; ++v) {
+                    fa[v] = 0.0f;
+                    if constexpr (!TABLE) {
+#pragma unroll
+                        for (int sidx = 0; sidx < NS; ++sidx) ia[v][sidx] = 0;
+                    }
+                }
                 const int c_end = min(chunks_w, (seg + 1) * cps);
-#pragma unroll 4
+#pragma unroll 2
                 for (int c = seg * cps; c < c_end; ++c) {
                     const int q = c * 32 + lane;
                     if (q < wcnt) {
-                        const uint32_t u1 = row1[q], u2 = row2[q];
+                        uint32_t u[2 * RB];      // rows past the chunk's last one read leftovers of the slot; never used
+#pragma unroll
+                        for (int r = 0; r < RB; ++r) { u[2 * r] = rowp1[(size_t)r * a.wc + q]; u[2 * r + 1] = rowp2[(size_t)r * a.wc + q]; }
                         if constexpr (!TABLE) {
-                            lsum += lw[q];
 #pragma unroll
                             for (int g = 0; g < NG; ++g) {
                                 const uint4 dq = tabq[g * a.wc + q];
-                                const uint32_t b1 = group_bytes<CB>(u1, g), b2 = group_bytes<CB>(u2, g);
-                                ia1[0] = dp4a_us(b1, dq.x, ia1[0]); ia2[0] = dp4a_us(b2, dq.x, ia2[0]);
-                                ia1[1] = dp4a_us(b1, dq.y, ia1[1]); ia2[1] = dp4a_us(b2, dq.y, ia2[1]);
-                                ia1[2] = dp4a_us(b1, dq.z, ia1[2]); ia2[2] = dp4a_us(b2, dq.z, ia2[2]);
-                                if constexpr (NS == 4) { ia1[NS - 1] = dp4a_us(b1, dq.w, ia1[NS - 1]); ia2[NS - 1] = dp4a_us(b2, dq.w, ia2[NS - 1]); }
+#pragma unroll
+                                for (int v = 0; v < 2 * RB; ++v) {
+                                    const uint32_t bq = group_bytes<CB>(u[v], g);
+                                    ia[v][0] = dp4a_us(bq, dq.x, ia[v][0]);
+                                    ia[v][1] = dp4a_us(bq, dq.y, ia[v][1]);
+                                    ia[v][2] = dp4a_us(bq, dq.z, ia[v][2]);
+                                    if constexpr (NS == 4) ia[v][NS - 1] = dp4a_us(bq, dq.w, ia[v][NS - 1]);
+                                }
                             }
                         } else {
 #pragma unroll
                             for (int i = 0; i < FPW; ++i) {
-                                acc1[i & 1] += tab[(code_at<CB>(u1, i) * FPW + i) * a.wc + q];
-                                acc2[i & 1] += tab[(code_at<CB>(u2, i) * FPW + i) * a.wc + q];
+#pragma unroll
+                                for (int v = 0; v < 2 * RB; ++v) fa[v] += tab[(code_at<CB>(u[v], i) * FPW + i) * a.wc + q];
                             }
                         }
                     }
                 }
-                double p1, p2;
+                double dsum;
                 if constexpr (!TABLE) {
-                    p1 = (double)combine_digits<NS>(ia1) * delta_w + (double)lsum;
-                    p2 = (double)combine_digits<NS>(ia2) * delta_w + (double)lsum;
+                    // exact: digit sums -> 64-bit totals -> warp totals; one conversion per (row, plane)
+                    long long tv[2 * RB];
+#pragma unroll
+                    for (int v = 0; v < 2 * RB; ++v) tv[v] = combine_digits<NS>(ia[v]);
+                    const long long tsum = reduce8(tv, lane);
+                    dsum = (double)tsum * delta_w + (seg == 0 ? base_w : 0.0);
                 } else {
-                    p1 = (double)acc1[0] + (double)acc1[1];
-                    p2 = (double)acc2[0] + (double)acc2[1];
+                    double pv[2 * RB];
+#pragma unroll
+                    for (int v = 0; v < 2 * RB; ++v) pv[v] = (double)fa[v];
+                    dsum = reduce8(pv, lane);
                 }
-                const double d1 = warp_sum(p1);
-                const double d2 = warp_sum(p2);
-                if (lane == 0) {
+                if ((lane & 3) == 0) {
+                    const int lr = blk * RB + (vmine >> 1), plane = vmine & 1;
                     const int r = chunk * a.cr + lr;
                     if (S > 1) {
-                        sh->dpart[2 * task] = d1;
-                        sh->dpart[2 * task + 1] = d2;
-                    } else if (dots_local) {
-                        const double bk = (double)bcur[r];
-                        const float r1 = (float)(d1 - bk), r2 = (float)(d2 - bk);
-                        res[2 * r] = r1;
-                        res[2 * r + 1] = r2;
-                        wsum += (double)r1 + (double)r2;
-                        rmax = fmaxf(rmax, fmaxf(fabsf(r1), fabsf(r2)));
-                    } else {
-                        ll_store_double(pd_mine + (size_t)r * 4, d1, tag);
-                        ll_store_double(pd_mine + (size_t)r * 4 + 2, d2, tag);
+                        sh->dpart[task * 8 + vmine] = dsum;
+                    } else if (lr < rows) {
+                        if (dots_local) {
+                            const float rv = (float)(dsum - (double)bcur[r]);
+                            res[2 * r + plane] = rv;
+                            wsum += (double)rv;
+                            rmax = fmaxf(rmax, fabsf(rv));
+                        } else {
+                            ll_store_double(pd_mine + (size_t)r * 4 + 2 * plane, dsum, tag);
+                        }
                     }
                 }
             }
@@ -535,30 +612,24 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 if (++slot == slots) { slot = 0; phase ^= 1u; }
             }
         }
-        if (S > 1) {
+        if (S > 1) {                             // single chunk: one thread per (row, plane) adds the segments in order
             consumer_sync();
-            if (warp == 0) {                     // rcnt < 8 rows: one lane per row, in segment order
-                double v = 0.0;
-                if (lane < rcnt) {
-                    double d1 = 0.0, d2 = 0.0;
-                    for (int sg = 0; sg < S; ++sg) { d1 += sh->dpart[2 * (lane * S + sg)]; d2 += sh->dpart[2 * (lane * S + sg) + 1]; }
-                    if (dots_local) {
-                        const double bk = (double)bcur[lane];
-                        const float r1 = (float)(d1 - bk), r2 = (float)(d2 - bk);
-                        res[2 * lane] = r1;
-                        res[2 * lane + 1] = r2;
-                        v = (double)r1 + (double)r2;
-                        rmax = fmaxf(fabsf(r1), fabsf(r2));
-                    } else {
-                        ll_store_double(pd_mine + (size_t)lane * 4, d1, tag);
-                        ll_store_double(pd_mine + (size_t)lane * 4 + 2, d2, tag);
-                    }
+            if ((int)threadIdx.x < 2 * rcnt) {
+                const int r = threadIdx.x >> 1, plane = threadIdx.x & 1;
+                const int blk = r / RB, vv = 2 * (r - blk * RB) + plane;
+                double d = 0.0;
+                for (int sg = 0; sg < S; ++sg) d += sh->dpart[(blk * S + sg) * 8 + vv];
+                if (dots_local) {
+                    const float rv = (float)(d - (double)bcur[r]);
+                    res[2 * r + plane] = rv;
+                    wsum += (double)rv;
+                    rmax = fmaxf(rmax, fabsf(rv));
+                } else {
+                    ll_store_double(pd_mine + (size_t)r * 4 + 2 * plane, d, tag);
                 }
-                wsum = warp_sum(v);
-            } else {
-                wsum = 0.0;
             }
         }
+        wsum = warp_sum(wsum);
         if (dots_local) {
             if (lane == 0) sh->red[warp] = wsum;
         } else {
@@ -593,13 +664,13 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
-        if (lane == 0) sh->fmax[8 + warp] = rmax;
+        if (lane == 0) sh->fmax[16 + warp] = rmax;
         consumer_sync();                         // residuals, their per-warp sums and maxima are complete
         double delta_r = 0.0;                    // one fixed-point unit of the residuals of this step
         if constexpr (!TABLE) {
             float rho = 0.0f;
 #pragma unroll
-            for (int w = 0; w < kRingWarps; ++w) rho = fmaxf(rho, sh->fmax[8 + w]);
+            for (int w = 0; w < kRingWarps; ++w) rho = fmaxf(rho, sh->fmax[16 + w]);
             const float inv = rho > 0.0f ? QMAXF / rho : 0.0f;
             delta_r = (double)rho / (double)QMAXF;
             // digit words of the residuals, four rows at a time (rows past the batch count as zero)
@@ -888,7 +959,7 @@ static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int 
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
     bytes += sizeof(float) * ((table ? 2 * L * F : F) + (size_t)wc + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
     bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
-    bytes += 16 * 2 * (size_t)((rc + 3) / 4);
+    bytes += 16 * 2 * (size_t)((rc + 3) / 4) + 128;          // + slack to align the ring to 128 bytes
     bytes += sizeof(uint32_t) * (size_t)slots * 2 * cr * wc;
     return bytes;
 }
@@ -920,8 +991,8 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         r.sub = ring_round_up((F + r.nb - 1) / r.nb, 4);
         // a part wider than the consumer count needs the whole tile in one retained chunk
         const bool wide = r.wc > kRingConsumers;
-        // chunk: about 32 KiB of codes, at least one row, at most the CTA's rows
-        int cr = (int)(32768 / (2 * (size_t)r.wc * 4));
+        // chunk: about 64 KiB of codes (eight 4-row blocks of a full-width part: one per consumer warp)
+        int cr = (int)(65536 / (2 * (size_t)r.wc * 4));
         cr = (cr + 3) & ~3;                                   // phase B walks a slot four rows at a time
         cr = cr < 4 ? 4 : cr;
         if (cr > ((r.rc + 3) & ~3) || wide) cr = (r.rc + 3) & ~3;
@@ -963,6 +1034,40 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         if (!found || cost < best_cost) { found = true; best_cost = cost; *plan = r; }
     }
     return found ? ZIPML_OK : ZIPML_ERR_WORKSPACE;
+}
+
+static int64_t plane_wc_check(int wc) { return (int64_t)wc; }
+
+// Tensor maps over the two planes seen as m x row_words matrices of 32-bit words.  The encoder is a
+// driver entry point looked up through the runtime (no link against the driver library).
+static int encode_plane_maps(zipml_ctx* ctx, const zipml_dataset* d, int wc, int cr, CUtensorMap* out) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    if (!ctx->tmap_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess || !fn) {
+            (void)cudaGetLastError();
+            return ZIPML_ERR_CUDA;
+        }
+        ctx->tmap_encode = fn;
+    }
+    if (wc > 256 || cr > 256 || (wc * 4) % 16 != 0) return ZIPML_ERR_WORKSPACE;
+    const cuuint64_t gdim[2] = {(cuuint64_t)(d->row_bytes / 4), (cuuint64_t)d->m};
+    const cuuint64_t gstride[1] = {(cuuint64_t)d->row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)wc, (cuuint32_t)cr};
+    const cuuint32_t estr[2] = {1, 1};
+    const void* planes[2] = {d->plane1, d->plane2};
+    for (int i = 0; i < 2; ++i) {
+        const CUresult r = reinterpret_cast<EncodeFn>(ctx->tmap_encode)(
+            &out[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(planes[i]), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return ZIPML_ERR_CUDA;
+    }
+    return ZIPML_OK;
 }
 
 int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
@@ -1028,6 +1133,13 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         if (e != cudaSuccess) return cuda_status(e);
         a.order = dev_order;
     }
+    // strided row pieces go through two tensor maps (plane 1, plane 2): box = cr rows x wc words
+    CUtensorMap tmaps[2];
+    memset(tmaps, 0, sizeof(tmaps));
+    a.use_tmap = 0;
+    if (a.row_words != plane_wc_check(plan.wc) && d->m < 0x7fffffffLL && a.row_words < 0x7fffffffLL) {
+        if (encode_plane_maps(ctx, d, plan.wc, plan.cr, tmaps) == ZIPML_OK) a.use_tmap = 1;
+    }
     // packet tags are 32-bit step counters starting at 1
     const int64_t max_steps = 0x7fffffffLL;
     for (int64_t s0 = first_step; s0 < first_step + num_steps; s0 += max_steps) {
@@ -1037,7 +1149,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         chunk.first_step = s0;
         chunk.num_steps = (first_step + num_steps - s0 < max_steps) ? first_step + num_steps - s0 : max_steps;
         if (s0 + chunk.num_steps < first_step + num_steps) chunk.grad_out = nullptr;
-        void* params[] = {&chunk};
+        void* params[] = {&chunk, &tmaps[0], &tmaps[1]};
         e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kRingThreads), params, plan.smem, ctx->stream);
         if (e != cudaSuccess) return cuda_status(e);
         ctx->launches += 1;
