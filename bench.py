@@ -114,11 +114,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
     ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
-    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring"])
     ap.add_argument("--feature-parts", type=int, default=0)
     ap.add_argument("--row-parts", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", dest="others", action="store_false",
+                    help="skip the brief epoch timings of the other workloads (N = 1 only)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -176,29 +178,36 @@ def main():
         dist.barrier()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT}[args.engine]
+    engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT,
+              "ring": binding.ENGINE_RING}[args.engine]
 
     w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
     ctx = binding.Context(dev)
     loss_dev = torch.zeros(1, dtype=torch.float64, device=dev)
     kw = dict(model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed, engine=engine,
               grid_feature_parts=args.feature_parts, grid_row_parts=args.row_parts)
-    epoch_events = []
+    epoch_events, quant_events, loss_events = [], [], []
+
+    def timed(events, record, fn):
+        if not record:
+            return fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = fn()
+        e1.record()
+        events.append((e0, e1))
+        return out
 
     def one_pass(record):
-        levels = ctx.zipml_optimal_levels(A, w.bits, w.hist_bins) if w.levels == "optimal" else None
-        ds = ctx.zipml_quantize(A, w.bits, seed=w.seed, level_mode=binding.LEVELS_TABLE if levels is not None else
-                                binding.LEVELS_UNIFORM, levels=levels)
+        def quant():
+            levels = ctx.zipml_optimal_levels(A, w.bits, w.hist_bins) if w.levels == "optimal" else None
+            return ctx.zipml_quantize(A, w.bits, seed=w.seed, level_mode=binding.LEVELS_TABLE if levels is not None else
+                                      binding.LEVELS_UNIFORM, levels=levels)
+        ds = timed(quant_events, record, quant)
         x = torch.zeros(w.n, dtype=torch.float32, device=dev)
         for ep in range(w.epochs):
-            if record:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-            ctx.zipml_sgd_epoch(ds, b, x, w.batch, w.lr, epoch=ep, **kw)
-            if record:
-                e1.record()
-                epoch_events.append((e0, e1))
-        ctx.zipml_loss(binding.LOSS_DENSE, b, x, A=A, out=loss_dev)
+            timed(epoch_events, record, lambda: ctx.zipml_sgd_epoch(ds, b, x, w.batch, w.lr, epoch=ep, **kw))
+        timed(loss_events, record, lambda: ctx.zipml_loss(binding.LOSS_DENSE, b, x, A=A, out=loss_dev))
         return ds, x
 
     def fence():
@@ -236,11 +245,28 @@ def main():
     packed_bytes = ds.packed_bytes
     peak, peak_kind = measured_peaks()
     achieved = packed_bytes / (epoch_avg_ms * 1e-3) / 1e9
+    steps_per_epoch = (w.m + w.batch - 1) // w.batch
+    step_us = 1e3 * epoch_avg_ms / steps_per_epoch
+    step_bytes = packed_bytes / steps_per_epoch
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None, "peak_kind": f"of {peak_kind} copy rate", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": "sgd_kernel (one launch per epoch)", "algorithmic_bytes_per_launch": packed_bytes,
+                "kernel": "sgd_ring_kernel (one cooperative launch per epoch)", "algorithmic_bytes_per_launch": packed_bytes,
                 "launch_ms_avg": epoch_avg_ms, "launch_ms_min": epoch_ms[0],
-                "epoch_samples_per_s": w.m / (epoch_avg_ms * 1e-3)}
+                "epoch_samples_per_s": w.m / (epoch_avg_ms * 1e-3),
+                # the minibatch chain is sequential: a step moves step_bytes and cannot start before the previous
+                # step's model exists, so the epoch is bound by steps * (exchange latency), not by bytes / bandwidth
+                "steps_per_launch": steps_per_epoch, "us_per_step": step_us, "bytes_per_step": step_bytes,
+                "us_per_step_at_hbm_peak": step_bytes / (peak * 1e3)}
+
+    def stage(events, nbytes):
+        ms_ = sorted(a_.elapsed_time(b_) for a_, b_ in events)
+        avg = sum(ms_) / len(ms_)
+        return {"ms": avg, "GB/s": nbytes / (avg * 1e-3) / 1e9, "frac_of_copy_rate": nbytes / (avg * 1e-3) / 1e9 / peak,
+                "algorithmic_bytes": nbytes}
+    a_bytes = 4 * w.m * w.n
+    stages = {"quantize" + ("+levels" if w.levels == "optimal" else ""):
+              stage(quant_events, a_bytes * (2 if w.levels != "optimal" else 4) + 2 * ds.m * ds.row_bytes),
+              "loss_dense": stage(loss_events, a_bytes + 4 * w.m)}
 
     # ------------------------------------------------------------------ end to end from host buffers
     e2e = None
@@ -270,6 +296,46 @@ def main():
                "d2h_bytes_per_step": int(xh.numel() * 4 + 8), "steps": k_e2e, "loss": e2e_loss}
         del Ah
 
+    # ------------------------------------------------------------------ the other workloads, briefly
+    others = None
+    if world == 1 and args.others:
+        others = {}
+        del A
+        torch.cuda.empty_cache()
+        for key in [k for k in ("c1", "c3", "c4", "c5") if k != args.workload]:
+            wo, Ao, bo, _ = synth.make(key, device=dev)
+            lev = ctx.zipml_optimal_levels(Ao, wo.bits, wo.hist_bins) if wo.levels == "optimal" else None
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record()
+            dso = ctx.zipml_quantize(Ao, wo.bits, seed=wo.seed, levels=lev,
+                                     level_mode=binding.LEVELS_TABLE if lev is not None else binding.LEVELS_UNIFORM)
+            q1.record()
+            xo = torch.zeros(wo.n, dtype=torch.float32, device=dev)
+            kwo = dict(model_bits=wo.model_bits, grad_bits=wo.grad_bits, seed=wo.seed, engine=engine)
+            ctx.zipml_sgd_epoch(dso, bo, xo, wo.batch, wo.lr, epoch=0, **kwo)
+            evs = []
+            for ep in range(1, 4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                ctx.zipml_sgd_epoch(dso, bo, xo, wo.batch, wo.lr, epoch=ep, **kwo)
+                e1.record()
+                evs.append((e0, e1))
+            l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            lc = torch.zeros(1, dtype=torch.float64, device=dev)
+            l0.record()
+            ctx.zipml_loss(binding.LOSS_CODES, bo, xo, data=dso, out=lc)
+            l1.record()
+            ctx.zipml_sync()
+            t_ep = min(a_.elapsed_time(b_) for a_, b_ in evs)
+            To = (wo.m + wo.batch - 1) // wo.batch
+            others[key] = {"workload": wo.name, "epoch_ms": t_ep, "us_per_step": 1e3 * t_ep / To,
+                           "samples_per_s": wo.m / (t_ep * 1e-3), "packed_GB/s": dso.packed_bytes / (t_ep * 1e-3) / 1e9,
+                           "frac_of_copy_rate": dso.packed_bytes / (t_ep * 1e-3) / 1e9 / peak,
+                           "quantize_GB/s": (8 * wo.m * wo.n + 2 * dso.m * dso.row_bytes) / (q0.elapsed_time(q1) * 1e-3) / 1e9,
+                           "loss_codes_GB/s": dso.packed_bytes / (l0.elapsed_time(l1) * 1e-3) / 1e9}
+            del Ao, dso, bo, xo
+            torch.cuda.empty_cache()
+
     # ------------------------------------------------------------------ the oracle beside it
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -291,7 +357,7 @@ def main():
                        "multi_gpu": "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline, "final_loss": final_loss,
-            "packed_gb_per_s_per_epoch": achieved,
+            "packed_gb_per_s_per_epoch": achieved, "stages": stages, "other_workloads": others,
         }))
     if world > 1:
         dist.destroy_process_group()
