@@ -88,7 +88,10 @@ typedef struct zipml_sgd_params {
     int32_t trace_steps;        /* profiling: number of steps to trace (0 = none)                    */
     uint64_t* trace;            /* profiling, DEVICE pointer or NULL: 8 uint64 per traced step; CTA 0
                                    stores its SM's cycle counter at the step's phase boundaries
-                                   (ring engine only)                                                */
+                                   (ring engine only): 0 step start, 1 residuals ready, 2 gradient
+                                   parts published, 3 own sub-slice collected, 4 model updated,
+                                   5 model published, 6 all owners' packets seen, 7 step end (the
+                                   last step of a call stops after mark 4)                            */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

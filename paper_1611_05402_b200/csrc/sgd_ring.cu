@@ -907,6 +907,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
 
         // -------------------------------------------------------------- all-gather: the part's model, word by word
         ll_wait_sentinels(ag_part, a.sub, (F + a.sub - 1) / a.sub, tag, sh, a.status, 4);  // each owner's first feature
+        trace_mark(a, it, 6);
         {
             const int q = threadIdx.x;
             const bool have = q < a.wc;
@@ -936,7 +937,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             for (int r = threadIdx.x + kRingConsumers; r < rcnt_next; r += kRingConsumers) bnext[r] = __ldg(a.b + r0_next + k0 + r);
         }
         consumer_sync();
-        trace_mark(a, it, 6);
+        trace_mark(a, it, 7);
     }
     consumer_sync();
     // every owner returns its sub-slice of the master model
