@@ -49,8 +49,10 @@ enum {
     ZIPML_ENGINE_AUTO = 0,
     ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
     ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
-    ZIPML_ENGINE_RING = 3        /* one cooperative launch; producer warp streams code chunks through a
+    ZIPML_ENGINE_RING = 3,       /* one cooperative launch; producer warp streams code chunks through a
                                     shared-memory ring, gradients meet by reduce-scatter / all-gather  */
+    ZIPML_ENGINE_LEAN = 4        /* one cooperative launch for small minibatch tiles: row parts only,
+                                    two barriers and two packet exchanges per step                    */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -88,10 +90,13 @@ typedef struct zipml_sgd_params {
     int32_t trace_steps;        /* profiling: number of steps to trace (0 = none)                    */
     uint64_t* trace;            /* profiling, DEVICE pointer or NULL: 8 uint64 per traced step; CTA 0
                                    stores its SM's cycle counter at the step's phase boundaries
-                                   (ring engine only): 0 step start, 1 residuals ready, 2 gradient
-                                   parts published, 3 own sub-slice collected, 4 model updated,
-                                   5 model published, 6 all owners' packets seen, 7 step end (the
-                                   last step of a call stops after mark 4)                            */
+                                   Ring engine: 0 step start, 1 residuals ready, 2 gradient parts
+                                   published, 3 own sub-slice collected, 4 model updated, 5 model
+                                   published, 6 all owners' packets seen, 7 step end.  Lean engine:
+                                   0 step start, 1 tile arrived, 2 residuals ready, 3 gradient
+                                   parts sent, 4 own features summed, 5 model published, 6 model
+                                   collected, 7 step end.  The last step of a call stops after
+                                   mark 4.  Other engines ignore the request.                         */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

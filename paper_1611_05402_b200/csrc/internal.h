@@ -74,6 +74,8 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
 
 int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                     int64_t first_step, int64_t num_steps, float* grad_out, bool probe_only);
+int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                    int64_t first_step, int64_t num_steps, float* grad_out);
 int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                      int64_t first_step, int64_t num_steps, float* grad_out);
