@@ -114,7 +114,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
     ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
-    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster"])
     ap.add_argument("--feature-parts", type=int, default=0)
     ap.add_argument("--row-parts", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -179,7 +179,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT,
-              "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN}[args.engine]
+              "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN, "cluster": binding.ENGINE_CLUSTER}[args.engine]
 
     w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
     ctx = binding.Context(dev)

@@ -51,8 +51,10 @@ enum {
     ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
     ZIPML_ENGINE_RING = 3,       /* one cooperative launch; producer warp streams code chunks through a
                                     shared-memory ring, gradients meet by reduce-scatter / all-gather  */
-    ZIPML_ENGINE_LEAN = 4        /* one cooperative launch for small minibatch tiles: row parts only,
+    ZIPML_ENGINE_LEAN = 4,       /* one cooperative launch for small minibatch tiles: row parts only,
                                     two barriers and two packet exchanges per step                    */
+    ZIPML_ENGINE_CLUSTER = 5     /* one thread-block cluster (at most 16 row parts) for small tiles:
+                                    gradients and model travel between the CTAs' shared memories      */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -92,7 +94,8 @@ typedef struct zipml_sgd_params {
                                    stores its SM's cycle counter at the step's phase boundaries
                                    Ring engine: 0 step start, 1 residuals ready, 2 gradient parts
                                    published, 3 own sub-slice collected, 4 model updated, 5 model
-                                   published, 6 all owners' packets seen, 7 step end.  Lean engine:
+                                   published, 6 all owners' packets seen, 7 step end.  Lean and
+                                   cluster engines:
                                    0 step start, 1 tile arrived, 2 residuals ready, 3 gradient
                                    parts sent, 4 own features summed, 5 model published, 6 model
                                    collected, 7 step end.  The last step of a call stops after

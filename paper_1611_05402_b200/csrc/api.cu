@@ -196,7 +196,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (!b || !x || params->batch <= 0) return ZIPML_ERR_INVALID_ARG;
     if (params->model_bits != 0 && (params->model_bits < 2 || params->model_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
     if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
-    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_LEAN) return ZIPML_ERR_INVALID_ARG;
+    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_CLUSTER) return ZIPML_ERR_INVALID_ARG;
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
@@ -210,6 +210,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (!guard.ok) return ZIPML_ERR_CUDA;
     if (params->engine == ZIPML_ENGINE_RING) return launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_LEAN) return launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
+    if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_AUTO) {
         rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
         if (rc != ZIPML_ERR_WORKSPACE) return rc;

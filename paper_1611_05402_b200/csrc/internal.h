@@ -76,6 +76,8 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
                     int64_t first_step, int64_t num_steps, float* grad_out, bool probe_only);
 int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                     int64_t first_step, int64_t num_steps, float* grad_out);
+int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                       int64_t first_step, int64_t num_steps, float* grad_out);
 int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                      int64_t first_step, int64_t num_steps, float* grad_out);

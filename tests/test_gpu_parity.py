@@ -144,7 +144,7 @@ GRIDS = [(0, 0), (1, 1), (1, 5), (2, 3), (3, 1)]
 
 
 @pytest.mark.parametrize("case", SGD_CASES, ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
-@pytest.mark.parametrize("engine", [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN])
+@pytest.mark.parametrize("engine", [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER])
 def test_sgd_epoch_parity(ctx, case, engine):
     key, m, n, bits, batch, lr = case
     _, A, b, _ = workload(key, m, n, seed=1)
@@ -200,7 +200,7 @@ def test_sgd_table_levels_parity(ctx):
     gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
     x0 = np.zeros(100, np.float32)
     x_ref, g_ref = oracle.sgd_epoch(ods, b, x0, 512, 1e-2, want_grad=True)
-    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN):
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER):
         for fa, fb in GRIDS:
             x = to_dev(x0, ctx)
             g = torch.zeros((2, 100), dtype=torch.float32, device=ctx.device)
@@ -228,7 +228,7 @@ def test_sgd_end_to_end_quantization(ctx, model_bits, grad_bits):
     # threshold (a sub-ulp difference in the norm may flip those)
     _, g_ref = oracle.sgd_epoch(ods, b, x0, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
                                 first_step=1, num_steps=1, want_grad=True)
-    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN):
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER):
         x = to_dev(x0, ctx)
         g = torch.zeros((2, 512), dtype=torch.float32, device=ctx.device)
         ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
