@@ -38,10 +38,11 @@
 
 namespace zipml {
 
-constexpr int kCluThreads = 256;
+constexpr int kCluThreads = 512;
 constexpr int kCluWarps = kCluThreads / 32;
 constexpr int kCluMaxSlots = 8;
-constexpr int kCluMaxCtas = 16;
+constexpr int kCluMaxCtas = 16;                   // one bulk copy per warp and destination: at most kCluWarps CTAs
+static_assert(kCluMaxCtas <= kCluWarps, "a warp per destination CTA");
 
 struct ClusterArgs {
     const uint32_t* p1;
@@ -62,7 +63,7 @@ struct ClusterArgs {
     int n, bits, row_words, words;   // words = ceil(n / codes per word) <= row_words
     int model_bits, grad_bits;
     int nb, rc, slots;
-    int sub_shift;               // a CTA owns 2^sub_shift consecutive features (at least 4)
+    int sub;                     // a CTA owns `sub` consecutive features (a multiple of 4)
     int p_shift;                 // 2^p_shift lanes share the sum of one owned feature
     int trace_steps;
 };
@@ -163,7 +164,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
     const int rw = a.row_words, nw = a.words, n = a.n;
     const int Fp = rw * FPW;
     const int L = 1 << a.bits;
-    const int sub = 1 << a.sub_shift;
+    const int sub = a.sub;
     const int nb = a.nb;
     const int Fs = nb * sub;
     float* tab = reinterpret_cast<float*>(s_raw + ((sizeof(ClusterShared) + 15) & ~(size_t)15));
@@ -371,11 +372,12 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
             // reduce-scatter: slice o of the part goes to owner o
             fence_async_smem();
             __syncthreads();
-            if (tid < nb)
-                bulk_copy_s2c(cluster_addr(gbuf + (size_t)bi * sub, tid), gpart + (size_t)tid * sub, slice_bytes,
-                              cluster_addr(&sh->rs_bar, tid));
+            // (one copy per warp: the copies of one warp's lanes would be issued one after the other)
+            if (lane == 0 && warp < nb)
+                bulk_copy_s2c(cluster_addr(gbuf + (size_t)bi * sub, warp), gpart + (size_t)warp * sub, slice_bytes,
+                              cluster_addr(&sh->rs_bar, warp));
             // the tile is consumed: refill its slot while the parts travel
-            if (tid == 32 && it + a.slots < step_end) issue_tile(it + a.slots, slot);
+            if (tid == 1 && it + a.slots < step_end) issue_tile(it + a.slots, slot);
             if (++slot == a.slots) { slot = 0; parity ^= 1u; }
             clu_mark(a, it, 3);
 
@@ -451,8 +453,8 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
         if (tid < rcnt) breg = __ldg(a.b + r0 + k0 + tid);
         fence_async_smem();
         __syncthreads();
-        if (tid < nb)
-            bulk_copy_s2c(cluster_addr(xs + (size_t)bi * sub, tid), xpub, slice_bytes, cluster_addr(&sh->ag_bar, tid));
+        if (lane == 0 && warp < nb)
+            bulk_copy_s2c(cluster_addr(xs + (size_t)bi * sub, warp), xpub, slice_bytes, cluster_addr(&sh->ag_bar, warp));
         clu_mark(a, it, 5);
 
         // -------------------------------------------------------------- the model arrives; build w
@@ -492,7 +494,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
 // Host side
 // ---------------------------------------------------------------------------------------------
 struct ClusterPlan {
-    int nb, rc, slots, sub_shift, p_shift;
+    int nb, rc, slots, sub, p_shift;
     size_t smem;
 };
 
@@ -532,17 +534,16 @@ static int make_cluster_plan(const zipml_ctx* ctx, const zipml_dataset* d, const
         r.rc = (int)((B + nb - 1) / nb);
         r.nb = (int)((B + r.rc - 1) / r.rc);                        // no CTA without rows in a full batch
         const int64_t per = (d->n + r.nb - 1) / r.nb;
-        r.sub_shift = 2;                                            // slices are copied in 16-byte units
-        while (((int64_t)1 << r.sub_shift) < per) ++r.sub_shift;
+        r.sub = (int)((per + 3) & ~(int64_t)3);                     // slices are copied in 16-byte units
         r.p_shift = 0;
-        while (r.p_shift < 5 && ((int64_t)2 << (r.sub_shift + r.p_shift)) <= kCluThreads && (1 << r.p_shift) < r.nb) ++r.p_shift;
+        while (r.p_shift < 5 && ((int64_t)r.sub << (r.p_shift + 1)) <= kCluThreads && (1 << r.p_shift) < r.nb) ++r.p_shift;
         if ((uint64_t)2 * r.rc * row_words * 4 >= (1u << 20)) continue;                     // mbarrier tx-count range
-        if (((uint64_t)r.nb << r.sub_shift) * 4 >= (1u << 20)) continue;
+        if ((uint64_t)r.nb * r.sub * 4 >= (1u << 20)) continue;
         int slots = kCluMaxSlots;
-        while (slots >= 2 && cluster_smem_bytes(cb, table, (int)row_words, d->bits, r.nb, 1 << r.sub_shift, r.rc, slots) > cap) --slots;
+        while (slots >= 2 && cluster_smem_bytes(cb, table, (int)row_words, d->bits, r.nb, r.sub, r.rc, slots) > cap) --slots;
         if (slots < 2) continue;
         r.slots = slots;
-        r.smem = cluster_smem_bytes(cb, table, (int)row_words, d->bits, r.nb, 1 << r.sub_shift, r.rc, slots);
+        r.smem = cluster_smem_bytes(cb, table, (int)row_words, d->bits, r.nb, r.sub, r.rc, slots);
         *plan = r;
         return ZIPML_OK;
     }
@@ -604,7 +605,7 @@ int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, f
     a.words = (int)((d->n + fpw - 1) / fpw);
     a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
     a.nb = plan.nb; a.rc = plan.rc; a.slots = plan.slots;
-    a.sub_shift = plan.sub_shift; a.p_shift = plan.p_shift;
+    a.sub = plan.sub; a.p_shift = plan.p_shift;
     if (p->batch_order) {
         int32_t* dev_order = reinterpret_cast<int32_t*>(ctx->ws + o_ord);
         e = cudaMemcpyAsync(dev_order, p->batch_order, sizeof(int32_t) * (size_t)T, cudaMemcpyHostToDevice, ctx->stream);
