@@ -212,6 +212,17 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->engine == ZIPML_ENGINE_LEAN) return launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_AUTO) {
+        // Small minibatch tiles are bound by the step-to-step chain, not by HBM: one cluster whose CTAs
+        // exchange through shared memory, else row parts exchanging through L2.  Larger tiles stream
+        // through the ring engine.  Each engine answers ZIPML_ERR_WORKSPACE when the shape does not fit it.
+        const int64_t B = params->batch < data->m ? params->batch : data->m;
+        const int64_t step_bytes = 2 * B * data->row_bytes;
+        if (step_bytes <= (2ll << 20)) {
+            rc = launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
+            if (rc != ZIPML_ERR_WORKSPACE) return rc;
+            rc = launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
+            if (rc != ZIPML_ERR_WORKSPACE) return rc;
+        }
         rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
         if (rc != ZIPML_ERR_WORKSPACE) return rc;
     }
