@@ -29,6 +29,11 @@ if ROOT not in sys.path:
 
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one epoch launch from the ncu capture summarised under profiles/
+# (workload, engine) -> bytes; an entry is removed when its kernel changes after the capture
+NCU_TRAFFIC_BYTES = {("c2", 5): 202.08e6 + 4.46e6}
+ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
+                  5: "sgd_cluster_kernel"}
 
 
 def measured_peaks():
@@ -249,8 +254,10 @@ def main():
     step_us = 1e3 * epoch_avg_ms / steps_per_epoch
     step_bytes = packed_bytes / steps_per_epoch
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": f"of {peak_kind} copy rate", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": "sgd_ring_kernel (one cooperative launch per epoch)", "algorithmic_bytes_per_launch": packed_bytes,
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, ctx.zipml_last_engine())) if args.m is None else None,
+                "peak_kind": f"of {peak_kind} copy rate", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "kernel": ENGINE_KERNELS.get(ctx.zipml_last_engine(), "?") + " (one launch per epoch)",
+                "algorithmic_bytes_per_launch": packed_bytes,
                 "launch_ms_avg": epoch_avg_ms, "launch_ms_min": epoch_ms[0],
                 "epoch_samples_per_s": w.m / (epoch_avg_ms * 1e-3),
                 # the minibatch chain is sequential: a step moves step_bytes and cannot start before the previous
@@ -328,7 +335,7 @@ def main():
             ctx.zipml_sync()
             t_ep = min(a_.elapsed_time(b_) for a_, b_ in evs)
             To = (wo.m + wo.batch - 1) // wo.batch
-            others[key] = {"workload": wo.name, "epoch_ms": t_ep, "us_per_step": 1e3 * t_ep / To,
+            others[key] = {"workload": wo.name, "kernel": ENGINE_KERNELS.get(ctx.zipml_last_engine(), "?"), "epoch_ms": t_ep, "us_per_step": 1e3 * t_ep / To,
                            "samples_per_s": wo.m / (t_ep * 1e-3), "packed_GB/s": dso.packed_bytes / (t_ep * 1e-3) / 1e9,
                            "frac_of_copy_rate": dso.packed_bytes / (t_ep * 1e-3) / 1e9 / peak,
                            "quantize_GB/s": (8 * wo.m * wo.n + 2 * dso.m * dso.row_bytes) / (q0.elapsed_time(q1) * 1e-3) / 1e9,

@@ -112,6 +112,9 @@ int zipml_sync(zipml_ctx* ctx);
 const char* zipml_strerror(int status);
 /* Diagnostics: how many of the library's kernels this context has launched since zipml_create. */
 int64_t zipml_kernel_launches(const zipml_ctx* ctx);
+/* Diagnostics: the ZIPML_ENGINE_* value that the context's latest zipml_sgd_epoch call ran (what
+ * AUTO resolved to), or ZIPML_ENGINE_AUTO before the first call. */
+int32_t zipml_last_engine(const zipml_ctx* ctx);
 /* Diagnostics for the latency model of zipml_sgd_epoch: runs `iterations` steps of the per-step
  * communication skeleton on `ctas` co-resident CTAs (each publishes floats_per_cta floats through
  * L2, a bounded-spin grid barrier, each reads 16 bytes of every other CTA) and writes the elapsed

@@ -16,7 +16,7 @@ LOSS_DENSE, LOSS_CODES = 0, 1
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER = 0, 1, 2, 3, 4, 5
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_barrier_latency", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -62,6 +62,8 @@ def lib():
         L.zipml_sync.argtypes = [vp]
         L.zipml_kernel_launches.argtypes = [vp]
         L.zipml_kernel_launches.restype = i64
+        L.zipml_last_engine.argtypes = [vp]
+        L.zipml_last_engine.restype = C.c_int32
         L.zipml_barrier_latency.argtypes = [vp, i32, i32, i32, vp]
         L.zipml_strerror.argtypes = [C.c_int]
         L.zipml_strerror.restype = C.c_char_p
@@ -159,6 +161,9 @@ class Context:
 
     def zipml_kernel_launches(self):
         return int(lib().zipml_kernel_launches(self._h))
+
+    def zipml_last_engine(self):
+        return int(lib().zipml_last_engine(self._h))
 
     def zipml_barrier_latency(self, ctas, floats_per_cta=0, iterations=1000):
         """Nanoseconds per step of the SGD step's communication skeleton on `ctas` CTAs."""

@@ -121,6 +121,8 @@ int zipml_destroy(zipml_ctx* ctx) {
 
 int64_t zipml_kernel_launches(const zipml_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int32_t zipml_last_engine(const zipml_ctx* ctx) { return ctx ? ctx->last_engine : 0; }
+
 int zipml_sync(zipml_ctx* ctx) {
     if (!ctx) return ZIPML_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);

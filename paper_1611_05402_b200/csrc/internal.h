@@ -25,6 +25,7 @@ struct zipml_ctx {
     unsigned char* stage = nullptr;
     size_t stage_bytes = 0;
     int64_t launches = 0;           // kernels launched so far (diagnostics)
+    int last_engine = 0;            // engine of the latest zipml_sgd_epoch call (diagnostics)
     void* tmap_encode = nullptr;    // cuTensorMapEncodeTiled, resolved on first use
 };
 

@@ -661,6 +661,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
             if (e != cudaSuccess) return cuda_status(e);
             ctx->launches += 1;
         }
+        ctx->last_engine = ZIPML_ENGINE_PERSISTENT;
         return ZIPML_OK;
     }
 
@@ -676,6 +677,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
             ctx->launches += 1;
         }
     }
+    ctx->last_engine = ZIPML_ENGINE_STEPWISE;
     return ZIPML_OK;
 }
 

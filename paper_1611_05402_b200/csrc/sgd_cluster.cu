@@ -616,6 +616,7 @@ int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, f
     e = cudaLaunchKernelExC(&cfg, kernel, params);
     if (e != cudaSuccess) return cuda_status(e);
     ctx->launches += 1;
+    ctx->last_engine = ZIPML_ENGINE_CLUSTER;
     return ZIPML_OK;
 }
 

@@ -583,6 +583,7 @@ int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         if (e != cudaSuccess) return cuda_status(e);
         ctx->launches += 1;
     }
+    ctx->last_engine = ZIPML_ENGINE_LEAN;
     return ZIPML_OK;
 }
 
