@@ -174,7 +174,7 @@ def main():
     # ------------------------------------------------------------------ our arm
     import torch
     import torch.distributed as dist
-    from paper_1611_05402_b200 import binding
+    from paper_1611_05402_b200 import binding, replicas
     from paper_1611_05402_b200.build import build as build_cuda
     if rank == 0:
         build_cuda()
@@ -237,11 +237,7 @@ def main():
     clocks = sampler.stop()
     ctx.zipml_sync()
     launches = ctx.zipml_kernel_launches() - launches0
-    ms = torch.tensor([t0.elapsed_time(t1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_total = float(ms.item())
-    value = world * w.m * w.epochs * args.steps / (ms_total * 1e-3)
+    value, ms_total = replicas.whole_job_value(w.m * w.epochs * args.steps, t0.elapsed_time(t1), dev)
     final_loss = float(loss_dev.item())
 
     # dominant kernel: the SGD epoch launch
@@ -290,15 +286,15 @@ def main():
                                         hist_bins=w.hist_bins, quantize_seed=w.seed, **kw)
         host_pass()
         fence()
-        h0 = time.perf_counter()
         k_e2e = max(1, min(args.steps, 3))
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record()
         for _ in range(k_e2e):
-            e2e_loss = host_pass()
+            e2e_loss = host_pass()                # returns the loss read back from the device: the call is synchronous
+        h1.record()
         torch.cuda.synchronize()
-        dt = torch.tensor([time.perf_counter() - h0], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(dt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * w.m * w.epochs * k_e2e / float(dt.item()), "unit": unit,
+        e2e_value, _ = replicas.whole_job_value(w.m * w.epochs * k_e2e, h0.elapsed_time(h1), dev)
+        e2e = {"value": e2e_value, "unit": unit,
                "h2d_bytes_per_step": int(Ah.numel() * 4 + bh.numel() * 4 + xh.numel() * 4),
                "d2h_bytes_per_step": int(xh.numel() * 4 + 8), "steps": k_e2e, "loss": e2e_loss}
         del Ah
