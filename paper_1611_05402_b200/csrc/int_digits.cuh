@@ -9,7 +9,7 @@ namespace zipml {
 // Both phases contract small unsigned codes with an fp32 vector that is constant for many rows (w in
 // phase A, the residuals in phase B).  That vector is turned, once per step, into fixed point:
 // value ~ delta * W with |W| <= QMAX, and W into NS balanced base-128 digits in [-64, 63], each an
-// int8.  Four codes times four digits are then one dp4a into an int32, the digit sums are combined
+// int8.  Codes times digits are integer products (dp4a, or the int8 tensor-core MMA below), the digit sums are combined
 // exactly in 64 bits, and the only rounding is the one quantization of the vector, 2^-27 of its
 // largest entry with four digits.  (Three digits, 2^-20, are not enough: the error of w is the same
 // for every row, survives the minibatch mean and is amplified where residuals are small against the
@@ -63,6 +63,45 @@ __device__ __forceinline__ long long combine_digits(const int (&acc)[NS]) {
 #pragma unroll
     for (int s = 0; s < NS; ++s) t += (long long)acc[s] << (7 * s);
     return t;
+}
+
+// ---- int8 tensor-core contraction ------------------------------------------------------------------
+// D += A (16 x 32, unsigned bytes, row-major) * B (32 x 8, signed bytes, column-major), 32-bit sums.
+// Lane = 4 * g + t.  A: a0 = (row g, k 4t..4t+3), a1 = (row g+8, same k), a2, a3 = the same rows at k+16;
+// B: b0 = (k 4t..4t+3, column g), b1 = k+16;  D: d0, d1 = (row g, columns 2t, 2t+1), d2, d3 = row g+8.
+// With the digit words of four entries as B's columns 0..3 (columns 4..7 zero) one instruction
+// contracts 16 x 32 codes with all four digits.
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Fragment loads from shared memory (ldmatrix, 8 x 8 matrices of 16-bit elements = 8 rows of 16 bytes).
+// Lanes 8j..8j+7 give the row addresses of matrix j (16-byte aligned, shared-memory byte addresses);
+// lane 4g + t receives from matrix j the four bytes 4t..4t+3 of its row g -- for byte data exactly an
+// A fragment register (rows x k) or, with rows = columns of B, a B fragment register.
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t& r0, uint32_t& r1, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr) : "memory");
+}
+// Transposed: lane 4g + t receives from matrix j the 16-bit elements (row 2t, column g) and (row 2t+1,
+// column g), i.e. bytes {2g, 2g+1} of row 2t in the low half and of row 2t+1 in the high half.
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+
+// Bytes (f0..f3) of four rows -> for each of the four features the bytes of the four rows.
+__device__ __forceinline__ void transpose4x4(uint32_t x0, uint32_t x1, uint32_t x2, uint32_t x3, uint32_t (&t)[4]) {
+    const uint32_t lo01 = __byte_perm(x0, x1, 0x5140), hi01 = __byte_perm(x0, x1, 0x7362);
+    const uint32_t lo23 = __byte_perm(x2, x3, 0x5140), hi23 = __byte_perm(x2, x3, 0x7362);
+    t[0] = __byte_perm(lo01, lo23, 0x5410);
+    t[1] = __byte_perm(lo01, lo23, 0x7632);
+    t[2] = __byte_perm(hi01, hi23, 0x5410);
+    t[3] = __byte_perm(hi01, hi23, 0x7632);
 }
 
 }  // namespace zipml

@@ -39,6 +39,7 @@ struct SgdArgs {
     int stages;             // shared-memory stages of the code ring (STAGED kernels)
     int cr;                 // ring engine: rows per chunk (one ring slot holds cr rows of both planes)
     int sub;                // ring engine: features of a part that one row-part CTA reduces and updates
+    int pitch;              // ring engine: words between consecutive rows of a chunk in shared memory (>= wc)
     // ring engine: exchange buffers of 8-byte packets {fp32 value, step tag}, zeroed before a launch
     unsigned long long* ll_pd;   // [2][nb][na][rc][4]   partial dots (hi, lo of two doubles); only na > 1
     unsigned long long* ll_rs;   // [na][nb][nb][sub+2]  partial gradients per (owner, writer) + residual sum

@@ -7,10 +7,22 @@
 //     step the chunks of phase A in order, then (if the tile has more than one chunk) the chunks
 //     of phase B in reverse order, so that the most recently streamed rows are fetched again
 //     first, while they are still in L2 -- and fills a ring of shared-memory slots with bulk
-//     asynchronous copies (cp.async.bulk + mbarrier transaction counts).  None of this depends on
-//     the model, so the producer runs ahead across phases and steps as far as the ring allows and
-//     HBM latency never sits on the step-to-step dependency chain;
+//     asynchronous copies (mbarrier transaction counts): for uniform grids one 2-D tensor-map box of
+//     32 rows of one plane per slot, its rows four words wider than the part so that they lie wc + 4
+//     words apart in shared memory (fragment loads of 8 rows then hit 8 different bank groups); for
+//     level tables both planes of a chunk per slot.  None of this depends on the model, so the
+//     producer runs ahead across phases and steps as far as the ring allows and HBM latency never
+//     sits on the step-to-step dependency chain;
 //   * consumers wait for a slot, compute on it and hand it back (one arrival per consumer warp).
+// Uniform grids contract on the int8 tensor cores (mma.sync m16n8k32, u8 x s8 -> s32): the fp32
+// vector that meets the codes (w = step * x~ in phase A, the residuals in phase B) is turned once
+// per step into four balanced base-128 digits per entry, stored as the B operand's columns; the
+// code bytes are the A operand, loaded with ldmatrix straight from the tile in phase A (16 rows x
+// 32 bytes) and with a transposing ldmatrix plus two byte permutes in phase B (16 byte columns x
+// 32 rows); 4- and 2-bit codes are split into their groups by a shift and a mask per fragment
+// register, each group meeting its own digit vectors.  Digit sums are exact 32-bit integers, combined
+// in 64 bits (or exactly in double); warps meet through shared-memory integer atomics, whose order
+// cannot change the result.  Level tables use fp32 look-ups.
 // Per step:  phase A dots -> residuals (with na > 1 the partial dots of a row meet first);
 //            phase B partial gradients of the CTA's rows;
 //            reduce-scatter: CTA (ai, bi) collects the nb row parts of its own sub-slice of feature
@@ -40,6 +52,7 @@ constexpr int kRingConsumers = 256;
 constexpr int kRingWarps = kRingConsumers / 32;
 constexpr int kRingThreads = kRingConsumers + 32;
 constexpr int kRingMaxSlots = 8;
+constexpr int kRingTasks = 8;              // integer phase B: accumulator sets (8 words of one group) per warp
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kRingConsumers) : "memory"); }
 
@@ -66,6 +79,7 @@ struct RingShared {
     unsigned long long empty[kRingMaxSlots];
     int abort_flag;
     int pad;
+    uint4 zero16;                  // sixteen zero bytes: the unused columns of the digit operands point here
 };
 
 // Bounded wait on an mbarrier phase; after the first failure of this CTA every wait is skipped.
@@ -152,12 +166,6 @@ __device__ __forceinline__ void ll_gather(const unsigned long long* src, int cou
     }
 }
 
-__device__ __forceinline__ int dp4a_us(uint32_t codes, uint32_t digits, int acc) {
-    int d;
-    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(codes), "r"(digits), "r"(acc));
-    return d;
-}
-
 // Eight values per lane -> their eight sums over the warp with 9 shuffles instead of 40: in each of
 // the first three steps a lane hands half of what it holds to its partner and keeps (and adds) the
 // other half.  Afterwards lane L holds sum number (L >> 2) & 7, complete, in a fixed order.
@@ -205,7 +213,9 @@ __device__ __forceinline__ float consumer_max(float v, RingShared* sh, int slot)
 //   nbuf[2*G] float             collected partial norms
 //   gred[kRingConsumers*FPW]    cross-group reduction of phase B
 //   res[2*rc] float             residuals
-//   rqs[2*ceil(rc/4)] uint4     uniform: digit words of the residuals, four rows each (r1 then r2)
+//   rdig[ceil(rc/32)][2][4][32] bytes  uniform: digits of the residuals as B operands: per 32 rows, per
+//                               residual (r1, r2), per digit a 32-byte k vector (row order of phase B)
+//   dacc[rc][2][4] int          uniform: digit sums of the dots per (row, plane), filled by the warps' atomics
 //   bsm[2][rc] float            labels of the current and the next step's rows
 //   ring[slots][2][cr][wc] u32  code chunks
 template <int CB, bool TABLE>
@@ -228,11 +238,14 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     float* nbuf = gbuf + ((a.nb * subp + 3) & ~3);
     float* gred = nbuf + ((2 * G + 3) & ~3);
     float* res = gred + kRingConsumers * FPW;
-    uint4* rqs = reinterpret_cast<uint4*>(res + ((2 * a.rc + 3) & ~3));
-    float* bsm = reinterpret_cast<float*>(rqs + 2 * ((a.rc + 3) / 4));
+    unsigned char* rdig = reinterpret_cast<unsigned char*>(res + ((2 * a.rc + 3) & ~3));
+    int* dacc = reinterpret_cast<int*>(rdig + (size_t)((a.rc + 31) / 32) * 256);
+    float* bsm = reinterpret_cast<float*>(dacc + (TABLE ? 0 : 8 * a.rc));
     uint32_t* ring = reinterpret_cast<uint32_t*>(
         (reinterpret_cast<uintptr_t>(bsm + ((2 * a.rc + 3) & ~3)) + 127) & ~(uintptr_t)127);      // tensor copies want 128 bytes
-    const size_t slot_words = (size_t)2 * a.cr * a.wc;
+    const int pitch = a.pitch;
+    constexpr int PPS = TABLE ? 2 : 1;           // planes per ring slot
+    const size_t slot_words = (size_t)PPS * a.cr * pitch;
 
     const int ai = blockIdx.x % a.na, bi = blockIdx.x / a.na;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -260,6 +273,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             mbar_init(reinterpret_cast<uint64_t*>(sh->empty + s), kRingWarps);
         }
         sh->abort_flag = 0;
+        sh->zero16 = make_uint4(0u, 0u, 0u, 0u);
         mbar_fence_init();
     }
     __syncthreads();
@@ -269,7 +283,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
         int slot = 0;
         uint32_t phase = 0;
         const uint32_t row_bytes = (uint32_t)wcopy * 4u;
-        const bool contiguous = (a.row_words == a.wc) && (wcopy == a.wc);
+        const bool contiguous = (a.row_words == a.wc) && (wcopy == a.wc) && (pitch == a.wc);
         for (int64_t it = a.first_step; it < step_end; ++it) {
             if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) break;   // a wait gave up: start no more copies
             int64_t r0; int bt, rcnt;
@@ -282,6 +296,36 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 uint64_t* full = reinterpret_cast<uint64_t*>(sh->full + slot);
                 uint32_t* dst = ring + (size_t)slot * slot_words;
                 const int64_t first = r0 + k0 + (int64_t)chunk * a.cr;
+                if constexpr (!TABLE) {
+                    // one slot per plane: rows of `row_bytes` bytes, `pitch` words apart
+#pragma unroll 1
+                    for (int pl = 0; pl < 2; ++pl) {
+                        uint64_t* fullp = reinterpret_cast<uint64_t*>(sh->full + slot);
+                        uint32_t* dstp = ring + (size_t)slot * slot_words;
+                        if (a.use_tmap) {
+                            // one box of cr rows x pitch words (64-bit elements): the four words past the part
+                            // (the neighbour's, or zeros past the row) and the rows past the chunk come along
+                            // unused; the box's dense rows are exactly `pitch` words apart
+                            if (lane == 0) {
+                                ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
+                                mbar_arrive_expect_tx(fullp, (uint32_t)a.cr * (uint32_t)pitch * 4u);
+                                tensor_copy_g2s(dstp, pl == 0 ? &tm1 : &tm2, (int)(w0 >> 1), (int)first, fullp);
+                            }
+                            __syncwarp();
+                        } else {
+                            if (lane == 0) {
+                                ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
+                                mbar_arrive_expect_tx(fullp, (uint32_t)rows * row_bytes);
+                            }
+                            __syncwarp();
+                            const uint32_t* src = (pl == 0 ? a.p1 : a.p2) + first * a.row_words + w0;
+                            for (int r = lane; r < rows; r += 32)
+                                bulk_copy_g2s(dstp + (size_t)r * pitch, src + (size_t)r * a.row_words, row_bytes, fullp);
+                        }
+                        if (++slot == slots) { slot = 0; phase ^= 1u; }
+                    }
+                    continue;
+                }
                 if (a.use_tmap) {
                     // one box of cr rows x wc words per plane; rows past the chunk (the next rows of the
                     // plane, or zeros past its end) come along and are never used
@@ -289,7 +333,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                         ring_wait(sh->empty + slot, phase ^ 1u, &sh->abort_flag, a.status, 5);
                         mbar_arrive_expect_tx(full, 2u * (uint32_t)a.cr * (uint32_t)a.wc * 4u);
                         tensor_copy_g2s(dst, &tm1, (int)w0, (int)first, full);
-                        tensor_copy_g2s(dst + (size_t)a.cr * a.wc, &tm2, (int)w0, (int)first, full);
+                        tensor_copy_g2s(dst + (size_t)a.cr * pitch, &tm2, (int)w0, (int)first, full);
                     }
                     __syncwarp();
                 } else {
@@ -300,12 +344,12 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                     __syncwarp();
                     if (contiguous) {
                         if (lane < 2)
-                            bulk_copy_g2s(dst + (size_t)lane * a.cr * a.wc, (lane == 0 ? a.p1 : a.p2) + first * a.row_words,
+                            bulk_copy_g2s(dst + (size_t)lane * a.cr * pitch, (lane == 0 ? a.p1 : a.p2) + first * a.row_words,
                                           (uint32_t)rows * row_bytes, full);
                     } else {
                         for (int i = lane; i < 2 * rows; i += 32) {
                             const int plane = i & 1, r = i >> 1;
-                            bulk_copy_g2s(dst + ((size_t)plane * a.cr + r) * a.wc,
+                            bulk_copy_g2s(dst + ((size_t)plane * a.cr + r) * pitch,
                                           (plane == 0 ? a.p1 : a.p2) + (first + r) * a.row_words + w0, row_bytes, full);
                         }
                     }
@@ -330,7 +374,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     // Turns the model values of this thread's word (as the gradient will see them) into what phase A
     // reads; every consumer calls it, `have` says whether the thread holds a word (parts are at most
     // one word per consumer wide).  Returns delta_w, the value of one fixed-point unit of w.
-    uint4* tabq = reinterpret_cast<uint4*>(tab);
+    uint32_t* wd32 = reinterpret_cast<uint32_t*>(tab);      // uniform: digits of w, [k-slab][group][digit][8 words]
     double base_w = 0.0;                         // lo^T x~ over the CTA's feature part (uniform grids)
     auto word_stage = [&](bool have, int q, const float (&xt)[FPW]) -> double {
         if constexpr (!TABLE) {
@@ -357,8 +401,11 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             if (have) {
 #pragma unroll
                 for (int g = 0; g < NG; ++g) {
+                    // B operand of phase A: per k-slab (8 words), group and digit a 32-byte k vector
                     const float v4[4] = {wv[0 * NG + g], wv[1 * NG + g], wv[2 * NG + g], wv[3 * NG + g]};
-                    tabq[g * a.wc + q] = digit_words<NS>(v4, inv);
+                    const uint4 o = digit_words<NS>(v4, inv);
+                    uint32_t* dst = wd32 + (size_t)(((q >> 3) * NG + g) * NS) * 8 + (q & 7);
+                    dst[0] = o.x; dst[8] = o.y; dst[16] = o.z; dst[24] = o.w;
                 }
             }
             return (double)wmax / (double)QMAXF;
@@ -403,6 +450,8 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             delta_w = word_stage(have, q, xt);
         }
         for (int k = threadIdx.x; k < nsub; k += kRingConsumers) xown[k] = (sub0 + k < fcnt) ? a.x[j0 + sub0 + k] : 0.0f;
+        if constexpr (!TABLE)
+            for (int i = threadIdx.x; i < 8 * a.rc; i += kRingConsumers) dacc[i] = 0;
         int64_t r0; int bt, rcnt;
         step_rows(a.first_step, r0, bt, rcnt);
         float* bcur = bsm + (size_t)(a.first_step & 1) * a.rc;
@@ -416,6 +465,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     const int group = threadIdx.x / lanes_q;
     const int ql = threadIdx.x % lanes_q;
     const int chunks_w = (wcnt + 31) / 32;
+    const int kw8 = (wcnt + 7) / 8;              // k-slabs (8 words) per code group in the integer path
     unsigned long long* rs_mine = a.ll_rs + (size_t)ai * a.nb * a.nb * subp;                 // + (owner*nb + writer)*subp
     const unsigned long long* rs_own = rs_mine + (size_t)bi * a.nb * subp;                   // collected by this owner
     unsigned long long* ag_part = a.ll_ag + j0;
@@ -452,7 +502,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
         // -------------------------------------------------------------- phase A: dots
         const bool dots_local = (a.na == 1);
         unsigned long long* pd_mine = a.ll_pd + (((size_t)par * a.nb + bi) * a.na + ai) * a.rc * 4;
-        const int slot_a = slot;                 // slot of the single chunk when C == 1
+        int slot_a = slot, slot_a2 = slot;       // slot(s) of the single chunk when C == 1 (uniform: one per plane)
         // A warp takes four rows at a time: one load of w's digit words serves them all and the
         // eight (row, plane) sums are independent chains.  When the tile has fewer row blocks than warps
         // (single-chunk tiles only) a block's words are split over S warps.
@@ -460,7 +510,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
         int S = 1;
         {
             const int nblk_all = (rcnt + RB - 1) / RB;
-            if (C == 1 && nblk_all > 0 && nblk_all < kRingWarps) S = max(1, min(chunks_w, kRingWarps / nblk_all));
+            if (TABLE && C == 1 && nblk_all > 0 && nblk_all < kRingWarps) S = max(1, min(chunks_w, kRingWarps / nblk_all));
         }
         const int cps = (chunks_w + S - 1) / S;
         double wsum = 0.0;                       // r1 + r2 (one of them per lane) over what this thread finished
@@ -470,44 +520,78 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             const int rows = min(a.cr, rcnt - chunk * a.cr);
             ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 6);
             const uint32_t* t1 = ring + (size_t)slot * slot_words;
-            const uint32_t* t2 = t1 + (size_t)a.cr * a.wc;
-            const int nblk = (rows + RB - 1) / RB;
-            for (int task = warp; task < nblk * S; task += kRingWarps) {
-                const int blk = task / S, seg = task - blk * S;
-                const uint32_t* rowp1 = t1 + (size_t)(blk * RB) * a.wc;
-                const uint32_t* rowp2 = t2 + (size_t)(blk * RB) * a.wc;
-                int ia[TABLE ? 1 : 2 * RB][NS];
-                float fa[2 * RB];
-#pragma unroll
-                for (int v = 0; v < 2 * RB; ++v) {
-                    fa[v] = 0.0f;
-                    if constexpr (!TABLE) {
-#pragma unroll
-                        for (int sidx = 0; sidx < NS; ++sidx) ia[v][sidx] = 0;
-                    }
-                }
-                const int c_end = min(chunks_w, (seg + 1) * cps);
+            const uint32_t* t2 = t1 + (size_t)a.cr * pitch;
+            if constexpr (!TABLE) {
+                // Integer dots on the tensor cores, one plane (one ring slot) after the other.  A k-slab is
+                // 8 words (32 bytes of codes) of a row; a warp takes every kRingWarps-th slab for the chunk's
+                // one or two blocks of 16 rows: the code bytes come as A fragments straight from the tile
+                // (ldmatrix), each code group of the bytes meets its own digit vectors of w (B fragments,
+                // ldmatrix), all in the same accumulators.  The warps' digit sums meet in dacc (integer sums:
+                // the order of the atomics does not matter).  Rows past the chunk's last one are read (clamped
+                // to the slot) and dropped; words past the part's last one meet zero digits.
+                const int gl = lane >> 2, tl = lane & 3, lm = lane >> 3, l8 = lane & 7;
+                const uint32_t wbase_addr = smem_u32(wd32), zero_addr = smem_u32(&sh->zero16);
+#pragma unroll 1
+                for (int pl = 0; pl < 2; ++pl) {
+                    if (pl == 1) ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 6);
+                    const uint32_t tile_addr = smem_u32(ring + (size_t)slot * slot_words);
+                    int c[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+                    const uint32_t arow0 = tile_addr + (uint32_t)min(l8 + (lm & 1) * 8, a.cr - 1) * (uint32_t)pitch * 4u + (lm >> 1) * 16u;
+                    const uint32_t arow1 = tile_addr + (uint32_t)min(16 + l8 + (lm & 1) * 8, a.cr - 1) * (uint32_t)pitch * 4u + (lm >> 1) * 16u;
+                    const bool two_blocks = rows > 16;
 #pragma unroll 2
-                for (int c = seg * cps; c < c_end; ++c) {
-                    const int q = c * 32 + lane;
-                    if (q < wcnt) {
-                        uint32_t u[2 * RB];      // rows past the chunk's last one read leftovers of the slot; never used
+                    for (int ks = warp; ks < kw8; ks += kRingWarps) {
+                        uint32_t bf[NG][2], ar0[4], ar1[4];
+                        ldsm_x4(ar0, arow0 + (uint32_t)ks * 32u);
+                        ldsm_x4(ar1, (two_blocks ? arow1 : arow0) + (uint32_t)ks * 32u);
 #pragma unroll
-                        for (int r = 0; r < RB; ++r) { u[2 * r] = rowp1[(size_t)r * a.wc + q]; u[2 * r + 1] = rowp2[(size_t)r * a.wc + q]; }
-                        if constexpr (!TABLE) {
+                        for (int g = 0; g < NG; ++g)
+                            ldsm_x2(bf[g][0], bf[g][1],
+                                    l8 < NS ? wbase_addr + (uint32_t)(((ks * NG + g) * NS + l8) * 32 + (lm & 1) * 16) : zero_addr);
 #pragma unroll
-                            for (int g = 0; g < NG; ++g) {
-                                const uint4 dq = tabq[g * a.wc + q];
+                        for (int g = 0; g < NG; ++g) {
+                            mma_u8s8(c[0], group_bytes<CB>(ar0[0], g), group_bytes<CB>(ar0[1], g), group_bytes<CB>(ar0[2], g),
+                                     group_bytes<CB>(ar0[3], g), bf[g][0], bf[g][1]);
+                            mma_u8s8(c[1], group_bytes<CB>(ar1[0], g), group_bytes<CB>(ar1[1], g), group_bytes<CB>(ar1[2], g),
+                                     group_bytes<CB>(ar1[3], g), bf[g][0], bf[g][1]);
+                        }
+                    }
+                    if (tl < 2) {                        // columns 2t, 2t+1 are digits; dacc is [row][plane][digit]
 #pragma unroll
-                                for (int v = 0; v < 2 * RB; ++v) {
-                                    const uint32_t bq = group_bytes<CB>(u[v], g);
-                                    ia[v][0] = dp4a_us(bq, dq.x, ia[v][0]);
-                                    ia[v][1] = dp4a_us(bq, dq.y, ia[v][1]);
-                                    ia[v][2] = dp4a_us(bq, dq.z, ia[v][2]);
-                                    if constexpr (NS == 4) ia[v][NS - 1] = dp4a_us(bq, dq.w, ia[v][NS - 1]);
-                                }
-                            }
-                        } else {
+                        for (int rb = 0; rb < 2; ++rb) {
+                            const int la = rb * 16 + gl, lh = la + 8;
+                            int* d = dacc + (size_t)(chunk * a.cr + la) * 8 + pl * 4 + 2 * tl;
+                            if (la < rows) { atomicAdd(d, c[rb][0]); atomicAdd(d + 1, c[rb][1]); }
+                            if (lh < rows) { atomicAdd(d + 64, c[rb][2]); atomicAdd(d + 65, c[rb][3]); }
+                        }
+                    }
+                    if (C > 1) {                         // hand the slot back; phase B fetches the chunk again
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
+                    } else if (pl == 0) {
+                        slot_a = slot;                   // the single chunk stays: plane 1 here, plane 2 in the next slot
+                    } else {
+                        slot_a2 = slot;
+                    }
+                    if (++slot == slots) { slot = 0; phase ^= 1u; }
+                }
+            } else {
+                const int nblk = (rows + RB - 1) / RB;
+                for (int task = warp; task < nblk * S; task += kRingWarps) {
+                    const int blk = task / S, seg = task - blk * S;
+                    const uint32_t* rowp1 = t1 + (size_t)(blk * RB) * pitch;
+                    const uint32_t* rowp2 = t2 + (size_t)(blk * RB) * pitch;
+                    float fa[2 * RB];
+#pragma unroll
+                    for (int v = 0; v < 2 * RB; ++v) fa[v] = 0.0f;
+                    const int c_end = min(chunks_w, (seg + 1) * cps);
+#pragma unroll 2
+                    for (int c = seg * cps; c < c_end; ++c) {
+                        const int q = c * 32 + lane;
+                        if (q < wcnt) {
+                            uint32_t u[2 * RB];      // rows past the chunk's last one read leftovers of the slot; never used
+#pragma unroll
+                            for (int r = 0; r < RB; ++r) { u[2 * r] = rowp1[(size_t)r * pitch + q]; u[2 * r + 1] = rowp2[(size_t)r * pitch + q]; }
 #pragma unroll
                             for (int i = 0; i < FPW; ++i) {
 #pragma unroll
@@ -515,45 +599,52 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                             }
                         }
                     }
-                }
-                double dsum;
-                if constexpr (!TABLE) {
-                    // exact: digit sums -> 64-bit totals -> warp totals; one conversion per (row, plane)
-                    long long tv[2 * RB];
-#pragma unroll
-                    for (int v = 0; v < 2 * RB; ++v) tv[v] = combine_digits<NS>(ia[v]);
-                    const long long tsum = reduce8(tv, lane);
-                    dsum = (double)tsum * delta_w + (seg == 0 ? base_w : 0.0);
-                } else {
                     double pv[2 * RB];
 #pragma unroll
                     for (int v = 0; v < 2 * RB; ++v) pv[v] = (double)fa[v];
-                    dsum = reduce8(pv, lane);
-                }
-                if ((lane & 3) == 0) {
-                    const int lr = blk * RB + (vmine >> 1), plane = vmine & 1;
-                    const int r = chunk * a.cr + lr;
-                    if (S > 1) {
-                        sh->dpart[task * 8 + vmine] = dsum;
-                    } else if (lr < rows) {
-                        if (dots_local) {
-                            const float rv = (float)(dsum - (double)bcur[r]);
-                            res[2 * r + plane] = rv;
-                            wsum += (double)rv;
-                            rmax = fmaxf(rmax, fabsf(rv));
-                        } else {
-                            ll_store_double(pd_mine + (size_t)r * 4 + 2 * plane, dsum, tag);
+                    const double dsum = reduce8(pv, lane);
+                    if ((lane & 3) == 0) {
+                        const int lr = blk * RB + (vmine >> 1), plane = vmine & 1;
+                        const int r = chunk * a.cr + lr;
+                        if (S > 1) {
+                            sh->dpart[task * 8 + vmine] = dsum;
+                        } else if (lr < rows) {
+                            if (dots_local) {
+                                const float rv = (float)(dsum - (double)bcur[r]);
+                                res[2 * r + plane] = rv;
+                                wsum += (double)rv;
+                                rmax = fmaxf(rmax, fabsf(rv));
+                            } else {
+                                ll_store_double(pd_mine + (size_t)r * 4 + 2 * plane, dsum, tag);
+                            }
                         }
                     }
                 }
             }
-            if (C > 1) {                         // hand the slot back; phase B fetches the chunk again
+            if (TABLE && C > 1) {                // hand the slot back; phase B fetches the chunk again
                 __syncwarp();
                 if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
                 if (++slot == slots) { slot = 0; phase ^= 1u; }
             }
         }
-        if (S > 1) {                             // single chunk: one thread per (row, plane) adds the segments in order
+        if constexpr (!TABLE) {                  // one thread per (row, plane) takes the digit sums and clears them
+            consumer_sync();
+            for (int idx = threadIdx.x; idx < 2 * rcnt; idx += kRingConsumers) {
+                const int4 dv = *reinterpret_cast<const int4*>(dacc + (size_t)idx * 4);
+                *reinterpret_cast<int4*>(dacc + (size_t)idx * 4) = make_int4(0, 0, 0, 0);
+                const int dd[NS] = {dv.x, dv.y, dv.z, dv.w};
+                const double d = (double)combine_digits<NS>(dd) * delta_w + base_w;
+                const int r = idx >> 1, plane = idx & 1;
+                if (dots_local) {
+                    const float rv = (float)(d - (double)bcur[r]);
+                    res[idx] = rv;
+                    wsum += (double)rv;
+                    rmax = fmaxf(rmax, fabsf(rv));
+                } else {
+                    ll_store_double(pd_mine + (size_t)r * 4 + 2 * plane, d, tag);
+                }
+            }
+        } else if (S > 1) {                      // single chunk: one thread per (row, plane) adds the segments in order
             consumer_sync();
             if ((int)threadIdx.x < 2 * rcnt) {
                 const int r = threadIdx.x >> 1, plane = threadIdx.x & 1;
@@ -580,18 +671,31 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             for (int r = threadIdx.x; r < rcnt; r += kRingConsumers) {
                 double d1 = 0.0, d2 = 0.0;
                 bool good = !*reinterpret_cast<volatile int*>(&sh->abort_flag);
-                for (int p = 0; p < a.na && good; ++p) {
-                    const unsigned long long* src = pd_row + ((size_t)p * a.rc + r) * 4;
-                    unsigned long long v[4];
+                // four parts at a time, their sixteen packets in flight together
+                for (int p0 = 0; p0 < a.na && good; p0 += 4) {
+                    const unsigned long long* src = pd_row + ((size_t)p0 * a.rc + r) * 4;
+                    const int np = min(4, a.na - p0);
+                    unsigned long long v[4][4];
                     bool ok = false;
                     for (long long spin = 0; spin < kPacketSpinLimit && !ok; ++spin) {
                         ok = true;
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) { v[u] = ll_load(src + u); ok = ok && ((uint32_t)(v[u] >> 32) == tag); }
+                        for (int pp = 0; pp < 4; ++pp)
+                            if (pp < np) {
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    v[pp][u] = ll_load(src + (size_t)pp * a.rc * 4 + u);
+                                    ok = ok && ((uint32_t)(v[pp][u] >> 32) == tag);
+                                }
+                            }
                     }
                     if (!ok) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 1); good = false; break; }
-                    d1 += (double)__uint_as_float((uint32_t)v[0]) + (double)__uint_as_float((uint32_t)v[1]);
-                    d2 += (double)__uint_as_float((uint32_t)v[2]) + (double)__uint_as_float((uint32_t)v[3]);
+#pragma unroll
+                    for (int pp = 0; pp < 4; ++pp)
+                        if (pp < np) {
+                            d1 += (double)__uint_as_float((uint32_t)v[pp][0]) + (double)__uint_as_float((uint32_t)v[pp][1]);
+                            d2 += (double)__uint_as_float((uint32_t)v[pp][2]) + (double)__uint_as_float((uint32_t)v[pp][3]);
+                        }
                 }
                 const double bk = (double)bcur[r];
                 const float r1 = good ? (float)(d1 - bk) : 0.0f, r2 = good ? (float)(d2 - bk) : 0.0f;
@@ -614,87 +718,147 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
             for (int w = 0; w < kRingWarps; ++w) rho = fmaxf(rho, sh->fmax[16 + w]);
             const float inv = rho > 0.0f ? QMAXF / rho : 0.0f;
             delta_r = (double)rho / (double)QMAXF;
-            // digit words of the residuals, four rows at a time (rows past the batch count as zero)
-            for (int k4 = threadIdx.x; k4 < (rcnt + 3) / 4; k4 += kRingConsumers) {
+            // digits of the residuals as B operands of phase B: per 32 rows and residual, per digit, 32 bytes
+            // in the row order the transposed code fragments come in (k = 16h + 4t + e <-> row 16h + 2t +
+            // (e & 1) + 8 (e >> 1)); rows past the batch count as zero
+            uint32_t* rd32w = reinterpret_cast<uint32_t*>(rdig);
+            for (int kk = threadIdx.x; kk < 8 * ((rcnt + 31) / 32); kk += kRingConsumers) {
+                const int rbase = (kk >> 3) * 32 + ((kk >> 2) & 1) * 16 + 2 * (kk & 3);
                 float v1[4], v2[4];
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int k = 4 * k4 + r;
-                    v1[r] = k < rcnt ? res[2 * k] : 0.0f;
-                    v2[r] = k < rcnt ? res[2 * k + 1] : 0.0f;
+                for (int e = 0; e < 4; ++e) {
+                    const int k = rbase + (e & 1) + 8 * (e >> 1);
+                    v1[e] = k < rcnt ? res[2 * k] : 0.0f;
+                    v2[e] = k < rcnt ? res[2 * k + 1] : 0.0f;
                 }
-                rqs[2 * k4] = digit_words<NS>(v1, inv);
-                rqs[2 * k4 + 1] = digit_words<NS>(v2, inv);
+                const uint4 o1 = digit_words<NS>(v1, inv), o2 = digit_words<NS>(v2, inv);
+                uint32_t* d1 = rd32w + (size_t)((kk >> 3) * 2 * NS) * 8 + (kk & 7);
+                d1[0] = o1.x; d1[8] = o1.y; d1[16] = o1.z; d1[24] = o1.w;
+                d1[32] = o2.x; d1[40] = o2.y; d1[48] = o2.z; d1[56] = o2.w;
             }
             consumer_sync();
         }
         trace_mark(a, it, 1);
 
         // -------------------------------------------------------------- phase B: gradient
-        {
-            const int q = ql;
-            const bool active = (group < ngroups) && (q < wcnt);
-            float acc[FPW];
+        if constexpr (!TABLE) {
+            // Integer gradient parts on the tensor cores, one plane (one ring slot) after the other.  A task
+            // is a 16-byte column of the tile over its 32 rows; a warp keeps the accumulators of its columns
+            // (every kRingWarps-th) across the chunks.  A transposing ldmatrix hands each lane the bytes
+            // {2g, 2g+1} of rows {2t, 2t+1} of the four 8-row groups; two permutes per half turn them into A
+            // fragments "byte 2g (or 2g+1) of the column, four rows", i.e. features x rows with the row order
+            // the residual digits were stored in.  Each code group of the bytes meets the residual digits
+            // (plane 1 those of r2, plane 2 those of r1) in its own accumulators.
+            constexpr int TI = (CB == 2) ? kRingTasks / 2 : kRingTasks;       // columns per warp
+            const int gl = lane >> 2, tl = lane & 3, lm = lane >> 3, l8 = lane & 7;
+            const uint32_t rbase_addr = smem_u32(rdig), zero_addr = smem_u32(&sh->zero16);
+            const int ncol = (wcnt + 3) / 4;
+            const unsigned sub_magic = (unsigned)((0x100000000ull + (unsigned)a.sub - 1) / (unsigned)a.sub);   // ceil(2^32 / sub)
+            int acc[TI][NG][4];
 #pragma unroll
-            for (int i = 0; i < FPW; ++i) acc[i] = 0.0f;
-            int ib[TABLE ? 1 : FPW][NS];         // uniform: digit sums per feature of the word
+            for (int ti = 0; ti < TI; ++ti)
 #pragma unroll
-            for (int i = 0; i < (TABLE ? 1 : FPW); ++i)
+                for (int g = 0; g < NG; ++g)
 #pragma unroll
-                for (int sidx = 0; sidx < NS; ++sidx) ib[i][sidx] = 0;
+                    for (int e = 0; e < 4; ++e) acc[ti][g][e] = 0;
             for (int ci = 0; ci < C; ++ci) {
                 const int chunk = C - 1 - ci;
-                const int rows = min(a.cr, rcnt - chunk * a.cr);
-                int use_slot = slot_a;
-                if (C > 1) {
-                    ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 7);
-                    use_slot = slot;
-                }
-                if (active) {
-                    const uint32_t* col1 = ring + (size_t)use_slot * slot_words + q;
-                    const uint32_t* col2 = col1 + (size_t)a.cr * a.wc;
-                    if constexpr (!TABLE) {
-                        // four rows at a time: transpose their codes so that a register holds one feature of
-                        // the four rows, then one dp4a per residual digit (slots hold a multiple of four rows;
-                        // rows past the chunk meet zero digits)
-                        const uint4* rq = rqs + 2 * (chunk * a.cr / 4);
-#pragma unroll 2
-                        for (int l4 = group; l4 < (rows + 3) / 4; l4 += ngroups) {
-                            uint32_t u1[4], u2[4];
+                const int slab = chunk * a.cr / 32;              // chunks are 32 rows, or the tile is one chunk
+#pragma unroll 1
+                for (int pl = 0; pl < 2; ++pl) {
+                    int use_slot = pl ? slot_a2 : slot_a;
+                    if (C > 1) {
+                        ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 7);
+                        use_slot = slot;
+                    }
+                    // digits of r2 for plane 1, of r1 for plane 2; rows past the chunk carry zero digits
+                    uint32_t b0, b1;
+                    ldsm_x2(b0, b1, l8 < NS ? rbase_addr + (uint32_t)(((slab * 2 + (1 - pl)) * NS + l8) * 32 + (lm & 1) * 16) : zero_addr);
+                    const uint32_t row_addr = smem_u32(ring + (size_t)use_slot * slot_words) +
+                                              (uint32_t)min(lane, a.cr - 1) * (uint32_t)pitch * 4u;
+                    // four columns at a time: their loads are issued together, then the permutes and MMAs
 #pragma unroll
-                            for (int r = 0; r < 4; ++r) {
-                                u1[r] = col1[(size_t)(4 * l4 + r) * a.wc];
-                                u2[r] = col2[(size_t)(4 * l4 + r) * a.wc];
-                            }
-                            const uint4 d1 = rq[2 * l4], d2 = rq[2 * l4 + 1];     // digits of r1, of r2
+                    for (int t0 = 0; t0 < TI; t0 += 4) {
+                        uint32_t r4[4][4];
 #pragma unroll
-                            for (int g = 0; g < NG; ++g) {
+                        for (int tj = 0; tj < 4; ++tj) {
+                            const int col = min(warp + (t0 + tj) * kRingWarps, ncol - 1);      // clamped: results dropped below
+                            ldsm_x4_trans(r4[tj], row_addr + (uint32_t)col * 16u);
+                        }
 #pragma unroll
-                                for (int pl = 0; pl < 2; ++pl) {
-                                    const uint32_t x0 = group_bytes<CB>(pl ? u2[0] : u1[0], g), x1 = group_bytes<CB>(pl ? u2[1] : u1[1], g);
-                                    const uint32_t x2 = group_bytes<CB>(pl ? u2[2] : u1[2], g), x3 = group_bytes<CB>(pl ? u2[3] : u1[3], g);
-                                    const uint32_t lo01 = __byte_perm(x0, x1, 0x5140), hi01 = __byte_perm(x0, x1, 0x7362);
-                                    const uint32_t lo23 = __byte_perm(x2, x3, 0x5140), hi23 = __byte_perm(x2, x3, 0x7362);
-                                    const uint32_t t[4] = {__byte_perm(lo01, lo23, 0x5410), __byte_perm(lo01, lo23, 0x7632),
-                                                           __byte_perm(hi01, hi23, 0x5410), __byte_perm(hi01, hi23, 0x7632)};
-                                    const uint4 dr = pl ? d1 : d2;             // plane 1 meets r2, plane 2 meets r1
+                        for (int tj = 0; tj < 4; ++tj) {
+                            if (warp + (t0 + tj) * kRingWarps < ncol) {
+                                const uint32_t pel = __byte_perm(r4[tj][0], r4[tj][1], 0x6420), pol = __byte_perm(r4[tj][0], r4[tj][1], 0x7531);
+                                const uint32_t peh = __byte_perm(r4[tj][2], r4[tj][3], 0x6420), poh = __byte_perm(r4[tj][2], r4[tj][3], 0x7531);
 #pragma unroll
-                                    for (int b = 0; b < 4; ++b) {
-                                        const int f = b * NG + g;
-                                        ib[f][0] = dp4a_us(t[b], dr.x, ib[f][0]);
-                                        ib[f][1] = dp4a_us(t[b], dr.y, ib[f][1]);
-                                        ib[f][2] = dp4a_us(t[b], dr.z, ib[f][2]);
-                                        if constexpr (NS == 4) ib[f][NS - 1] = dp4a_us(t[b], dr.w, ib[f][NS - 1]);
-                                    }
-                                }
+                                for (int g = 0; g < NG; ++g)
+                                    mma_u8s8(acc[t0 + tj][g], group_bytes<CB>(pel, g), group_bytes<CB>(pol, g), group_bytes<CB>(peh, g),
+                                             group_bytes<CB>(poh, g), b0, b1);
                             }
                         }
-                    } else {
+                    }
+                    if (C > 1) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
+                        if (++slot == slots) { slot = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (C == 1) {                        // the retained single chunk goes back now, both planes
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot_a));
+                    mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot_a2));
+                }
+            }
+            // columns 2t, 2t+1 of lane t < 2 are digits 2t, 2t+1: combine, add the pair of lanes, send.
+            // Accumulator rows g, g+8 are bytes 2g, 2g+1 of the column.
+#pragma unroll
+            for (int ti = 0; ti < TI; ++ti) {
+                const int col = warp + ti * kRingWarps;
+                if (col < ncol) {
+#pragma unroll
+                    for (int g = 0; g < NG; ++g) {
+#pragma unroll
+                        for (int odd = 0; odd < 2; ++odd) {
+                            // digit pair of this lane in double (exact), the other pair comes from lane t+1
+                            const double pair = (double)acc[ti][g][2 * odd] + 128.0 * (double)acc[ti][g][2 * odd + 1];
+                            const double upper = __shfl_down_sync(0xffffffffu, pair, 1);
+                            const int byte_in_part = col * 16 + 2 * gl + odd;
+                            const int q = byte_in_part >> 2, b = byte_in_part & 3;
+                            if (tl == 0 && q < wcnt) {
+                                const int f = q * FPW + b * NG + g;
+                                const int owner = min((int)__umulhi((unsigned)f, sub_magic), a.nb - 1);     // f / sub, f < 2^16
+                                ll_store(rs_mine + ((size_t)owner * a.nb + bi) * subp + (f - owner * a.sub),
+                                         (float)((pair + 16384.0 * upper) * delta_r), tag);
+                            }
+                        }
+                    }
+                }
+            }
+        } else
+            {
+                const int q = ql;
+                const bool active = (group < ngroups) && (q < wcnt);
+                float acc[FPW];
+#pragma unroll
+                for (int i = 0; i < FPW; ++i) acc[i] = 0.0f;
+                for (int ci = 0; ci < C; ++ci) {
+                    const int chunk = C - 1 - ci;
+                    const int rows = min(a.cr, rcnt - chunk * a.cr);
+                    int use_slot = slot_a;
+                    if (C > 1) {
+                        ring_wait(sh->full + slot, phase, &sh->abort_flag, a.status, 7);
+                        use_slot = slot;
+                    }
+                    if (active) {
+                        const uint32_t* col1 = ring + (size_t)use_slot * slot_words + q;
+                        const uint32_t* col2 = col1 + (size_t)a.cr * pitch;
                         const float* rr = res + 2 * chunk * a.cr;
 #pragma unroll 4
                         for (int lr = group; lr < rows; lr += ngroups) {
-                            const uint32_t u1 = col1[(size_t)lr * a.wc];
-                            const uint32_t u2 = col2[(size_t)lr * a.wc];
+                            const uint32_t u1 = col1[(size_t)lr * pitch];
+                            const uint32_t u2 = col2[(size_t)lr * pitch];
                             const float2 rv = *reinterpret_cast<const float2*>(rr + 2 * lr);
                             const float r1 = rv.x, r2 = rv.y;
 #pragma unroll
@@ -705,39 +869,34 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                             }
                         }
                     }
-                }
-                if (C > 1) {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
-                    if (++slot == slots) { slot = 0; phase ^= 1u; }
-                }
-            }
-            if constexpr (!TABLE) {
-#pragma unroll
-                for (int i = 0; i < FPW; ++i) acc[i] = (float)((double)combine_digits<NS>(ib[i]) * delta_r);
-            }
-            if (ngroups > 1) {
-                consumer_sync();
-                if (active) {
-#pragma unroll
-                    for (int i = 0; i < FPW; ++i) gred[(group * FPW + i) * lanes_q + ql] = acc[i];
-                }
-                consumer_sync();
-                if (active && group == 0) {
-#pragma unroll
-                    for (int i = 0; i < FPW; ++i) {
-                        float tsum = gred[i * lanes_q + ql];
-                        for (int gidx = 1; gidx < ngroups; ++gidx) tsum += gred[(gidx * FPW + i) * lanes_q + ql];
-                        acc[i] = tsum;
+                    if (C > 1) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
+                        if (++slot == slots) { slot = 0; phase ^= 1u; }
                     }
                 }
-            }
-            if (active && group == 0) {
+                if (ngroups > 1) {
+                    consumer_sync();
+                    if (active) {
 #pragma unroll
-                for (int i = 0; i < FPW; ++i) ll_store(rs_mine + rs_off[i], acc[i], tag);
+                        for (int i = 0; i < FPW; ++i) gred[(group * FPW + i) * lanes_q + ql] = acc[i];
+                    }
+                    consumer_sync();
+                    if (active && group == 0) {
+#pragma unroll
+                        for (int i = 0; i < FPW; ++i) {
+                            float tsum = gred[i * lanes_q + ql];
+                            for (int gidx = 1; gidx < ngroups; ++gidx) tsum += gred[(gidx * FPW + i) * lanes_q + ql];
+                            acc[i] = tsum;
+                        }
+                    }
+                }
+                if (active && group == 0) {
+#pragma unroll
+                    for (int i = 0; i < FPW; ++i) ll_store(rs_mine + rs_off[i], acc[i], tag);
+                }
             }
-        }
-        if (C == 1) {                            // the retained single chunk goes back now
+        if (TABLE && C == 1) {                   // the retained single chunk goes back now
             __syncwarp();
             if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
             if (++slot == slots) { slot = 0; phase ^= 1u; }
@@ -890,9 +1049,13 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
 // Host side
 // ---------------------------------------------------------------------------------------------
 struct RingPlan {
-    int na, nb, wc, rc, cr, slots, sub;
+    int na, nb, wc, rc, cr, slots, sub, pitch;
     size_t smem;
 };
+
+// Rows of a chunk lie `pitch` words apart in shared memory.  The integer path reads 8 rows x 4 words per
+// tensor-core fragment load; a pitch of wc (a multiple of 32 words) would put all rows in the same banks.
+static int ring_pitch(bool table, int wc) { return table ? wc : wc + 4; }
 
 static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int sub, int cr, int slots, int nb, int G) {
     const int fpw = 32 / cb;
@@ -901,8 +1064,8 @@ static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int 
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
     bytes += sizeof(float) * ((table ? 2 * L * F : F) + (size_t)wc + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
     bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
-    bytes += 16 * 2 * (size_t)((rc + 3) / 4) + 128;          // + slack to align the ring to 128 bytes
-    bytes += sizeof(uint32_t) * (size_t)slots * 2 * cr * wc;
+    bytes += 256 * (size_t)((rc + 31) / 32) + (table ? 0 : sizeof(int) * 8 * (size_t)rc) + 128;   // + slack to align the ring
+    bytes += sizeof(uint32_t) * (size_t)slots * (table ? 2 : 1) * cr * ring_pitch(table, wc);   // uniform: one plane per slot
     return bytes;
 }
 
@@ -938,7 +1101,9 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         cr = (cr + 3) & ~3;                                   // phase B walks a slot four rows at a time
         cr = cr < 4 ? 4 : cr;
         if (cr > ((r.rc + 3) & ~3) || wide) cr = (r.rc + 3) & ~3;
+        if (!table) cr = r.rc <= 16 ? 16 : 32;                // integer path: fragments of 16 rows, k-slabs of 32 rows
         r.cr = cr;
+        r.pitch = ring_pitch(table, r.wc);
         if (sizeof(uint32_t) * 2 * (size_t)cr * r.wc >= (1u << 20)) return false;   // mbarrier tx-count range
         int slots = kRingMaxSlots;
         while (slots >= 2 && ring_smem_bytes(cb, table, r.wc, r.rc, d->bits, r.sub, cr, slots, r.nb, r.na * r.nb) > cap) --slots;
@@ -949,14 +1114,20 @@ static int make_ring_plan(const zipml_ctx* ctx, const zipml_dataset* d, const zi
         return true;
     };
 
-    const int na_min = (int)((words + kRingConsumers - 1) / kRingConsumers);
+    // parts are at most one word per consumer wide; phase B of the integer path keeps at most kRingTasks
+    // accumulator sets per warp (8 words x groups each), which caps 2-bit parts at 128 words
+    const int wc_max = table ? kRingConsumers : min(kRingConsumers, 64 * kRingTasks / (8 / cb));
+    const int na_min = (int)((words + wc_max - 1) / wc_max);
     if (p->grid_feature_parts > 0 || p->grid_row_parts > 0) {
         int na = p->grid_feature_parts > 0 ? p->grid_feature_parts : 1;
         int nb = p->grid_row_parts > 0 ? p->grid_row_parts : 1;
         if ((int64_t)na * 32 > ring_round_up((int)words, 32)) na = (int)((words + 31) / 32);
         if (na < na_min) na = na_min;          // the request is a hint: parts never exceed one word column per thread
         if (nb > B) nb = (int)B;
-        return shape(na, nb, plan) ? ZIPML_OK : ZIPML_ERR_WORKSPACE;
+        // more row parts than asked for when the tile of a part does not fit shared memory
+        for (; nb <= B && na * nb <= sms; ++nb)
+            if (shape(na, nb, plan)) return ZIPML_OK;
+        return ZIPML_ERR_WORKSPACE;
     }
     // Fewest feature parts (widest contiguous row pieces).  Row parts: small steps are bound by the
     // exchange, whose cost grows with the number of CTAs, not by the tile -- measured on 0.25-1 MiB
@@ -983,7 +1154,7 @@ static int64_t plane_wc_check(int wc) { return (int64_t)wc; }
 
 // Tensor maps over the two planes seen as m x row_words matrices of 32-bit words.  The encoder is a
 // driver entry point looked up through the runtime (no link against the driver library).
-static int encode_plane_maps(zipml_ctx* ctx, const zipml_dataset* d, int wc, int cr, CUtensorMap* out) {
+static int encode_plane_maps(zipml_ctx* ctx, const zipml_dataset* d, int box_words, int cr, bool wide_elements, CUtensorMap* out) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -997,15 +1168,18 @@ static int encode_plane_maps(zipml_ctx* ctx, const zipml_dataset* d, int wc, int
         }
         ctx->tmap_encode = fn;
     }
-    if (wc > 256 || cr > 256 || (wc * 4) % 16 != 0) return ZIPML_ERR_WORKSPACE;
-    const cuuint64_t gdim[2] = {(cuuint64_t)(d->row_bytes / 4), (cuuint64_t)d->m};
+    // 32-bit elements, or 64-bit ones for boxes wider than 256 words (a box dimension holds at most 256 elements)
+    const int esz = wide_elements ? 8 : 4;
+    const int box_elems = box_words * 4 / esz;
+    if (box_elems > 256 || cr > 256 || (box_words * 4) % 16 != 0) return ZIPML_ERR_WORKSPACE;
+    const cuuint64_t gdim[2] = {(cuuint64_t)(d->row_bytes / esz), (cuuint64_t)d->m};
     const cuuint64_t gstride[1] = {(cuuint64_t)d->row_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)wc, (cuuint32_t)cr};
+    const cuuint32_t box[2] = {(cuuint32_t)box_elems, (cuuint32_t)cr};
     const cuuint32_t estr[2] = {1, 1};
     const void* planes[2] = {d->plane1, d->plane2};
     for (int i = 0; i < 2; ++i) {
         const CUresult r = reinterpret_cast<EncodeFn>(ctx->tmap_encode)(
-            &out[i], CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(planes[i]), gdim, gstride, box, estr,
+            &out[i], wide_elements ? CU_TENSOR_MAP_DATA_TYPE_UINT64 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(planes[i]), gdim, gstride, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return ZIPML_ERR_CUDA;
@@ -1060,7 +1234,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.lr = p->lr; a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
     a.seed = p->seed; a.epoch = (uint32_t)p->epoch;
     a.na = plan.na; a.nb = plan.nb; a.wc = plan.wc; a.rc = plan.rc; a.stages = plan.slots;
-    a.cr = plan.cr; a.sub = plan.sub;
+    a.cr = plan.cr; a.sub = plan.sub; a.pitch = plan.pitch;
     a.pd = nullptr; a.pg = nullptr; a.ps = nullptr; a.barrier = nullptr;
     a.ll_pd = reinterpret_cast<unsigned long long*>(ctx->ws + o_ll);
     a.ll_rs = a.ll_pd + n_pd;
@@ -1080,8 +1254,13 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     CUtensorMap tmaps[2];
     memset(tmaps, 0, sizeof(tmaps));
     a.use_tmap = 0;
-    if (a.row_words != plane_wc_check(plan.wc) && d->m < 0x7fffffffLL && a.row_words < 0x7fffffffLL) {
-        if (encode_plane_maps(ctx, d, plan.wc, plan.cr, tmaps) == ZIPML_OK) a.use_tmap = 1;
+    if (d->m < 0x7fffffffLL && a.row_words < 0x7fffffffLL) {
+        if (table) {
+            if (a.row_words != plane_wc_check(plan.wc) && encode_plane_maps(ctx, d, plan.wc, plan.cr, false, tmaps) == ZIPML_OK)
+                a.use_tmap = 1;
+        } else if (encode_plane_maps(ctx, d, plan.pitch, plan.cr, true, tmaps) == ZIPML_OK) {
+            a.use_tmap = 1;                    // uniform grids: one padded box per plane and chunk
+        }
     }
     // packet tags are 32-bit step counters starting at 1
     const int64_t max_steps = 0x7fffffffLL;
