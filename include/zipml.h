@@ -54,7 +54,10 @@ enum {
     ZIPML_ENGINE_LEAN = 4,       /* one cooperative launch for small minibatch tiles: row parts only,
                                     two barriers and two packet exchanges per step                    */
     ZIPML_ENGINE_CLUSTER = 5     /* one thread-block cluster (at most 16 row parts) for small tiles:
-                                    gradients and model travel between the CTAs' shared memories      */
+                                    gradients and model travel between the CTAs' shared memories.
+                                    Uniform grids contract in fp32 or, on taller tiles, on the int8
+                                    tensor cores; the environment variable ZIPML_CLUSTER_INT8=0/1
+                                    overrides that choice                                             */
 };
 
 typedef struct zipml_ctx zipml_ctx;

@@ -175,6 +175,33 @@ def test_sgd_epoch_parity(ctx, case, engine):
         assert rel(xb.cpu().numpy(), x_ref) <= MODEL_TOL
 
 
+@pytest.mark.parametrize("int8", ["0", "1"])
+@pytest.mark.parametrize("case", SGD_CASES[:5], ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
+def test_cluster_engine_both_contractions(ctx, case, int8, monkeypatch):
+    """The cluster engine's fp32 and int8 tensor-core contractions, forced, against the oracle."""
+    monkeypatch.setenv("ZIPML_CLUSTER_INT8", int8)
+    key, m, n, bits, batch, lr = case
+    _, A, b, _ = workload(key, m, n, seed=3)
+    ods = oracle.quantize(A, bits, seed=5)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    T = (m + batch - 1) // batch
+    x0 = (np.random.default_rng(2).standard_normal(n) * 0.1).astype(np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr)
+    x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, num_steps=T - 1)
+    _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=T - 1, num_steps=1, want_grad=True)
+    for fb in (0, 3, 16):
+        x = to_dev(x0, ctx)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=binding.ENGINE_CLUSTER, grid_row_parts=fb)
+        ctx.zipml_sync()
+        assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL, fb
+        xb = to_dev(x_before, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=T - 1, num_steps=1, engine=binding.ENGINE_CLUSTER,
+                            grid_row_parts=fb, grad_out=g)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL, fb
+
+
 def test_sgd_engines_and_grids_agree_bitwise_where_the_reduction_order_is_the_same(ctx):
     _, A, b, _ = workload("c2", 1500, 300, seed=2)
     ods = oracle.quantize(A, 8, seed=1)
