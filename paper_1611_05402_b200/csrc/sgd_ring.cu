@@ -204,20 +204,19 @@ __device__ __forceinline__ float consumer_max(float v, RingShared* sh, int slot)
 
 // Shared memory plan, F = wc * FPW features per CTA:
 //   RingShared
-//   tab                         uniform: digit words of w, uint4 [group][word]; table: WL[L*F] then LV[L*F] floats
-//                               ([code][slot][word])
-//   lw[wc] float                uniform: sum over a word's features of lo * x~ (its share of lo^T x~)
+//   tab                         uniform: digits of w as B operands, bytes [k-slab of 8 words][group][digit][32];
+//                               table: WL[L*F] then LV[L*F] floats ([code][slot][word])
 //   xown[sub] float             master model of the CTA's own sub-slice
 //   gsub[sub] float             gradient of the own sub-slice
 //   gbuf[nb*(sub+2)] float      collected row parts of the own sub-slice (+ residual sums)
 //   nbuf[2*G] float             collected partial norms
-//   gred[kRingConsumers*FPW]    cross-group reduction of phase B
+//   gred[kRingConsumers*FPW]    table: cross-group reduction of phase B
 //   res[2*rc] float             residuals
 //   rdig[ceil(rc/32)][2][4][32] bytes  uniform: digits of the residuals as B operands: per 32 rows, per
 //                               residual (r1, r2), per digit a 32-byte k vector (row order of phase B)
 //   dacc[rc][2][4] int          uniform: digit sums of the dots per (row, plane), filled by the warps' atomics
 //   bsm[2][rc] float            labels of the current and the next step's rows
-//   ring[slots][2][cr][wc] u32  code chunks
+//   ring[slots][planes][cr][pitch] u32  code chunks (uniform: one plane per slot, pitch = wc + 4; table: both, pitch = wc)
 template <int CB, bool TABLE>
 __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs a, const __grid_constant__ CUtensorMap tm1,
                                                                   const __grid_constant__ CUtensorMap tm2) {
@@ -231,13 +230,12 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
     const int G = a.na * a.nb;
     const int subp = a.sub + 2;                                  // packets per (owner, writer)
     float* tab = reinterpret_cast<float*>(s_raw + ((sizeof(RingShared) + 15) & ~(size_t)15));
-    float* lw = tab + (TABLE ? 2 * L * F : F);
-    float* xown = lw + a.wc;
+    float* xown = tab + (TABLE ? 2 * L * F : F);
     float* gsub = xown + a.sub;
     float* gbuf = gsub + a.sub;
     float* nbuf = gbuf + ((a.nb * subp + 3) & ~3);
     float* gred = nbuf + ((2 * G + 3) & ~3);
-    float* res = gred + kRingConsumers * FPW;
+    float* res = gred + (TABLE ? kRingConsumers * FPW : 0);
     unsigned char* rdig = reinterpret_cast<unsigned char*>(res + ((2 * a.rc + 3) & ~3));
     int* dacc = reinterpret_cast<int*>(rdig + (size_t)((a.rc + 31) / 32) * 256);
     float* bsm = reinterpret_cast<float*>(dacc + (TABLE ? 0 : 8 * a.rc));
@@ -1062,8 +1060,8 @@ static size_t ring_smem_bytes(int cb, bool table, int wc, int rc, int bits, int 
     const size_t F = (size_t)wc * fpw, L = (size_t)1 << bits;
     const size_t subp = (size_t)sub + 2;
     size_t bytes = (sizeof(RingShared) + 15) & ~(size_t)15;
-    bytes += sizeof(float) * ((table ? 2 * L * F : F) + (size_t)wc + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
-    bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (size_t)kRingConsumers * fpw + 2 * (size_t)((2 * rc + 3) & ~3));
+    bytes += sizeof(float) * ((table ? 2 * L * F : F) + 2 * (size_t)sub + (((size_t)nb * subp + 3) & ~(size_t)3));
+    bytes += sizeof(float) * (((2 * (size_t)G + 3) & ~(size_t)3) + (table ? (size_t)kRingConsumers * fpw : 0) + 2 * (size_t)((2 * rc + 3) & ~3));
     bytes += 256 * (size_t)((rc + 31) / 32) + (table ? 0 : sizeof(int) * 8 * (size_t)rc) + 128;   // + slack to align the ring
     bytes += sizeof(uint32_t) * (size_t)slots * (table ? 2 : 1) * cr * ring_pitch(table, wc);   // uniform: one plane per slot
     return bytes;
