@@ -254,7 +254,8 @@ int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t 
     int rc = check_dataset(data);
     if (rc != ZIPML_OK) return rc;
     const size_t tab = (data->level_mode == ZIPML_LEVELS_TABLE ? ((size_t)1 << data->bits) : 1) * (size_t)data->n;
-    rc = ws_reserve(ctx, carve_size(sizeof(double) * (kLossPartials + 2) + sizeof(float) * tab));
+    // (+ slack: the digit vectors of the uniform path round the row up to 64 bytes)
+    rc = ws_reserve(ctx, carve_size(sizeof(double) * (kLossPartials + 2) + sizeof(float) * tab + 2048));
     if (rc != ZIPML_OK) return rc;
     return launch_loss_codes(ctx, data, b, x, reinterpret_cast<double*>(ctx->ws), kLossPartials, loss_out);
 }

@@ -1,6 +1,7 @@
 // Training loss (paper Eq. (leastsquares) with l = a^T x - b) on the dense samples, its unbiased
 // estimate from the two code planes, and the allocation-free variant of the latter.
 #include "common.cuh"
+#include "int_digits.cuh"
 #include "internal.h"
 
 namespace zipml {
@@ -87,6 +88,115 @@ __global__ void __launch_bounds__(256) loss_codes_kernel(const uint32_t* __restr
     if (threadIdx.x == 0) partials[blockIdx.x] = total;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same estimate for uniform grids on the int8 tensor cores: a pure streaming pass (no step-to-step
+// dependency), so it shows what the unpack-and-dot arithmetic of the SGD step reaches against HBM.
+// w = step * x becomes four balanced base-128 int8 digits per entry (one rounding, 2^-27 of the
+// largest |w|); a warp takes 16 rows, its lanes load 16 bytes of codes per row and 64-byte span
+// straight from global memory (rows g and g+8 of lane group g; four lanes cover the span), and every
+// 8 bytes of a lane's 16 are one mma.sync m16n8k32 (u8 x s8) against the matching 8 bytes of each
+// digit's vector (digits in the byte order of the codes, so the operand's k order is simply the
+// lane's own byte order).  Digit sums are exact; they are combined in double.
+// ---------------------------------------------------------------------------------------------
+// Digit vectors of w: wdig[group][digit][byte of the row], row_bytes rounded up to 64 per vector.
+template <int CB>
+__global__ void __launch_bounds__(1024) loss_digits_kernel(const float* __restrict__ lo, const float* __restrict__ step,
+                                                           const float* __restrict__ x, int64_t n, int64_t vec_bytes,
+                                                           signed char* __restrict__ wdig, double* __restrict__ base_out) {
+    constexpr int NG = IntPath<CB>::NG, NS = IntPath<CB>::NS, FPW = 32 / CB;
+    __shared__ double red[40];
+    __shared__ float smax[32];
+    double base = 0.0;
+    float wm = 0.0f;
+    for (int64_t j = threadIdx.x; j < n; j += blockDim.x) {
+        const float xv = x[j];
+        wm = fmaxf(wm, fabsf(step[j] * xv));
+        base += (double)lo[j] * (double)xv;
+    }
+    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+    if ((threadIdx.x & 31) == 0) smax[threadIdx.x >> 5] = wm;
+    base = block_sum(base, red);                  // its barriers also publish smax
+    float wmax = 0.0f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) wmax = fmaxf(wmax, smax[w]);
+    const float inv = wmax > 0.0f ? (float)IntPath<CB>::QMAX / wmax : 0.0f;
+    if (threadIdx.x == 0) { base_out[0] = base; base_out[1] = (double)wmax / (double)IntPath<CB>::QMAX; }
+    // feature j sits in byte (j / FPW) * 4 + (j % FPW) / NG of the row, code group (j % FPW) % NG
+    for (int64_t idx = threadIdx.x; idx < vec_bytes * NG; idx += blockDim.x) {
+        const int64_t byte = idx / NG;
+        const int g = (int)(idx - byte * NG);
+        const int64_t j = (byte >> 2) * FPW + (byte & 3) * NG + g;
+        int d[NS];
+        balanced_digits<NS>(j < n ? __float2int_rn(step[j] * x[j] * inv) : 0, d);
+#pragma unroll
+        for (int s = 0; s < NS; ++s) wdig[((int64_t)g * NS + s) * vec_bytes + byte] = (signed char)d[s];
+    }
+}
+
+template <int CB>
+__global__ void __launch_bounds__(512) loss_codes_imma_kernel(const unsigned char* __restrict__ p1, const unsigned char* __restrict__ p2,
+                                                              int64_t row_bytes, int64_t m, int64_t vec_bytes,
+                                                              const signed char* __restrict__ wdig, const double* __restrict__ base_in,
+                                                              const float* __restrict__ b, double* __restrict__ partials) {
+    constexpr int NG = IntPath<CB>::NG, NS = IntPath<CB>::NS;
+    __shared__ double red[40];
+    const int lane = threadIdx.x & 31, gl = lane >> 2, tl = lane & 3;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const double base = base_in[0], delta = base_in[1];
+    const int64_t nblocks = (m + 15) / 16;
+    const int64_t nspans = (row_bytes + 63) / 64;
+    double total = 0.0;
+    for (int64_t blk = warp_global; blk < nblocks; blk += nwarps) {
+        const int64_t ra = min(blk * 16 + gl, m - 1), rh = min(blk * 16 + gl + 8, m - 1);
+        const unsigned char* a1 = p1 + ra * row_bytes + 16 * tl;
+        const unsigned char* h1 = p1 + rh * row_bytes + 16 * tl;
+        const unsigned char* a2 = p2 + ra * row_bytes + 16 * tl;
+        const unsigned char* h2 = p2 + rh * row_bytes + 16 * tl;
+        int c1[4] = {0, 0, 0, 0}, c2[4] = {0, 0, 0, 0};
+#pragma unroll 2
+        for (int64_t sp = 0; sp < nspans; ++sp) {
+            const int64_t off = sp * 64;
+            uint4 ua = make_uint4(0u, 0u, 0u, 0u), uh = ua, va = ua, vh = ua;
+            if (off + 16 * tl < row_bytes) {                      // rows are whole multiples of 16 bytes
+                ua = __ldcs(reinterpret_cast<const uint4*>(a1 + off));
+                uh = __ldcs(reinterpret_cast<const uint4*>(h1 + off));
+                va = __ldcs(reinterpret_cast<const uint4*>(a2 + off));
+                vh = __ldcs(reinterpret_cast<const uint4*>(h2 + off));
+            }
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+                uint4 bd = make_uint4(0u, 0u, 0u, 0u);            // digit gl of this lane's 16 bytes
+                if (gl < NS) bd = __ldg(reinterpret_cast<const uint4*>(wdig + ((int64_t)g * NS + gl) * vec_bytes + off + 16 * tl));
+                mma_u8s8(c1, group_bytes<CB>(ua.x, g), group_bytes<CB>(uh.x, g), group_bytes<CB>(ua.y, g), group_bytes<CB>(uh.y, g), bd.x, bd.y);
+                mma_u8s8(c1, group_bytes<CB>(ua.z, g), group_bytes<CB>(uh.z, g), group_bytes<CB>(ua.w, g), group_bytes<CB>(uh.w, g), bd.z, bd.w);
+                mma_u8s8(c2, group_bytes<CB>(va.x, g), group_bytes<CB>(vh.x, g), group_bytes<CB>(va.y, g), group_bytes<CB>(vh.y, g), bd.x, bd.y);
+                mma_u8s8(c2, group_bytes<CB>(va.z, g), group_bytes<CB>(vh.z, g), group_bytes<CB>(va.w, g), group_bytes<CB>(vh.w, g), bd.z, bd.w);
+            }
+        }
+        // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3])
+        double v[4];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const double q1 = (double)c1[2 * e] + 128.0 * (double)c1[2 * e + 1];
+            const double q2 = (double)c2[2 * e] + 128.0 * (double)c2[2 * e + 1];
+            v[2 * e] = q1 + 16384.0 * __shfl_down_sync(0xffffffffu, q1, 1);
+            v[2 * e + 1] = q2 + 16384.0 * __shfl_down_sync(0xffffffffu, q2, 1);
+        }
+        if (tl == 0) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int64_t k = blk * 16 + gl + 8 * e;
+                if (k < m) {
+                    const double bk = (double)__ldg(b + k);
+                    total += (v[2 * e] * delta + base - bk) * (v[2 * e + 1] * delta + base - bk);
+                }
+            }
+        }
+    }
+    total = block_sum(total, red);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
 __global__ void loss_finish_kernel(const double* __restrict__ partials, int count, double scale, double* out) {
     __shared__ double red[40];
     double v = 0.0;
@@ -100,9 +210,26 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
     const int cb = container_bits(d->bits);
     const bool table = d->level_mode == ZIPML_LEVELS_TABLE;
     const int L = 1 << d->bits;
-    // scratch behind the partials: base (1 double) then the w table
+    // scratch behind the partials: base and the fixed-point unit (2 doubles), then the w table or digit vectors
     double* base = partials + max_partials;
     float* wtab = reinterpret_cast<float*>(base + 2);
+    if (!table) {
+        // digit vectors take (8 / cb) * 4 * roundup64(row_bytes) bytes <= 4 n + slack: they fit the table's space
+        const int64_t vec_bytes = (d->row_bytes + 63) / 64 * 64;
+        signed char* wdig = reinterpret_cast<signed char*>(wtab);
+        int blocks = ctx->sm_count * 2;                            // 2 x 16 warps per SM, 16 rows per warp and turn
+        if (blocks > max_partials) blocks = max_partials;
+        const int64_t need = ((d->m + 15) / 16 + 15) / 16;
+        if (blocks > need) blocks = (int)need;
+#define ZIPML_LAUNCH_LI(CB_) \
+    loss_digits_kernel<CB_><<<1, 1024, 0, ctx->stream>>>(d->feat_lo, d->feat_step, x, d->n, vec_bytes, wdig, base); \
+    loss_codes_imma_kernel<CB_><<<blocks, 512, 0, ctx->stream>>>(d->plane1, d->plane2, d->row_bytes, d->m, vec_bytes, wdig, base, b, partials)
+        if (cb == 2) { ZIPML_LAUNCH_LI(2); } else if (cb == 4) { ZIPML_LAUNCH_LI(4); } else { ZIPML_LAUNCH_LI(8); }
+#undef ZIPML_LAUNCH_LI
+        loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)d->m), loss_out);
+        ctx->launches += 3;
+        return cuda_status(cudaGetLastError());
+    }
     loss_prepare_kernel<<<1, 1024, 0, ctx->stream>>>(d->feat_lo, d->feat_step, d->levels, x, d->n, L, table, wtab, base);
     int blocks = ctx->sm_count * 8;
     if (blocks > max_partials) blocks = max_partials;
