@@ -29,12 +29,18 @@ def test_static_scratch_loss_matches_regular_entry_point_twice_in_a_row():
             x = (xs * 0.8).contiguous()
             want = ctx.zipml_loss(binding.LOSS_CODES, b, x, data=ds)
             ctx.zipml_sync()
-            before = torch.cuda.memory_allocated(dev)
-            got = binding.zipml_loss_codes_static(ds, b, x, out=torch.empty(1, dtype=torch.float64, device=dev))
-            again = binding.zipml_loss_codes_static(ds, b, x, out=torch.empty(1, dtype=torch.float64, device=dev))
+            out1 = torch.empty(1, dtype=torch.float64, device=dev)
+            out2 = torch.empty(1, dtype=torch.float64, device=dev)
+            # the first call on a device looks up the scratch address and loads the kernels; the second
+            # call is watched at the driver level (torch's own counters do not see a cudaMalloc
+            # made inside the library): the device's free memory must not shrink
+            got = binding.zipml_loss_codes_static(ds, b, x, out=out1)
             torch.cuda.synchronize(dev)
+            free_before = torch.cuda.mem_get_info(dev)[0]
+            again = binding.zipml_loss_codes_static(ds, b, x, out=out2)
+            torch.cuda.synchronize(dev)
+            assert free_before - torch.cuda.mem_get_info(dev)[0] < (1 << 20)
             results.append((want.item(), got.item(), again.item()))
-            assert before <= torch.cuda.memory_allocated(dev) <= before + 1024   # only the two 8-byte outputs
         for want, got, again in results:
             assert abs(got - want) <= 1e-6 * abs(want)        # the tolerance of the other loss tests
             assert again == got                                  # same scratch, same order: bit-identical
