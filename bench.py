@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # (workload, engine) -> bytes; an entry is removed when its kernel changes after the capture
 NCU_TRAFFIC_BYTES = {("c2", 5): 202.07e6 + 4.11e6}
 ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
-                  5: "sgd_cluster_kernel"}
+                  5: "sgd_cluster_kernel", 6: "sgd_stream_kernel"}
 
 
 def measured_peaks():
@@ -119,7 +119,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
     ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
-    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster", "stream"])
     ap.add_argument("--feature-parts", type=int, default=0)
     ap.add_argument("--row-parts", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -184,7 +184,8 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT,
-              "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN, "cluster": binding.ENGINE_CLUSTER}[args.engine]
+              "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN, "cluster": binding.ENGINE_CLUSTER,
+              "stream": binding.ENGINE_STREAM}[args.engine]
 
     w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
     ctx = binding.Context(dev)

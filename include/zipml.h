@@ -46,18 +46,25 @@ enum { ZIPML_LEVELS_UNIFORM = 0, ZIPML_LEVELS_TABLE = 1 };
 enum { ZIPML_LOSS_DENSE = 0, ZIPML_LOSS_CODES = 1 };
 /* How zipml_sgd_epoch runs its minibatch chain.  Results do not depend on the choice. */
 enum {
-    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; else ring  */
+    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; beyond that
+                                   stream where it applies, else ring                                 */
     ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
     ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
     ZIPML_ENGINE_RING = 3,       /* one cooperative launch; producer warp streams code chunks through a
                                     shared-memory ring, gradients meet by reduce-scatter / all-gather  */
     ZIPML_ENGINE_LEAN = 4,       /* one cooperative launch for small minibatch tiles: row parts only,
                                     two barriers and two packet exchanges per step                    */
-    ZIPML_ENGINE_CLUSTER = 5     /* one thread-block cluster (at most 16 row parts) for small tiles:
+    ZIPML_ENGINE_CLUSTER = 5,    /* one thread-block cluster (at most 16 row parts) for small tiles:
                                     gradients and model travel between the CTAs' shared memories.
                                     Uniform grids contract in fp32 or, on taller tiles, on the int8
                                     tensor cores; the environment variable ZIPML_CLUSTER_INT8=0/1
                                     overrides that choice                                             */
+    ZIPML_ENGINE_STREAM = 6      /* one cooperative launch for large tiles on uniform grids with an fp32
+                                    model and gradient: both passes of a step read the codes straight
+                                    from global memory into int8 tensor-core fragments (the second pass
+                                    from L2), a CTA owns whole column blocks of the gradient, one grid
+                                    barrier per step.  ZIPML_ERR_WORKSPACE for level tables, quantized
+                                    model or gradient, batches above 8192 rows                        */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -102,7 +109,10 @@ typedef struct zipml_sgd_params {
                                    0 step start, 1 tile arrived, 2 residuals ready, 3 gradient
                                    parts sent, 4 own features summed, 5 model published, 6 model
                                    collected, 7 step end.  The last step of a call stops after
-                                   mark 4.  Other engines ignore the request.                         */
+                                   mark 4.  Stream engine: 0 step start, 1 own dots added, 2 barrier
+                                   passed, 3 residual digits ready, 4 own gradient blocks summed,
+                                   5 model updated and digits published.  Other engines ignore the
+                                   request.                                                           */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

@@ -13,7 +13,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
-ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER = 0, 1, 2, 3, 4, 5
+ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM = 0, 1, 2, 3, 4, 5, 6
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
 EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",

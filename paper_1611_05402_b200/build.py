@@ -5,7 +5,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libzipml.so")
-SOURCES = ["api.cu", "quantize.cu", "levels.cu", "sgd.cu", "sgd_ring.cu", "sgd_lean.cu", "sgd_cluster.cu", "loss.cu"]
+SOURCES = ["api.cu", "quantize.cu", "levels.cu", "sgd.cu", "sgd_ring.cu", "sgd_lean.cu", "sgd_cluster.cu", "sgd_stream.cu", "loss.cu"]
 HEADERS = ["common.cuh", "internal.h", "sgd_common.cuh", "int_digits.cuh", os.path.join("..", "..", "include", "zipml.h")]
 
 

@@ -198,7 +198,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (!b || !x || params->batch <= 0) return ZIPML_ERR_INVALID_ARG;
     if (params->model_bits != 0 && (params->model_bits < 2 || params->model_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
     if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
-    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_CLUSTER) return ZIPML_ERR_INVALID_ARG;
+    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_STREAM) return ZIPML_ERR_INVALID_ARG;
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
@@ -213,6 +213,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->engine == ZIPML_ENGINE_RING) return launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_LEAN) return launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
+    if (params->engine == ZIPML_ENGINE_STREAM) return launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_AUTO) {
         // Small minibatch tiles are bound by the step-to-step chain, not by HBM: one cluster whose CTAs
         // exchange through shared memory, else row parts exchanging through L2.  Larger tiles stream
@@ -223,6 +224,10 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
             rc = launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
             if (rc != ZIPML_ERR_WORKSPACE) return rc;
             rc = launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
+            if (rc != ZIPML_ERR_WORKSPACE) return rc;
+        }
+        else {
+            rc = launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, true);
             if (rc != ZIPML_ERR_WORKSPACE) return rc;
         }
         rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);

@@ -79,6 +79,10 @@ int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
                     int64_t first_step, int64_t num_steps, float* grad_out);
 int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                        int64_t first_step, int64_t num_steps, float* grad_out);
+// Stream engine (uniform grids, fp32 model and gradient).  With only_if_profitable it declines
+// (ZIPML_ERR_WORKSPACE) shapes whose steps are too narrow or too short for it.
+int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                      int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
 int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                      int64_t first_step, int64_t num_steps, float* grad_out);

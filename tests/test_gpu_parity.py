@@ -144,7 +144,8 @@ GRIDS = [(0, 0), (1, 1), (1, 5), (2, 3), (3, 1)]
 
 
 @pytest.mark.parametrize("case", SGD_CASES, ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
-@pytest.mark.parametrize("engine", [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER])
+@pytest.mark.parametrize("engine", [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER,
+                                    binding.ENGINE_STREAM])
 def test_sgd_epoch_parity(ctx, case, engine):
     key, m, n, bits, batch, lr = case
     _, A, b, _ = workload(key, m, n, seed=1)
@@ -200,6 +201,45 @@ def test_cluster_engine_both_contractions(ctx, case, int8, monkeypatch):
                             grid_row_parts=fb, grad_out=g)
         ctx.zipml_sync()
         assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL, fb
+
+
+@pytest.mark.parametrize("case", [
+    # key, m, n, bits, batch, lr: rows wide enough for many column blocks and several pass-A parts
+    ("c5", 700, 20000, 4, 300, 1e-4),
+    ("c2", 1300, 9001, 8, 520, 1e-3),
+    ("c3", 1100, 40000, 2, 500, 5e-4),
+    ("c4u", 900, 12345, 3, 333, 1e-3),
+], ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
+def test_stream_engine_wide_rows(ctx, case):
+    """The stream engine on shapes that give it many CTAs, from a zero and from a non-zero model, twice."""
+    key, m, n, bits, batch, lr = case
+    _, A, b, _ = workload(key, m, n, seed=8)
+    ods = oracle.quantize(A, bits, seed=9)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    T = (m + batch - 1) // batch
+    for x0 in (np.zeros(n, np.float32), (np.random.default_rng(4).standard_normal(n) * 0.05).astype(np.float32)):
+        x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr)
+        x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, num_steps=T - 1)
+        _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=T - 1, num_steps=1, want_grad=True)
+        runs = []
+        for fb in (0, 0, 61):
+            x = to_dev(x0, ctx)
+            ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=binding.ENGINE_STREAM, grid_row_parts=fb)
+            ctx.zipml_sync()
+            assert ctx.zipml_last_engine() == binding.ENGINE_STREAM
+            runs.append(x.cpu().numpy())
+            assert rel(runs[-1], x_ref) <= MODEL_TOL, fb
+        # integer sums in any order: the same bits run to run and for any grid
+        assert (runs[0] == runs[1]).all() and (runs[0] == runs[2]).all()
+        xb = to_dev(x_before, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=T - 1, num_steps=1, engine=binding.ENGINE_STREAM, grad_out=g)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL
+    # what it does not cover is declined, not approximated
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=binding.ENGINE_STREAM, model_bits=8)
+    assert e.value.code == binding.ERR_WORKSPACE
 
 
 def test_sgd_engines_and_grids_agree_bitwise_where_the_reduction_order_is_the_same(ctx):
