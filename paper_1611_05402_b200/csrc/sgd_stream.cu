@@ -3,29 +3,33 @@
 // A step of the double-sampled minibatch SGD (paper Eq. (double) in its symmetrised form, footnote
 // of "Double Sampling"; update in full precision, "End-to-end Quantization") is two passes over the
 // step's code tile: the dots q1^T x, q2^T x of every row (pass A), then the gradient
-// 1/(2B) sum_k [q1_k r2_k + q2_k r1_k] (pass B), with r = dot - b between them.  Here both passes
-// read the codes straight from global memory into int8 tensor-core fragments (no shared-memory
-// staging): pass A streams the tile from HBM and leaves it in L2, pass B re-reads it from L2.
+// 1/(2B) sum_k [q1_k r2_k + q2_k r1_k] (pass B), with r = dot - b between them.  Both passes feed the
+// int8 tensor cores with code bytes exactly as they lie in memory: pass A streams the tile from HBM
+// and leaves it in L2, pass B re-reads it from L2.  Every warp moves its own bytes through a private
+// ring of shared-memory stages with cp.async (each lane reads back only what it copied itself, so
+// the ring needs no barrier), several stages ahead of the arithmetic.
 //
-//   pass A   a warp takes 16 rows x a run of 64-byte spans; code bytes are the A operand of
-//            mma.sync m16n8k32 (u8 x s8), the four balanced base-128 digits of w = step * x the B
-//            operand's columns; digit sums are exact integers, combined in 64 bits and added to
-//            dots[plane][row] with integer atomics (order-free).
+//   pass A   a CTA takes one column part of the row (a run of 64-byte spans) for 256 rows, a warp 16
+//            of them; the part's digits of w = step * x (four balanced base-128 int8 digits) are
+//            staged once per CTA.  Code bytes are the A operand of mma.sync m16n8k32 (u8 x s8), the
+//            digits the B operand's columns; digit sums are exact integers, combined in 64 bits and
+//            added to dots[plane][row] with integer atomics (order-free).
 //   barrier  one grid barrier per step: every dot is complete.
 //   resid.   every CTA computes all residuals (2B values), their common fixed-point scale and digits
 //            (shared memory), redundantly and identically.
-//   pass B   a CTA owns whole column blocks (CW bytes of the row = CW * 8 / CB features) for all rows
+//   pass B   a CTA owns whole column blocks (64 bytes of the row = 512 / CB features) for all rows
 //            of the step, so its gradient entries never leave it.  The contraction runs over rows:
-//            a lane loads LB bytes of 8 rows, transposes 4 x 4 byte blocks with byte permutes and
+//            a lane copies 8 bytes of 8 rows, transposes 4 x 4 byte blocks with byte permutes and
 //            feeds (features x rows) fragments; the residual digits are the B operand.
-//   update   the owner updates its features of x, turns w = step * x into digits for the next
-//            step and raises a per-block flag; pass A of the next step waits only for the flags of
-//            the blocks it reads (no second grid barrier).
+//   update   the owner updates its features of x (kept in shared memory for the whole launch), turns
+//            w = step * x into digits for the next step and raises a per-block flag; pass A of the
+//            next step waits only for the flags of the blocks it reads (no second grid barrier).
 //
 // The digit scale of w must be known to writers and readers without another exchange: it is a bound,
 // |w_j(t+1)| <= max|w(t)| + lr * max_j(step_j * max|a_j|) * max_k|r_k(t)|, whose pieces every CTA
 // already holds after the step's barrier (owners publish their part of max|w| and of lo^T x with
 // the flags).  The bound costs a few of the 27 fixed-point bits while the model is still near zero.
+#include <stdlib.h>
 #include <string.h>
 
 #include "int_digits.cuh"
@@ -37,6 +41,11 @@ constexpr int kStreamThreads = 512;
 constexpr int kStreamWarps = kStreamThreads / 32;
 constexpr int kStreamMaxBatch = 8192;      // residual digits of a step live in shared memory
 constexpr int kStreamMaxOwn = 4;           // column blocks per CTA
+constexpr int kStreamStages = 4;           // ring stages per warp
+constexpr int kStreamStageBytes = 2048;    // pass A: 4 x 32 lanes x 16 B; pass B: 8 x 32 lanes x 8 B
+constexpr int kStreamRingBytes = kStreamWarps * kStreamStages * kStreamStageBytes;
+constexpr int kStreamBlock = 64;           // bytes of a column block = one span
+constexpr int kStreamMaxPartSpans = 64;    // spans of a pass-A column part
 
 struct StreamArgs {
     const unsigned char* p1;
@@ -51,14 +60,16 @@ struct StreamArgs {
     int64_t batch, first_step, num_steps;
     const int32_t* order;
     float lr;
-    int ca;                  // pass A: column parts per 16-row block
-    int spans;               // 64-byte spans of a row
-    int ncb;                 // pass B: column blocks of the row
+    int ca;                  // pass A: column parts of the row
+    int spans;               // 64-byte spans of a row = pass B's column blocks
+    int part_spans;          // most spans a part holds
     int bpc;                 // column blocks per CTA
     int bpad;                // batch rounded up to 32
-    int64_t vec_bytes;       // bytes of one digit vector (row_bytes rounded up to 128)
+    int union_bytes;         // shared memory shared by pass A's digits and pass B's residual digits + sums
+    int l2_prefetch;         // ask L2 for the next step's tile while pass B runs
+    int64_t vec_bytes;       // bytes of one digit vector (spans * 64)
     signed char* wdig;       // [NG][NS][vec_bytes] digits of w, in the byte order of the codes
-    unsigned* ready;         // [ncb] number of digit versions published for the block
+    unsigned* ready;         // [spans] number of digit versions published for the block
     long long* dots;         // [3][2][bpad] fixed-point dots of the step (three steps in rotation)
     float* wmax_part;        // [2][G] owners' max |w| (by step parity)
     double* base_part;       // [2][G] owners' part of lo^T x
@@ -80,63 +91,73 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 __device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void l2_prefetch_bulk(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 
-// Max over the block; every thread gets it.  `sh` holds 33 floats.  Ends with the block synchronised.
-__device__ __forceinline__ float block_max(float v, float* sh) {
+// Two maxima and a sum over the block in one round; every thread combines the warps' results in the
+// same fixed order, so every thread (and every CTA given the same inputs) gets the same bits.
+// Its two barriers come after the caller's earlier shared-memory writes and before anyone returns.
+__device__ __forceinline__ void block_reduce_mms(float& m1, float& m2, double& s, float* shf, double* shd) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float t = 0.0f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t = fmaxf(t, sh[w]);
-        sh[32] = t;
+    for (int o = 16; o > 0; o >>= 1) {
+        m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+        m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, o));
+        s += __shfl_xor_sync(0xffffffffu, s, o);
     }
+    const int warp = threadIdx.x >> 5;
     __syncthreads();
-    return sh[32];
+    if ((threadIdx.x & 31) == 0) { shf[warp] = m1; shf[kStreamWarps + warp] = m2; shd[warp] = s; }
+    __syncthreads();
+    m1 = 0.0f; m2 = 0.0f; s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kStreamWarps; ++w) { m1 = fmaxf(m1, shf[w]); m2 = fmaxf(m2, shf[kStreamWarps + w]); s += shd[w]; }
 }
 
 __device__ __forceinline__ int fixed_point(float v, float inv) {
-    int W = __float2int_rn(v * inv);
+    const int W = __float2int_rn(v * inv);
     return max(-IntPath<8>::QMAX, min(IntPath<8>::QMAX, W));
 }
 
-template <int LB>
-struct LaneBytes;
-template <>
-struct LaneBytes<16> {
-    using T = uint4;
-    static __device__ __forceinline__ T zero() { return make_uint4(0u, 0u, 0u, 0u); }
-    static __device__ __forceinline__ uint32_t word(const T& v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
-};
-template <>
-struct LaneBytes<8> {
-    using T = uint2;
-    static __device__ __forceinline__ T zero() { return make_uint2(0u, 0u); }
-    static __device__ __forceinline__ uint32_t word(const T& v, int i) { return i == 0 ? v.x : v.y; }
-};
-
-template <int CB, int LB>
+template <int CB>
 __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const StreamArgs a) {
     constexpr int NG = IntPath<CB>::NG, NS = IntPath<CB>::NS, FPW = 32 / CB;
-    constexpr int CW = 8 * LB, WPL = LB / 4;
+    constexpr int CW = kStreamBlock, S = kStreamStages;
     constexpr int QMAX = IntPath<CB>::QMAX;
-    using Vec = typename LaneBytes<LB>::T;
     static_assert(NS == 4, "four digits");
-    extern __shared__ __align__(16) unsigned char smem[];
-    signed char* rdig = reinterpret_cast<signed char*>(smem);                    // [2][NS][bpad]
-    int* gacc = reinterpret_cast<int*>(smem + (size_t)2 * NS * a.bpad);          // [bpc][NG][CW][NS]
-    __shared__ double red[40];
-    __shared__ float fsh[40];
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* ring = smem;                                                  // [warps][S][stage]
+    unsigned char* uni = smem + kStreamRingBytes;
+    signed char* wds = reinterpret_cast<signed char*>(uni);                      // pass A: [NG * NS][part_spans * 64]
+    signed char* rdig = reinterpret_cast<signed char*>(uni);                     // pass B: [2][NS][bpad + 16]
+    int* gacc = reinterpret_cast<int*>(uni + (size_t)2 * NS * (a.bpad + 16));    // pass B: [bpc][NG][CW][NS]
+    float* own = reinterpret_cast<float*>(uni + a.union_bytes);                  // [3][bpc * CW * NG]: lo, step, x of the own features
+    double2* rres = reinterpret_cast<double2*>(ring);                            // dots minus labels, between the passes
+    __shared__ double shd[kStreamWarps];
+    __shared__ float shf[2 * kStreamWarps];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gl = lane >> 2, tl = lane & 3;
     const int cta = blockIdx.x, G = gridDim.x;
     const int n = a.n;
     const int64_t rb = a.row_bytes, vb = a.vec_bytes;
-    const int cb0 = min(a.ncb, cta * a.bpc), cb1 = min(a.ncb, cb0 + a.bpc);
-    const int own_bytes = (cb1 - cb0) * CW;
+    const int cb0 = min(a.spans, cta * a.bpc), cb1 = min(a.spans, cb0 + a.bpc);
+    const int own_n = (cb1 - cb0) * CW * NG, own_cap = a.bpc * CW * NG;
+    float* lo_o = own;
+    float* st_o = own + own_cap;
+    float* x_o = own + 2 * own_cap;
     const float smax = (float)((1 << a.bits) - 1);
+    const uint32_t ring_w = smem_u32(ring) + (uint32_t)warp * S * kStreamStageBytes;
+    const int pstride = a.part_spans * 64 + 16;            // bytes between the digit vectors in wds (16 more: no bank conflicts)
+    const int rstride = a.bpad + 16;                       // bytes between the residual digit vectors
 
     // ---- set-up: every CTA scans the model once (identical arithmetic everywhere)
     float cmax = 0.0f, wm = 0.0f;
@@ -147,23 +168,23 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
         wm = fmaxf(wm, fabsf(s * xv));
         base += (double)l * (double)xv;
     }
-    cmax = block_max(cmax, fsh);
-    wm = block_max(wm, fsh);
-    base = block_sum(base, red);
+    block_reduce_mms(cmax, wm, base, shf, shd);
     float bound = wm;                      // digit scale of the w that the coming step reads
 
-    // digits of w for the first step, from the caller's model
+    // own features into shared memory; digits of w for the first step, from the caller's model
     {
         const float inv = bound > 0.0f ? (float)QMAX / bound : 0.0f;
-        for (int idx = tid; idx < own_bytes * NG; idx += kStreamThreads) {
+        for (int idx = tid; idx < own_n; idx += kStreamThreads) {
             const int bl = idx / NG, grp = idx - bl * NG;
             const int64_t byte = (int64_t)cb0 * CW + bl;
-            if (byte >= vb) continue;
             const int64_t j = (byte >> 2) * FPW + (byte & 3) * NG + grp;
+            const bool real = j < n;
+            const float l = real ? a.lo[j] : 0.0f, s = real ? a.step[j] : 0.0f, xv = real ? a.x[j] : 0.0f;
+            lo_o[idx] = l; st_o[idx] = s; x_o[idx] = xv;
             int d[NS];
-            balanced_digits<NS>(j < n ? fixed_point(a.step[j] * a.x[j], inv) : 0, d);
+            balanced_digits<NS>(real ? fixed_point(s * xv, inv) : 0, d);
 #pragma unroll
-            for (int s = 0; s < NS; ++s) a.wdig[((int64_t)grp * NS + s) * vb + byte] = (signed char)d[s];
+            for (int k = 0; k < NS; ++k) a.wdig[((int64_t)grp * NS + k) * vb + byte] = (signed char)d[k];
         }
         __syncthreads();
         if (tid == 0) {
@@ -185,16 +206,36 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
 
         // ------------------------------------------------------------------ pass A: dots
         {
-            const int nrb = (bt + 15) >> 4;
-            const int ntasks = nrb * a.ca;
-            for (int q = cta * kStreamWarps + warp; q < ntasks; q += G * kStreamWarps) {
-                const int rblk = q / a.ca, part = q - rblk * a.ca;
+            const int nrb = (bt + 15) >> 4, nrg = (nrb + kStreamWarps - 1) / kStreamWarps;
+            const int units = a.ca * nrg;
+#pragma unroll 1
+            for (int u = cta; u < units; u += G) {
+                const int rg = u / a.ca, part = u - rg * a.ca;
                 const int s0 = (int)((int64_t)part * a.spans / a.ca), s1 = (int)((int64_t)(part + 1) * a.spans / a.ca);
-                // digits of this column part present?
+                const int rblk = rg * kStreamWarps + warp;
+                const bool active = rblk < nrb;
+                // A lane copies 16 bytes of rows g and g+8 of both planes per span.  Copies of rows past the
+                // batch or bytes past the row are skipped: what the stage then holds meets zero digits
+                // (pad features) or is never stored (pad rows).
+                const bool ok_a = active && rblk * 16 + gl < bt, ok_h = active && rblk * 16 + gl + 8 < bt;
+                const uint32_t off_a = (uint32_t)(rblk * 16 + gl) * (uint32_t)rb + 16 * tl, off_h = off_a + 8 * (uint32_t)rb;
+                const int sp_end = min(s1, (int)((rb - 16 * tl + 63) / 64));      // spans whose 16 bytes of this lane lie in the row
+                const uint32_t stage0 = ring_w + lane * 16;
+                auto issue = [&](int sp) {
+                    if (sp < sp_end) {
+                        const uint32_t dst = stage0 + (uint32_t)((sp - s0) & (S - 1)) * kStreamStageBytes;
+                        const uint32_t o = (uint32_t)sp * 64;
+                        if (ok_a) { cp_async16(dst, t1 + (off_a + o)); cp_async16(dst + 1024, t2 + (off_a + o)); }
+                        if (ok_h) { cp_async16(dst + 512, t1 + (off_h + o)); cp_async16(dst + 1536, t2 + (off_h + o)); }
+                    }
+                    cp_async_commit();
+                };
+                // the codes do not depend on the model: start copying before looking at the flags
+#pragma unroll
+                for (int k = 0; k < S - 1; ++k) issue(s0 + k);
                 {
-                    const int f0 = (s0 * 64) / CW, f1 = min(a.ncb, (s1 * 64 + CW - 1) / CW);
                     const unsigned want = (unsigned)(t_rel + 1);
-                    for (int f = f0 + lane; f < f1; f += 32) {
+                    for (int f = s0 + tid; f < s1; f += kStreamThreads) {
                         long long spin = 0;
                         while (ld_acquire_u32(a.ready + f) < want) {
                             if (++spin > kBarrierSpinLimit) { set_status(a.status, ZIPML_ERR_TIMEOUT, 20); break; }
@@ -204,49 +245,65 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                             }
                         }
                     }
-                    __syncwarp();
-                    __threadfence();
-                }
-                const int ra = min(rblk * 16 + gl, bt - 1), rh = min(rblk * 16 + gl + 8, bt - 1);
-                const unsigned char* a1 = t1 + ra * rb + 16 * tl;
-                const unsigned char* h1 = t1 + rh * rb + 16 * tl;
-                const unsigned char* a2 = t2 + ra * rb + 16 * tl;
-                const unsigned char* h2 = t2 + rh * rb + 16 * tl;
-                int c1[4] = {0, 0, 0, 0}, c2[4] = {0, 0, 0, 0};
-#pragma unroll 2
-                for (int sp = s0; sp < s1; ++sp) {
-                    const int64_t off = (int64_t)sp * 64;
-                    uint4 ua = make_uint4(0u, 0u, 0u, 0u), uh = ua, va = ua, vh = ua;
-                    const bool in = off + 16 * tl < rb;
-                    if (in) {
-                        ua = __ldcg(reinterpret_cast<const uint4*>(a1 + off));
-                        uh = __ldcg(reinterpret_cast<const uint4*>(h1 + off));
-                        va = __ldcg(reinterpret_cast<const uint4*>(a2 + off));
-                        vh = __ldcg(reinterpret_cast<const uint4*>(h2 + off));
+                    __syncthreads();
+                    const int pb16 = (s1 - s0) * 4;                        // 16-byte pieces of one digit vector
+                    for (int idx = tid; idx < NG * NS * pb16; idx += kStreamThreads) {
+                        const int v = idx / pb16, q = idx - v * pb16;
+                        *reinterpret_cast<uint4*>(wds + (size_t)v * pstride + q * 16) =
+                            __ldcg(reinterpret_cast<const uint4*>(a.wdig + (int64_t)v * vb + (int64_t)s0 * 64 + q * 16));
                     }
+                    __syncthreads();
+                }
+                // group g's codes stay where they are in the byte (one mask): its sums come out 2^(g CB) times too large
+                int c1[NG][4], c2[NG][4];
 #pragma unroll
-                    for (int g = 0; g < NG; ++g) {
-                        uint4 bd = make_uint4(0u, 0u, 0u, 0u);
-                        if (gl < NS && in) bd = __ldcg(reinterpret_cast<const uint4*>(a.wdig + ((int64_t)g * NS + gl) * vb + off + 16 * tl));
-                        mma_u8s8(c1, group_bytes<CB>(ua.x, g), group_bytes<CB>(uh.x, g), group_bytes<CB>(ua.y, g), group_bytes<CB>(uh.y, g), bd.x, bd.y);
-                        mma_u8s8(c1, group_bytes<CB>(ua.z, g), group_bytes<CB>(uh.z, g), group_bytes<CB>(ua.w, g), group_bytes<CB>(uh.w, g), bd.z, bd.w);
-                        mma_u8s8(c2, group_bytes<CB>(va.x, g), group_bytes<CB>(vh.x, g), group_bytes<CB>(va.y, g), group_bytes<CB>(vh.y, g), bd.x, bd.y);
-                        mma_u8s8(c2, group_bytes<CB>(va.z, g), group_bytes<CB>(vh.z, g), group_bytes<CB>(va.w, g), group_bytes<CB>(vh.w, g), bd.z, bd.w);
+                for (int g = 0; g < NG; ++g)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) { c1[g][e] = 0; c2[g][e] = 0; }
+                if (active) {
+                    const unsigned char* stage_r = ring + (size_t)warp * S * kStreamStageBytes + lane * 16;
+                    const signed char* dig_r = wds + (size_t)gl * pstride + 16 * tl;       // lanes with gl < NS read digit gl
+#pragma unroll 1
+                    for (int sp = s0; sp < s1; ++sp) {
+                        issue(sp + S - 1);
+                        cp_async_wait<S - 1>();
+                        const unsigned char* st = stage_r + (size_t)((sp - s0) & (S - 1)) * kStreamStageBytes;
+                        const uint4 ua = *reinterpret_cast<const uint4*>(st);
+                        const uint4 uh = *reinterpret_cast<const uint4*>(st + 512);
+                        const uint4 va = *reinterpret_cast<const uint4*>(st + 1024);
+                        const uint4 vh = *reinterpret_cast<const uint4*>(st + 1536);
+#pragma unroll
+                        for (int g = 0; g < NG; ++g) {
+                            constexpr uint32_t kLow = CB == 8 ? 0xFFFFFFFFu : CB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
+                            const uint32_t mk = kLow << (g * CB);
+                            uint4 bd = make_uint4(0u, 0u, 0u, 0u);
+                            if (gl < NS) bd = *reinterpret_cast<const uint4*>(dig_r + (size_t)g * NS * pstride + (sp - s0) * 64);
+                            mma_u8s8(c1[g], ua.x & mk, uh.x & mk, ua.y & mk, uh.y & mk, bd.x, bd.y);
+                            mma_u8s8(c1[g], ua.z & mk, uh.z & mk, ua.w & mk, uh.w & mk, bd.z, bd.w);
+                            mma_u8s8(c2[g], va.x & mk, vh.x & mk, va.y & mk, vh.y & mk, bd.x, bd.y);
+                            mma_u8s8(c2[g], va.z & mk, vh.z & mk, va.w & mk, vh.w & mk, bd.z, bd.w);
+                        }
                     }
                 }
+                cp_async_wait<0>();
                 // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3])
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const long long q1 = (long long)c1[2 * e] + 128ll * (long long)c1[2 * e + 1];
-                    const long long q2 = (long long)c2[2 * e] + 128ll * (long long)c2[2 * e + 1];
+                    long long q1 = 0, q2 = 0;
+#pragma unroll
+                    for (int g = 0; g < NG; ++g) {         // exact: the sums are multiples of 2^(g CB)
+                        q1 += (long long)(c1[g][2 * e] >> (g * CB)) + 128ll * (long long)(c1[g][2 * e + 1] >> (g * CB));
+                        q2 += (long long)(c2[g][2 * e] >> (g * CB)) + 128ll * (long long)(c2[g][2 * e + 1] >> (g * CB));
+                    }
                     const long long v1 = q1 + 16384ll * __shfl_down_sync(0xffffffffu, q1, 1);
                     const long long v2 = q2 + 16384ll * __shfl_down_sync(0xffffffffu, q2, 1);
                     const int k = rblk * 16 + gl + 8 * e;
-                    if (tl == 0 && k < bt) {
+                    if (active && tl == 0 && k < bt) {
                         atomicAdd(reinterpret_cast<unsigned long long*>(dots + k), (unsigned long long)v1);
                         atomicAdd(reinterpret_cast<unsigned long long*>(dots + a.bpad + k), (unsigned long long)v2);
                     }
                 }
+                __syncthreads();           // the next unit overwrites the staged digits
             }
         }
         stream_mark(a, t_rel, 1);
@@ -259,124 +316,176 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             long long* z = a.dots + (size_t)((t_rel + 2) % 3) * 2 * a.bpad;
             for (int i = cta * kStreamThreads + tid; i < 2 * a.bpad; i += G * kStreamThreads) z[i] = 0;
         }
-        if (t_rel > 0) {                   // max |w| and lo^T x of the model this step saw
-            const size_t par = (size_t)(t_rel & 1) * G;
-            float pm = 0.0f;
-            double pb = 0.0;
-            for (int i = tid; i < G; i += kStreamThreads) { pm = fmaxf(pm, __ldcg(a.wmax_part + par + i)); pb += __ldcg(a.base_part + par + i); }
-            wm = block_max(pm, fsh);
-            base = block_sum(pb, red);
-        }
         const double delta_w = (double)bound / (double)QMAX;
-        float rmax = 0.0f;
-        for (int k = tid; k < bt; k += kStreamThreads) {
-            const double bk = (double)a.b[row0 + k];
-            const float r1 = (float)((double)__ldcg(dots + k) * delta_w + base - bk);
-            const float r2 = (float)((double)__ldcg(dots + a.bpad + k) * delta_w + base - bk);
-            rmax = fmaxf(rmax, fmaxf(fabsf(r1), fabsf(r2)));
+        float rmax = 0.0f, pm = 0.0f;
+        double pb = 0.0;
+        if (t_rel > 0) {                   // the owners' parts of max |w| and lo^T x of the model this step saw
+            const size_t par = (size_t)(t_rel & 1) * G;
+            for (int i = tid; i < G; i += kStreamThreads) { pm = fmaxf(pm, __ldcg(a.wmax_part + par + i)); pb += __ldcg(a.base_part + par + i); }
         }
-        rmax = block_max(rmax, fsh);
+        for (int k = tid; k < bt; k += kStreamThreads) {
+            const long long v1 = __ldcg(dots + k), v2 = __ldcg(dots + a.bpad + k);
+            const double bk = (double)a.b[row0 + k];
+            rres[k] = make_double2((double)v1 * delta_w - bk, (double)v2 * delta_w - bk);
+        }
+        block_reduce_mms(rmax, pm, pb, shf, shd);          // rmax is not known yet: this round carries pm and pb
+        if (t_rel > 0) { wm = pm; base = pb; }
+        // r = delta_w V + lo^T x - b in double, rounded to fp32 once; the same on every CTA
+        for (int k = tid; k < bt; k += kStreamThreads) {
+            const double2 d = rres[k];
+            rmax = fmaxf(rmax, fmaxf(fabsf((float)(d.x + base)), fabsf((float)(d.y + base))));
+        }
+        {
+            float unused = 0.0f;
+            double none = 0.0;
+            block_reduce_mms(rmax, unused, none, shf, shd);
+        }
         const float inv_r = rmax > 0.0f ? (float)QMAX / rmax : 0.0f;
         const double delta_r = (double)rmax / (double)QMAX;
         double rsum = 0.0;                 // sum of all fixed-point residuals (exact in double)
         for (int k = tid; k < a.bpad; k += kStreamThreads) {
             int R1 = 0, R2 = 0;
             if (k < bt) {
-                const double bk = (double)a.b[row0 + k];
-                R1 = fixed_point((float)((double)__ldcg(dots + k) * delta_w + base - bk), inv_r);
-                R2 = fixed_point((float)((double)__ldcg(dots + a.bpad + k) * delta_w + base - bk), inv_r);
+                const double2 d = rres[k];
+                R1 = fixed_point((float)(d.x + base), inv_r);
+                R2 = fixed_point((float)(d.y + base), inv_r);
             }
             rsum += (double)R1 + (double)R2;
+            // within a group of 16 rows, row r sits at 4 (r % 4) + r / 4: a 32-bit word holds rows t, t+4, t+8, t+12
+            const int kp = (k & ~15) | ((k & 3) << 2) | ((k >> 2) & 3);
             int d1[NS], d2[NS];
             balanced_digits<NS>(R1, d1);
             balanced_digits<NS>(R2, d2);
 #pragma unroll
-            for (int s = 0; s < NS; ++s) {
-                rdig[(size_t)s * a.bpad + k] = (signed char)d2[s];                 // plane 1 meets r2
-                rdig[(size_t)(NS + s) * a.bpad + k] = (signed char)d1[s];          // plane 2 meets r1
+            for (int q = 0; q < NS; ++q) {
+                rdig[(size_t)q * rstride + kp] = (signed char)d2[q];               // plane 1 meets r2
+                rdig[(size_t)(NS + q) * rstride + kp] = (signed char)d1[q];        // plane 2 meets r1
             }
         }
         for (int i = tid; i < (cb1 - cb0) * NG * CW * NS; i += kStreamThreads) gacc[i] = 0;
-        rsum = block_sum(rsum, red);       // its barriers publish rdig and the cleared gacc
+        {
+            float u1 = 0.0f, u2 = 0.0f;
+            block_reduce_mms(u1, u2, rsum, shf, shd);      // its barriers publish rdig and the cleared sums
+        }
         // scale of the next model's digits: a bound that writers and readers both know now
         const float bound_next = (wm + fabsf(a.lr) * cmax * rmax) * 1.0001f;
         stream_mark(a, t_rel, 3);
 
+        // the next step's tile can travel to L2 while this step's second pass reads from L2
+        if (a.l2_prefetch && !last && warp == kStreamWarps - 1 && lane < 2) {
+            const int64_t itn = it + 1;
+            const int64_t rown = (a.order ? (int64_t)a.order[itn] : itn) * a.batch;
+            const int64_t bytes = min(a.batch, a.m - rown) * rb;          // a multiple of 16
+            const int64_t per = ((bytes / 16 + G - 1) / G) * 16;
+            const int64_t lo_b = min(bytes, per * cta), hi_b = min(bytes, lo_b + per);
+            const unsigned char* srcn = (lane == 0 ? a.p1 : a.p2) + rown * rb;
+            for (int64_t o = lo_b; o < hi_b; o += 32768) l2_prefetch_bulk(srcn + o, (uint32_t)min((int64_t)32768, hi_b - o));
+        }
+
         // ------------------------------------------------------------------ pass B: gradient of the own blocks
         {
             const int nrb = (bt + 31) >> 5;
-            for (int c = cb0; c < cb1; ++c) {
-                const int64_t coff = (int64_t)c * CW + gl * LB;
-                const bool in = coff < rb;
-                int acc[NG][WPL][2][4];
+            const int mine = nrb > warp ? (nrb - 1 - warp) / kStreamWarps + 1 : 0;     // 32-row blocks of this warp
+            const int per_c = 2 * mine, total = (cb1 - cb0) * per_c;
+            // Iteration i: column block i / per_c, then (row block, plane); newest rows first (likeliest in L2).
+            // A stage holds 32 rows x 64 bytes, row-major; a lane copies 16 bytes of rows l/4, l/4+8, l/4+16,
+            // l/4+24.  Copies of rows past the batch or of bytes past the row are skipped: the former meet
+            // zero residual digits, the latter end in sums of pad features that nobody reads.  Lane 4g+t
+            // then takes the 8 bytes of column piece g from rows t, t+4, t+8, t+12 (and 16 more): for one
+            // load the four t's read four consecutive rows, 256 contiguous bytes, no bank conflict; the
+            // residual digits are stored in the matching row order.
+            const uint32_t rb32 = (uint32_t)rb;
+            const uint32_t stage0 = ring_w + lane * 16;
+            int i_ci = 0, i_rem = 0;                       // issue side: column block and position within it
+            auto issue = [&]() {
+                if (i_ci < cb1 - cb0) {
+                    const int r0 = (nrb - 1 - warp - kStreamWarps * (i_rem >> 1)) * 32 + gl;
+                    const uint32_t coff = (uint32_t)(cb0 + i_ci) * CW + tl * 16;
+                    if (coff < rb32) {
+                        const unsigned char* tp = ((i_rem & 1) ? t2 : t1) + coff;
+                        const uint32_t dst = stage0 + (uint32_t)((i_ci * per_c + i_rem) & (S - 1)) * kStreamStageBytes;
+                        const uint32_t o = (uint32_t)r0 * rb32;
 #pragma unroll
-                for (int g = 0; g < NG; ++g)
+                        for (int k = 0; k < 4; ++k)
+                            if (r0 + 8 * k < bt) cp_async16(dst + k * 512, tp + (o + 8 * k * rb32));
+                    }
+                    if (++i_rem == per_c) { i_rem = 0; ++i_ci; }
+                }
+                cp_async_commit();
+            };
+            int acc[NG][2][2][4];
 #pragma unroll
-                    for (int w = 0; w < WPL; ++w)
+            for (int g = 0; g < NG; ++g)
+#pragma unroll
+                for (int w = 0; w < 2; ++w)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[g][w][u][e] = 0;
+            if (total > 0) {
+#pragma unroll
+                for (int k = 0; k < S - 1; ++k) issue();
+            }
+            const unsigned char* stage_r = ring + (size_t)warp * S * kStreamStageBytes + tl * 64 + gl * 8;
+            const signed char* rd_lane = rdig + (size_t)(gl & (NS - 1)) * rstride + 4 * tl;
+            int ci = 0, rem = 0;
+#pragma unroll 1
+            for (int i = 0; i < total; ++i) {
+                cp_async_wait<S - 2>();    // this lane's copies of stage i have landed ...
+                __syncwarp();              // ... and everyone's; and everyone is done reading stage i - 1,
+                issue();                   // which this refills
+                const int r0 = (nrb - 1 - warp - kStreamWarps * (rem >> 1)) * 32;
+                const unsigned char* st = stage_r + (size_t)(i & (S - 1)) * kStreamStageBytes;
+                uint2 lo4[4], hi4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    lo4[k] = *reinterpret_cast<const uint2*>(st + k * 256);            // row t + 4k
+                    hi4[k] = *reinterpret_cast<const uint2*>(st + 1024 + k * 256);     // row 16 + t + 4k
+                }
+                uint32_t b0 = 0u, b1 = 0u;
+                if (gl < NS) {
+                    const signed char* rd = rd_lane + (size_t)((rem & 1) * NS) * rstride + r0;
+                    b0 = *reinterpret_cast<const uint32_t*>(rd);
+                    b1 = *reinterpret_cast<const uint32_t*>(rd + 16);
+                }
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    uint32_t ta[4], th[4];
+                    if (w == 0) { transpose4x4(lo4[0].x, lo4[1].x, lo4[2].x, lo4[3].x, ta); transpose4x4(hi4[0].x, hi4[1].x, hi4[2].x, hi4[3].x, th); }
+                    else { transpose4x4(lo4[0].y, lo4[1].y, lo4[2].y, lo4[3].y, ta); transpose4x4(hi4[0].y, hi4[1].y, hi4[2].y, hi4[3].y, th); }
+#pragma unroll
+                    for (int g = 0; g < NG; ++g) {
+                        constexpr uint32_t kLow = CB == 8 ? 0xFFFFFFFFu : CB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
+                        const uint32_t mk = kLow << (g * CB);      // codes stay in place: sums 2^(g CB) times too large
 #pragma unroll
                         for (int u = 0; u < 2; ++u)
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[g][w][u][e] = 0;
-                bool any = false;
-                // newest rows first: they are the likeliest to be still in L2
-#pragma unroll 1
-                for (int rblk = nrb - 1 - warp; rblk >= 0; rblk -= kStreamWarps) {
-                    any = true;
-                    const int r0 = rblk * 32;
-#pragma unroll
-                    for (int pl = 0; pl < 2; ++pl) {
-                        const unsigned char* tp = pl == 0 ? t1 : t2;
-                        Vec lo4[4], hi4[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            lo4[i] = LaneBytes<LB>::zero();
-                            hi4[i] = LaneBytes<LB>::zero();
-                            if (in) {
-                                const int ka = min(r0 + 4 * tl + i, bt - 1), kh = min(r0 + 16 + 4 * tl + i, bt - 1);
-                                lo4[i] = __ldcs(reinterpret_cast<const Vec*>(tp + ka * rb + coff));
-                                hi4[i] = __ldcs(reinterpret_cast<const Vec*>(tp + kh * rb + coff));
-                            }
-                        }
-                        uint32_t b0 = 0u, b1 = 0u;
-                        if (gl < NS) {
-                            const signed char* rd = rdig + (size_t)(pl * NS + gl) * a.bpad + r0 + 4 * tl;
-                            b0 = *reinterpret_cast<const uint32_t*>(rd);
-                            b1 = *reinterpret_cast<const uint32_t*>(rd + 16);
-                        }
-#pragma unroll
-                        for (int w = 0; w < WPL; ++w) {
-                            uint32_t ta[4], th[4];
-                            transpose4x4(LaneBytes<LB>::word(lo4[0], w), LaneBytes<LB>::word(lo4[1], w), LaneBytes<LB>::word(lo4[2], w),
-                                         LaneBytes<LB>::word(lo4[3], w), ta);
-                            transpose4x4(LaneBytes<LB>::word(hi4[0], w), LaneBytes<LB>::word(hi4[1], w), LaneBytes<LB>::word(hi4[2], w),
-                                         LaneBytes<LB>::word(hi4[3], w), th);
-#pragma unroll
-                            for (int g = 0; g < NG; ++g)
-#pragma unroll
-                                for (int u = 0; u < 2; ++u)
-                                    mma_u8s8(acc[g][w][u], group_bytes<CB>(ta[2 * u], g), group_bytes<CB>(ta[2 * u + 1], g),
-                                             group_bytes<CB>(th[2 * u], g), group_bytes<CB>(th[2 * u + 1], g), b0, b1);
-                        }
+                            mma_u8s8(acc[g][w][u], ta[2 * u] & mk, ta[2 * u + 1] & mk, th[2 * u] & mk, th[2 * u + 1] & mk, b0, b1);
                     }
                 }
-                // lane t < 2: acc[g][w][u][0..1] = digits 2t, 2t+1 of byte 4w+2u of the lane's bytes, [2..3] of byte 4w+2u+1
-                if (any && tl < 2) {
-                    int* dst = gacc + (size_t)(c - cb0) * NG * CW * NS;
+                if (++rem == per_c) {
+                    // lane t < 2: acc[g][w][u][0..1] = digits 2t, 2t+1 of byte 4w+2u of the lane's bytes, [2..3] of byte 4w+2u+1
+                    int* dst = gacc + (size_t)ci * NG * CW * NS;
 #pragma unroll
                     for (int g = 0; g < NG; ++g)
 #pragma unroll
-                        for (int w = 0; w < WPL; ++w)
+                        for (int w = 0; w < 2; ++w)
 #pragma unroll
                             for (int u = 0; u < 2; ++u) {
-                                const int byte = gl * LB + 4 * w + 2 * u;
-                                int* p = dst + ((size_t)g * CW + byte) * NS + 2 * tl;
-                                atomicAdd(p, acc[g][w][u][0]);
-                                atomicAdd(p + 1, acc[g][w][u][1]);
-                                atomicAdd(p + NS, acc[g][w][u][2]);
-                                atomicAdd(p + NS + 1, acc[g][w][u][3]);
+                                if (tl < 2) {
+                                    int* p = dst + ((size_t)g * CW + gl * 8 + 4 * w + 2 * u) * NS + 2 * tl;
+                                    atomicAdd(p, acc[g][w][u][0] >> (g * CB));
+                                    atomicAdd(p + 1, acc[g][w][u][1] >> (g * CB));
+                                    atomicAdd(p + NS, acc[g][w][u][2] >> (g * CB));
+                                    atomicAdd(p + NS + 1, acc[g][w][u][3] >> (g * CB));
+                                }
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) acc[g][w][u][e] = 0;
                             }
+                    rem = 0;
+                    ++ci;
                 }
             }
+            cp_async_wait<0>();
         }
         __syncthreads();
         stream_mark(a, t_rel, 4);
@@ -386,43 +495,42 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             const double scale = 1.0 / (2.0 * (double)bt);
             const double lo_term = delta_r * rsum;
             const float inv = bound_next > 0.0f ? (float)QMAX / bound_next : 0.0f;
-            float pm = 0.0f;
-            double pb = 0.0;
-            for (int idx = tid; idx < own_bytes * NG; idx += kStreamThreads) {
+            float pmax = 0.0f, unused = 0.0f;
+            double pbase = 0.0;
+            for (int idx = tid; idx < own_n; idx += kStreamThreads) {
                 const int bl = idx / NG, grp = idx - bl * NG;
                 const int64_t byte = (int64_t)cb0 * CW + bl;
-                if (byte >= vb) continue;
                 const int64_t j = (byte >> 2) * FPW + (byte & 3) * NG + grp;
                 int W = 0;
                 if (j < n) {
                     const int cl = bl / CW, bb = bl - cl * CW;
                     const int* src = gacc + (((size_t)cl * NG + grp) * CW + bb) * NS;
                     const int sv[NS] = {src[0], src[1], src[2], src[3]};
-                    const long long S = combine_digits<NS>(sv);
-                    const float l = a.lo[j], s = a.step[j];
-                    const float g = (float)(((double)l * lo_term + (double)s * (delta_r * (double)S)) * scale);
+                    const long long Sj = combine_digits<NS>(sv);
+                    const float l = lo_o[idx], st = st_o[idx];
+                    const float g = (float)(((double)l * lo_term + (double)st * (delta_r * (double)Sj)) * scale);
                     if (last && a.grad_out) { a.grad_out[j] = g; a.grad_out[n + j] = g; }
-                    const float xn = fmaf(-a.lr, g, a.x[j]);
+                    const float xn = fmaf(-a.lr, g, x_o[idx]);
+                    x_o[idx] = xn;
                     a.x[j] = xn;
-                    const float w = s * xn;
-                    pm = fmaxf(pm, fabsf(w));
-                    pb += (double)l * (double)xn;
+                    const float w = st * xn;
+                    pmax = fmaxf(pmax, fabsf(w));
+                    pbase += (double)l * (double)xn;
                     W = fixed_point(w, inv);
                 }
                 if (!last) {
                     int d[NS];
                     balanced_digits<NS>(W, d);
 #pragma unroll
-                    for (int s = 0; s < NS; ++s) a.wdig[((int64_t)grp * NS + s) * vb + byte] = (signed char)d[s];
+                    for (int k = 0; k < NS; ++k) a.wdig[((int64_t)grp * NS + k) * vb + byte] = (signed char)d[k];
                 }
             }
             if (last) break;
-            pm = block_max(pm, fsh);
-            pb = block_sum(pb, red);       // ends with a barrier: every digit store of the CTA is issued
+            block_reduce_mms(pmax, unused, pbase, shf, shd);   // its barriers: every digit store of the CTA is issued
             if (tid == 0) {
                 const size_t par = (size_t)((t_rel + 1) & 1) * G;
-                a.wmax_part[par + cta] = pm;
-                a.base_part[par + cta] = pb;
+                a.wmax_part[par + cta] = pmax;
+                a.base_part[par + cta] = pbase;
                 __threadfence();
                 for (int c = cb0; c < cb1; ++c) st_release_u32(a.ready + c, (unsigned)(t_rel + 2));
             }
@@ -436,9 +544,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
 // Host side
 // ---------------------------------------------------------------------------------------------
 static const void* stream_kernel_ptr(int cb) {
-    if (cb == 2) return reinterpret_cast<const void*>(&sgd_stream_kernel<2, 8>);
-    if (cb == 4) return reinterpret_cast<const void*>(&sgd_stream_kernel<4, 8>);
-    return reinterpret_cast<const void*>(&sgd_stream_kernel<8, 16>);
+    if (cb == 2) return reinterpret_cast<const void*>(&sgd_stream_kernel<2>);
+    if (cb == 4) return reinterpret_cast<const void*>(&sgd_stream_kernel<4>);
+    return reinterpret_cast<const void*>(&sgd_stream_kernel<8>);
 }
 
 int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
@@ -447,34 +555,38 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     if (d->level_mode != ZIPML_LEVELS_UNIFORM || p->model_bits != 0 || p->grad_bits != 0) return ZIPML_ERR_WORKSPACE;
     if (d->n > (1 << 30) / 8) return ZIPML_ERR_WORKSPACE;
     const int cb = container_bits(d->bits);
-    const int lb = cb == 8 ? 16 : 8, cw = 8 * lb, ng = 8 / cb;
+    const int ng = 8 / cb, cw = kStreamBlock;
     const int64_t T = (d->m + p->batch - 1) / p->batch;
     const int64_t B = p->batch < d->m ? p->batch : d->m;
     if (B > kStreamMaxBatch) return ZIPML_ERR_WORKSPACE;
     const int bpad = (int)((B + 31) / 32 * 32);
     const int64_t rb = d->row_bytes;
-    const int64_t ncb64 = (rb + cw - 1) / cw;
+    const int64_t spans = (rb + 63) / 64;
     int G = ctx->sm_count;
     if (p->grid_row_parts > 0 && p->grid_row_parts < G) G = p->grid_row_parts;      // tuning: fewer CTAs
-    int64_t bpc = (ncb64 + G - 1) / G;
+    int64_t bpc = (spans + G - 1) / G;
     if (bpc > kStreamMaxOwn) {             // the hint does not fit: plan for the whole device
         G = ctx->sm_count;
-        bpc = (ncb64 + G - 1) / G;
+        bpc = (spans + G - 1) / G;
     }
     if (bpc > kStreamMaxOwn) return ZIPML_ERR_WORKSPACE;
-    G = (int)((ncb64 + bpc - 1) / bpc);
+    G = (int)((spans + bpc - 1) / bpc);
     // worth it only where a step is wide enough to occupy the device and long enough to hide the barrier
     if (only_if_profitable && (G < ctx->sm_count / 2 || B < 256)) return ZIPML_ERR_WORKSPACE;
-    const int spans = (int)((rb + 63) / 64);
-    const int64_t nrb16 = (B + 15) / 16;
-    int64_t ca = ((int64_t)G * kStreamWarps) / nrb16;
+    // pass A: 256-row groups x column parts, about one unit per CTA
+    const int64_t nrg = ((B + 15) / 16 + kStreamWarps - 1) / kStreamWarps;
+    int64_t ca = G / nrg;
+    if (ca < (spans + kStreamMaxPartSpans - 1) / kStreamMaxPartSpans) ca = (spans + kStreamMaxPartSpans - 1) / kStreamMaxPartSpans;
     if (ca < 1) ca = 1;
     if (ca > spans) ca = spans;
-    // a task's digit sums must stay within 32 bits: at most 255 * 64 * codes per group
-    while ((int64_t)(spans + ca - 1) / ca * 64 > 65536) ++ca;
-    const int64_t vec_bytes = (rb + 127) / 128 * 128;
+    const int part_spans = (int)((spans + ca - 1) / ca);
+    const int64_t vec_bytes = spans * 64;
 
-    const size_t smem = (size_t)2 * 4 * bpad + sizeof(int) * (size_t)bpc * ng * cw * 4;
+    const size_t pass_a = (size_t)ng * 4 * (part_spans * 64 + 16);
+    const size_t pass_b = (size_t)2 * 4 * (bpad + 16) + sizeof(int) * (size_t)bpc * ng * cw * 4;
+    const size_t uni = ((pass_a > pass_b ? pass_a : pass_b) + 127) / 128 * 128;
+    const size_t smem = (size_t)kStreamRingBytes + uni + sizeof(float) * 3 * (size_t)bpc * cw * ng;
+    if (smem > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
     const void* kernel = stream_kernel_ptr(cb);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_status(e);
@@ -487,7 +599,7 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     auto piece = [&](size_t bytes) { const size_t o = off; off += carve_size(bytes); return o; };
     // zeroed before a launch: barrier counter, flags, dots
     const size_t o_bar = piece(sizeof(unsigned) * 64);
-    const size_t o_ready = piece(sizeof(unsigned) * (size_t)ncb64);
+    const size_t o_ready = piece(sizeof(unsigned) * (size_t)spans);
     const size_t o_dots = piece(sizeof(long long) * 3 * 2 * (size_t)bpad);
     const size_t zero_bytes = off;
     const size_t o_wdig = piece((size_t)ng * 4 * vec_bytes);
@@ -502,7 +614,13 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     a.p1 = d->plane1; a.p2 = d->plane2; a.row_bytes = rb; a.m = d->m; a.n = (int)d->n; a.bits = d->bits;
     a.lo = d->feat_lo; a.step = d->feat_step; a.b = b; a.x = x; a.grad_out = grad_out;
     a.batch = B; a.lr = p->lr;
-    a.ca = (int)ca; a.spans = spans; a.ncb = (int)ncb64; a.bpc = (int)bpc; a.bpad = bpad; a.vec_bytes = vec_bytes;
+    a.ca = (int)ca; a.spans = (int)spans; a.part_spans = part_spans; a.bpc = (int)bpc; a.bpad = bpad;
+    a.union_bytes = (int)uni; a.vec_bytes = vec_bytes;
+    // two tiles must fit in L2 for the prefetch of the next one to pay; ZIPML_STREAM_PREFETCH=0/1 overrides
+    int l2_bytes = 0;
+    cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, ctx->device);
+    a.l2_prefetch = 4 * B * rb <= (int64_t)l2_bytes ? 1 : 0;
+    if (const char* env = getenv("ZIPML_STREAM_PREFETCH")) a.l2_prefetch = atoi(env) != 0;
     a.barrier = reinterpret_cast<unsigned*>(ctx->ws + o_bar);
     a.ready = reinterpret_cast<unsigned*>(ctx->ws + o_ready);
     a.dots = reinterpret_cast<long long*>(ctx->ws + o_dots);
