@@ -64,7 +64,9 @@ enum {
                                     from global memory into int8 tensor-core fragments (the second pass
                                     from L2), a CTA owns whole column blocks of the gradient, one grid
                                     barrier per step.  ZIPML_ERR_WORKSPACE for level tables, quantized
-                                    model or gradient, batches above 8192 rows                        */
+                                    model or gradient, batches above 8192 rows.  The environment
+                                    variable ZIPML_STREAM_PREFETCH=0..8 overrides how many eighths of
+                                    the next step's tile are requested into L2 ahead of time           */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -111,8 +113,8 @@ typedef struct zipml_sgd_params {
                                    collected, 7 step end.  The last step of a call stops after
                                    mark 4.  Stream engine: 0 step start, 1 own dots added, 2 barrier
                                    passed, 3 residual digits ready, 4 own gradient blocks summed,
-                                   5 model updated and digits published.  Other engines ignore the
-                                   request.                                                           */
+                                   5 model updated and digits published, 6 dots and labels read,
+                                   7 residual scale known.  Other engines ignore the request.         */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

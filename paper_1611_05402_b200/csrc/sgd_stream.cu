@@ -66,7 +66,7 @@ struct StreamArgs {
     int bpc;                 // column blocks per CTA
     int bpad;                // batch rounded up to 32
     int union_bytes;         // shared memory shared by pass A's digits and pass B's residual digits + sums
-    int l2_prefetch;         // ask L2 for the next step's tile while pass B runs
+    int l2_prefetch;         // eighths of the next step's tile to ask L2 for while pass B runs (0..8)
     int64_t vec_bytes;       // bytes of one digit vector (spans * 64)
     signed char* wdig;       // [NG][NS][vec_bytes] digits of w, in the byte order of the codes
     unsigned* ready;         // [spans] number of digit versions published for the block
@@ -88,8 +88,18 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+// Flag store that follows one __threadfence() covering everything published before it.
+__device__ __forceinline__ void st_relaxed_u32(unsigned* p, unsigned v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -139,7 +149,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
     unsigned char* uni = smem + kStreamRingBytes;
     signed char* wds = reinterpret_cast<signed char*>(uni);                      // pass A: [NG * NS][part_spans * 64]
     signed char* rdig = reinterpret_cast<signed char*>(uni);                     // pass B: [2][NS][bpad + 16]
-    int* gacc = reinterpret_cast<int*>(uni + (size_t)2 * NS * (a.bpad + 16));    // pass B: [bpc][NG][CW][NS]
+    int* gacc = reinterpret_cast<int*>(uni + (size_t)2 * NS * (a.bpad + 16));    // pass B: [bpc][NG][CW][NS], one pad word per 32
     float* own = reinterpret_cast<float*>(uni + a.union_bytes);                  // [3][bpc * CW * NG]: lo, step, x of the own features
     double2* rres = reinterpret_cast<double2*>(ring);                            // dots minus labels, between the passes
     __shared__ double shd[kStreamWarps];
@@ -150,13 +160,14 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
     const int n = a.n;
     const int64_t rb = a.row_bytes, vb = a.vec_bytes;
     const int cb0 = min(a.spans, cta * a.bpc), cb1 = min(a.spans, cb0 + a.bpc);
-    const int own_n = (cb1 - cb0) * CW * NG, own_cap = a.bpc * CW * NG;
+    const int own_bytes = (cb1 - cb0) * CW, own_n = own_bytes * NG, own_cap = a.bpc * CW * NG;
+    signed char* dstage = reinterpret_cast<signed char*>(ring);                  // update: [NG * NS][own_bytes]
     float* lo_o = own;
     float* st_o = own + own_cap;
     float* x_o = own + 2 * own_cap;
     const float smax = (float)((1 << a.bits) - 1);
     const uint32_t ring_w = smem_u32(ring) + (uint32_t)warp * S * kStreamStageBytes;
-    const int pstride = a.part_spans * 64 + 16;            // bytes between the digit vectors in wds (16 more: no bank conflicts)
+    const int pstride = a.part_spans * 64 + 64;            // bytes between the digit vectors in wds (64 more: no bank conflicts)
     const int rstride = a.bpad + 16;                       // bytes between the residual digit vectors
 
     // ---- set-up: every CTA scans the model once (identical arithmetic everywhere)
@@ -189,7 +200,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            for (int c = cb0; c < cb1; ++c) st_release_u32(a.ready + c, 1u);
+            for (int c = cb0; c < cb1; ++c) st_relaxed_u32(a.ready + c, 1u);
         }
     }
 
@@ -203,6 +214,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
         const unsigned char* t2 = a.p2 + row0 * rb;
         long long* dots = a.dots + (size_t)(t_rel % 3) * 2 * a.bpad;
         stream_mark(a, t_rel, 0);
+        if (warp == kStreamWarps - 1)          // the step's labels are read right after the barrier: have them in L2 by then
+            for (int k = lane * 32; k < bt; k += 32 * 32) prefetch_l2(a.b + row0 + k);
 
         // ------------------------------------------------------------------ pass A: dots
         {
@@ -310,6 +323,18 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
         if (!grid_barrier(a.barrier, (unsigned)((t_rel + 1) * G), a.status, 21)) return;
         stream_mark(a, t_rel, 2);
 
+        // HBM is idle from here to the next step's first pass: part of the next tile can travel to L2 now
+        // (the whole of it would push this step's tile out before the second pass has read it)
+        if (a.l2_prefetch && !last && warp == kStreamWarps - 1 && lane < 2) {
+            const int64_t itn = it + 1;
+            const int64_t rown = (a.order ? (int64_t)a.order[itn] : itn) * a.batch;
+            const int64_t bytes = min(a.batch, a.m - rown) * rb;          // a multiple of 16
+            const int64_t per = ((bytes / 16 + G - 1) / G) * 16;
+            const int64_t lo_b = min(bytes, per * cta), hi_b = min(bytes, lo_b + (per * a.l2_prefetch / 128) * 16);
+            const unsigned char* srcn = (lane == 0 ? a.p1 : a.p2) + rown * rb;
+            for (int64_t o = lo_b; o < hi_b; o += 32768) l2_prefetch_bulk(srcn + o, (uint32_t)min((int64_t)32768, hi_b - o));
+        }
+
         // ------------------------------------------------------------------ residuals (every CTA, all rows)
         // clear the dots two steps ahead (its last readers passed the previous barrier)
         {
@@ -323,13 +348,23 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             const size_t par = (size_t)(t_rel & 1) * G;
             for (int i = tid; i < G; i += kStreamThreads) { pm = fmaxf(pm, __ldcg(a.wmax_part + par + i)); pb += __ldcg(a.base_part + par + i); }
         }
-        for (int k = tid; k < bt; k += kStreamThreads) {
-            const long long v1 = __ldcg(dots + k), v2 = __ldcg(dots + a.bpad + k);
-            const double bk = (double)a.b[row0 + k];
-            rres[k] = make_double2((double)v1 * delta_w - bk, (double)v2 * delta_w - bk);
+        for (int k0 = tid; k0 < bt; k0 += 4 * kStreamThreads) {           // four rows' loads in flight together
+            long long v1[4], v2[4];
+            float bk[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int k = k0 + q * kStreamThreads;
+                if (k < bt) { v1[q] = __ldcg(dots + k); v2[q] = __ldcg(dots + a.bpad + k); bk[q] = a.b[row0 + k]; }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int k = k0 + q * kStreamThreads;
+                if (k < bt) rres[k] = make_double2((double)v1[q] * delta_w - (double)bk[q], (double)v2[q] * delta_w - (double)bk[q]);
+            }
         }
         block_reduce_mms(rmax, pm, pb, shf, shd);          // rmax is not known yet: this round carries pm and pb
         if (t_rel > 0) { wm = pm; base = pb; }
+        stream_mark(a, t_rel, 6);
         // r = delta_w V + lo^T x - b in double, rounded to fp32 once; the same on every CTA
         for (int k = tid; k < bt; k += kStreamThreads) {
             const double2 d = rres[k];
@@ -340,29 +375,37 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             double none = 0.0;
             block_reduce_mms(rmax, unused, none, shf, shd);
         }
+        stream_mark(a, t_rel, 7);
         const float inv_r = rmax > 0.0f ? (float)QMAX / rmax : 0.0f;
         const double delta_r = (double)rmax / (double)QMAX;
         double rsum = 0.0;                 // sum of all fixed-point residuals (exact in double)
-        for (int k = tid; k < a.bpad; k += kStreamThreads) {
-            int R1 = 0, R2 = 0;
-            if (k < bt) {
-                const double2 d = rres[k];
-                R1 = fixed_point((float)(d.x + base), inv_r);
-                R2 = fixed_point((float)(d.y + base), inv_r);
+        // a thread takes rows t, t+4, t+8, t+12 of a group of 16: their digits are one 32-bit word of pass B's operand
+        for (int q4 = tid; q4 < a.bpad / 4; q4 += kStreamThreads) {
+            const int kb = (q4 >> 2) * 16 + (q4 & 3);
+            uint32_t w1[NS] = {0u, 0u, 0u, 0u}, w2[NS] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = kb + 4 * i;
+                int R1 = 0, R2 = 0;
+                if (k < bt) {
+                    const double2 d = rres[k];
+                    R1 = fixed_point((float)(d.x + base), inv_r);
+                    R2 = fixed_point((float)(d.y + base), inv_r);
+                }
+                rsum += (double)R1 + (double)R2;
+                int d1[NS], d2[NS];
+                balanced_digits<NS>(R1, d1);
+                balanced_digits<NS>(R2, d2);
+#pragma unroll
+                for (int q = 0; q < NS; ++q) { w1[q] |= (uint32_t)(d1[q] & 255) << (8 * i); w2[q] |= (uint32_t)(d2[q] & 255) << (8 * i); }
             }
-            rsum += (double)R1 + (double)R2;
-            // within a group of 16 rows, row r sits at 4 (r % 4) + r / 4: a 32-bit word holds rows t, t+4, t+8, t+12
-            const int kp = (k & ~15) | ((k & 3) << 2) | ((k >> 2) & 3);
-            int d1[NS], d2[NS];
-            balanced_digits<NS>(R1, d1);
-            balanced_digits<NS>(R2, d2);
 #pragma unroll
             for (int q = 0; q < NS; ++q) {
-                rdig[(size_t)q * rstride + kp] = (signed char)d2[q];               // plane 1 meets r2
-                rdig[(size_t)(NS + q) * rstride + kp] = (signed char)d1[q];        // plane 2 meets r1
+                *reinterpret_cast<uint32_t*>(rdig + (size_t)q * rstride + 4 * q4) = w2[q];             // plane 1 meets r2
+                *reinterpret_cast<uint32_t*>(rdig + (size_t)(NS + q) * rstride + 4 * q4) = w1[q];      // plane 2 meets r1
             }
         }
-        for (int i = tid; i < (cb1 - cb0) * NG * CW * NS; i += kStreamThreads) gacc[i] = 0;
+        for (int i = tid; i < (cb1 - cb0) * NG * CW * NS * 33 / 32; i += kStreamThreads) gacc[i] = 0;
         {
             float u1 = 0.0f, u2 = 0.0f;
             block_reduce_mms(u1, u2, rsum, shf, shd);      // its barriers publish rdig and the cleared sums
@@ -370,17 +413,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
         // scale of the next model's digits: a bound that writers and readers both know now
         const float bound_next = (wm + fabsf(a.lr) * cmax * rmax) * 1.0001f;
         stream_mark(a, t_rel, 3);
-
-        // the next step's tile can travel to L2 while this step's second pass reads from L2
-        if (a.l2_prefetch && !last && warp == kStreamWarps - 1 && lane < 2) {
-            const int64_t itn = it + 1;
-            const int64_t rown = (a.order ? (int64_t)a.order[itn] : itn) * a.batch;
-            const int64_t bytes = min(a.batch, a.m - rown) * rb;          // a multiple of 16
-            const int64_t per = ((bytes / 16 + G - 1) / G) * 16;
-            const int64_t lo_b = min(bytes, per * cta), hi_b = min(bytes, lo_b + per);
-            const unsigned char* srcn = (lane == 0 ? a.p1 : a.p2) + rown * rb;
-            for (int64_t o = lo_b; o < hi_b; o += 32768) l2_prefetch_bulk(srcn + o, (uint32_t)min((int64_t)32768, hi_b - o));
-        }
 
         // ------------------------------------------------------------------ pass B: gradient of the own blocks
         {
@@ -396,6 +428,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             // residual digits are stored in the matching row order.
             const uint32_t rb32 = (uint32_t)rb;
             const uint32_t stage0 = ring_w + lane * 16;
+            const uint64_t dead = l2_evict_first_policy();    // the tile is not read again: its lines may leave L2 first
             int i_ci = 0, i_rem = 0;                       // issue side: column block and position within it
             auto issue = [&]() {
                 if (i_ci < cb1 - cb0) {
@@ -407,7 +440,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                         const uint32_t o = (uint32_t)r0 * rb32;
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            if (r0 + 8 * k < bt) cp_async16(dst + k * 512, tp + (o + 8 * k * rb32));
+                            if (r0 + 8 * k < bt) cp_async16_hint(dst + k * 512, tp + (o + 8 * k * rb32), dead);
                     }
                     if (++i_rem == per_c) { i_rem = 0; ++i_ci; }
                 }
@@ -464,7 +497,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                 }
                 if (++rem == per_c) {
                     // lane t < 2: acc[g][w][u][0..1] = digits 2t, 2t+1 of byte 4w+2u of the lane's bytes, [2..3] of byte 4w+2u+1
-                    int* dst = gacc + (size_t)ci * NG * CW * NS;
+                    // entry e lives at e + e / 32: the eight lane groups, 32 entries apart, hit eight banks
+                    const int e0 = ci * NG * CW * NS;
 #pragma unroll
                     for (int g = 0; g < NG; ++g)
 #pragma unroll
@@ -472,7 +506,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
 #pragma unroll
                             for (int u = 0; u < 2; ++u) {
                                 if (tl < 2) {
-                                    int* p = dst + ((size_t)g * CW + gl * 8 + 4 * w + 2 * u) * NS + 2 * tl;
+                                    const int e = e0 + (g * CW + gl * 8 + 4 * w + 2 * u) * NS + 2 * tl;
+                                    int* p = gacc + e + (e >> 5);
                                     atomicAdd(p, acc[g][w][u][0] >> (g * CB));
                                     atomicAdd(p + 1, acc[g][w][u][1] >> (g * CB));
                                     atomicAdd(p + NS, acc[g][w][u][2] >> (g * CB));
@@ -504,7 +539,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                 int W = 0;
                 if (j < n) {
                     const int cl = bl / CW, bb = bl - cl * CW;
-                    const int* src = gacc + (((size_t)cl * NG + grp) * CW + bb) * NS;
+                    const int e = ((cl * NG + grp) * CW + bb) * NS;
+                    const int* src = gacc + e + (e >> 5);
                     const int sv[NS] = {src[0], src[1], src[2], src[3]};
                     const long long Sj = combine_digits<NS>(sv);
                     const float l = lo_o[idx], st = st_o[idx];
@@ -518,21 +554,30 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                     pbase += (double)l * (double)xn;
                     W = fixed_point(w, inv);
                 }
-                if (!last) {
+                if (!last) {               // digits meet in shared memory (the ring is idle) and leave as 16-byte stores
                     int d[NS];
                     balanced_digits<NS>(W, d);
 #pragma unroll
-                    for (int k = 0; k < NS; ++k) a.wdig[((int64_t)grp * NS + k) * vb + byte] = (signed char)d[k];
+                    for (int k = 0; k < NS; ++k) dstage[(grp * NS + k) * own_bytes + bl] = (signed char)d[k];
                 }
             }
             if (last) break;
-            block_reduce_mms(pmax, unused, pbase, shf, shd);   // its barriers: every digit store of the CTA is issued
+            block_reduce_mms(pmax, unused, pbase, shf, shd);
+            {
+                const int p16 = own_bytes / 16;
+                for (int idx = tid; idx < NG * NS * p16; idx += kStreamThreads) {
+                    const int v = idx / p16, q = idx - v * p16;
+                    *reinterpret_cast<uint4*>(a.wdig + (int64_t)v * vb + (int64_t)cb0 * CW + q * 16) =
+                        *reinterpret_cast<const uint4*>(dstage + v * own_bytes + q * 16);
+                }
+            }
+            __syncthreads();               // every digit store of the CTA is issued; the ring is free again
             if (tid == 0) {
                 const size_t par = (size_t)((t_rel + 1) & 1) * G;
                 a.wmax_part[par + cta] = pmax;
                 a.base_part[par + cta] = pbase;
                 __threadfence();
-                for (int c = cb0; c < cb1; ++c) st_release_u32(a.ready + c, (unsigned)(t_rel + 2));
+                for (int c = cb0; c < cb1; ++c) st_relaxed_u32(a.ready + c, (unsigned)(t_rel + 2));
             }
             bound = bound_next;
         }
@@ -582,8 +627,8 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     const int part_spans = (int)((spans + ca - 1) / ca);
     const int64_t vec_bytes = spans * 64;
 
-    const size_t pass_a = (size_t)ng * 4 * (part_spans * 64 + 16);
-    const size_t pass_b = (size_t)2 * 4 * (bpad + 16) + sizeof(int) * (size_t)bpc * ng * cw * 4;
+    const size_t pass_a = (size_t)ng * 4 * (part_spans * 64 + 64);
+    const size_t pass_b = (size_t)2 * 4 * (bpad + 16) + sizeof(int) * (size_t)bpc * ng * cw * 4 * 33 / 32;
     const size_t uni = ((pass_a > pass_b ? pass_a : pass_b) + 127) / 128 * 128;
     const size_t smem = (size_t)kStreamRingBytes + uni + sizeof(float) * 3 * (size_t)bpc * cw * ng;
     if (smem > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
@@ -616,11 +661,13 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     a.batch = B; a.lr = p->lr;
     a.ca = (int)ca; a.spans = (int)spans; a.part_spans = part_spans; a.bpc = (int)bpc; a.bpad = bpad;
     a.union_bytes = (int)uni; a.vec_bytes = vec_bytes;
-    // two tiles must fit in L2 for the prefetch of the next one to pay; ZIPML_STREAM_PREFETCH=0/1 overrides
+    // The whole next tile where two tiles fit L2 with room to spare, a quarter of it where one and a half do
+    // (measured on 64 MB tiles in a 126 MB L2: 2/8 gains 3 %, 8/8 loses 6 %); ZIPML_STREAM_PREFETCH=0..8 overrides
     int l2_bytes = 0;
     cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, ctx->device);
-    a.l2_prefetch = 4 * B * rb <= (int64_t)l2_bytes ? 1 : 0;
-    if (const char* env = getenv("ZIPML_STREAM_PREFETCH")) a.l2_prefetch = atoi(env) != 0;
+    const int64_t step_bytes = 2 * B * rb;
+    a.l2_prefetch = 9 * step_bytes <= 4 * (int64_t)l2_bytes ? 8 : 3 * step_bytes <= 2 * (int64_t)l2_bytes ? 2 : 0;
+    if (const char* env = getenv("ZIPML_STREAM_PREFETCH")) { a.l2_prefetch = atoi(env); if (a.l2_prefetch < 0 || a.l2_prefetch > 8) a.l2_prefetch = 0; }
     a.barrier = reinterpret_cast<unsigned*>(ctx->ws + o_bar);
     a.ready = reinterpret_cast<unsigned*>(ctx->ws + o_ready);
     a.dots = reinterpret_cast<long long*>(ctx->ws + o_dots);
