@@ -438,9 +438,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                         const unsigned char* tp = ((i_rem & 1) ? t2 : t1) + coff;
                         const uint32_t dst = stage0 + (uint32_t)((i_ci * per_c + i_rem) & (S - 1)) * kStreamStageBytes;
                         const uint32_t o = (uint32_t)r0 * rb32;
+                        // A 128-byte line holds two column blocks.  Once this CTA has read both, nobody reads the
+                        // line again this step: only then may it leave L2 ahead of the rest.
+                        const bool second = i_ci > 0 && ((cb0 + i_ci) & 1);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            if (r0 + 8 * k < bt) cp_async16_hint(dst + k * 512, tp + (o + 8 * k * rb32), dead);
+                            if (r0 + 8 * k < bt) {
+                                if (second) cp_async16_hint(dst + k * 512, tp + (o + 8 * k * rb32), dead);
+                                else cp_async16(dst + k * 512, tp + (o + 8 * k * rb32));
+                            }
                     }
                     if (++i_rem == per_c) { i_rem = 0; ++i_ci; }
                 }
