@@ -232,6 +232,22 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
         }
     };
 
+    // the same for padded rows, called by every warp: lane 0 of warp w issues pieces w, w + 16, ...
+    auto issue_tile_rows = [&](int64_t it, int slot) {
+        int64_t r0; int bt, rcnt;
+        step_rows(it, r0, bt, rcnt);
+        uint64_t* full = reinterpret_cast<uint64_t*>(sh->full + slot);
+        if (lane != 0) return;
+        // (bytes that land before the count is armed are held against it: the phase cannot complete earlier)
+        if (warp == kCluWarps - 1) mbar_arrive_expect_tx(full, 2u * (uint32_t)rcnt * (uint32_t)rw * 4u);
+        uint32_t* dst = ring + (size_t)slot * slot_words;
+        const size_t src = (size_t)(r0 + k0) * rw;
+        for (int i = warp; i < 2 * rcnt; i += kCluWarps) {
+            const int pl = i & 1, r = i >> 1;
+            bulk_copy_g2s(dst + (size_t)(pl * a.rc + r) * pitch, (pl ? a.p2 : a.p1) + src + (size_t)r * rw, (uint32_t)rw * 4u, full);
+        }
+    };
+
     if (tid == 0) {
         for (int s = 0; s < a.slots; ++s) mbar_init(reinterpret_cast<uint64_t*>(sh->full + s), 1);
         mbar_init(reinterpret_cast<uint64_t*>(&sh->rs_bar), 1);
@@ -577,7 +593,12 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                 bulk_copy_s2c(cluster_addr(gbuf + (size_t)bi * sub, warp), gpart + (size_t)warp * sub, slice_bytes,
                               cluster_addr(&sh->rs_bar, warp));
             // the tile is consumed: refill its slot while the parts travel
-            if (warp == kCluWarps - 1 && it + a.slots < step_end) issue_tile(it + a.slots, slot);
+            // (row-by-row tiles: the warps share the rows, since one warp issues its copies one after the other
+            // and a whole tile from one warp held the CTA's next barrier back by thousands of cycles)
+            if (it + a.slots < step_end) {
+                if (pitch == rw) { if (warp == kCluWarps - 1) issue_tile(it + a.slots, slot); }
+                else issue_tile_rows(it + a.slots, slot);
+            }
             if (++slot == a.slots) { slot = 0; parity ^= 1u; }
             clu_mark(a, it, 3);
 
