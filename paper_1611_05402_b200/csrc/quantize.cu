@@ -115,12 +115,18 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
 }
 
 // ---------------------------------------------------------------------------------------------
-// Quantize + pack.  One thread produces one 32-bit word of each plane: FPW = 32/CB consecutive
-// features of one row.  It reads them as float4s when the row is 16-byte aligned, decides the cell
-// and the up-probability in pinned fp32 arithmetic, draws one Philox block per feature pair (four
-// words = two features x two copies) and writes the two words.  Words past the last feature are
-// written as zero so that the planes are fully defined.
+// Quantize + pack.  A thread owns one 32-bit word column of the planes (FPW = 32/CB consecutive
+// features) for kQuantRows consecutive rows: the features' lo and inv are loaded once, the rows'
+// Philox chains are independent and overlap.  Per row it reads the FPW samples as float4s when the
+// row is 16-byte aligned, decides cell and up-probability in pinned fp32 arithmetic, draws one
+// Philox block per feature pair (four words = two features x two copies) and writes the two
+// words.  A pair whose up-probabilities are all 0 or 1 (values on a level: the zeros of sparse
+// rows, the column extremes) needs no random numbers -- the comparison u * 2^-24 < p is decided
+// without them -- and skips its Philox block; the codes are the same.  Words past the last
+// feature are written as zero so that the planes are fully defined.
 // ---------------------------------------------------------------------------------------------
+constexpr int kQuantRows = 4;
+
 template <int CB, bool TABLE>
 __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__ A, int64_t m, int64_t n, int64_t lda,
                                                        int bits, const float* __restrict__ lo,
@@ -128,58 +134,77 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                                                        uint64_t seed, uint32_t* __restrict__ plane1,
                                                        uint32_t* __restrict__ plane2, int64_t row_words, bool vec_ok) {
     constexpr int FPW = 32 / CB;
-    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (id >= m * row_words) return;
-    const int64_t row = id / row_words;
-    const int64_t q = id - row * row_words;
+    // blockDim = (word columns, row groups); blockIdx.x runs over the rows, blockIdx.y over the columns
+    const int64_t q = (int64_t)blockIdx.y * blockDim.x + threadIdx.x;
+    const int64_t row_first = ((int64_t)blockIdx.x * blockDim.y + threadIdx.y) * kQuantRows;
+    if (q >= row_words || row_first >= m) return;
     const int64_t j0 = q * FPW;
     const int L = 1 << bits, s = L - 1;
-    uint32_t w1 = 0u, w2 = 0u;
-    if (j0 < n) {
-        float v[FPW];
-        const float* src = A + row * lda + j0;
-        if (vec_ok && j0 + FPW <= n) {
+    const int nf = (int)min((int64_t)FPW, n - j0);                 // real features of this word (<= 0: padding only)
+    float flo[TABLE ? 1 : FPW], finv[TABLE ? 1 : FPW];
+    if constexpr (!TABLE) {
 #pragma unroll
-            for (int i = 0; i < FPW / 4; ++i) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(src) + i);
-                v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < FPW; ++i) v[i] = (j0 + i < n) ? __ldg(src + i) : 0.0f;
-        }
-#pragma unroll
-        for (int pr = 0; pr < FPW / 2; ++pr) {
-            const int64_t ja = j0 + 2 * pr;
-            if (ja >= n) break;
-            const Philox4 rnd = sample_block(seed, (uint64_t)row, (uint32_t)(ja >> 1));
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int64_t j = ja + h;
-                if (j >= n) break;
-                uint32_t cell;
-                float p;
-                if (!TABLE) {
-                    uniform_cell(v[2 * pr + h], __ldg(lo + j), __ldg(inv + j), s, cell, p);
-                } else {
-                    const float* lev = levels + j * L;
-                    const float val = v[2 * pr + h];
-                    int l = 0;
-                    for (int i = 1; i <= s - 1; ++i) l = (__ldg(lev + i) <= val) ? i : l;
-                    const float base = __ldg(lev + l);
-                    const float width = __fsub_rn(__ldg(lev + l + 1), base);
-                    cell = (uint32_t)l;
-                    p = width > 0.0f ? __fdiv_rn(__fsub_rn(val, base), width) : 0.0f;
-                }
-                const uint32_t c1 = round_up_if(cell, p, rnd.v[2 * h]);
-                const uint32_t c2 = round_up_if(cell, p, rnd.v[2 * h + 1]);
-                w1 |= c1 << ((2 * pr + h) * CB);
-                w2 |= c2 << ((2 * pr + h) * CB);
-            }
+        for (int i = 0; i < FPW; ++i) {
+            flo[i] = i < nf ? __ldg(lo + j0 + i) : 0.0f;
+            finv[i] = i < nf ? __ldg(inv + j0 + i) : 0.0f;
         }
     }
-    plane1[row * row_words + q] = w1;
-    plane2[row * row_words + q] = w2;
+    const bool vec = vec_ok && nf == FPW;
+#pragma unroll 2
+    for (int rr = 0; rr < kQuantRows; ++rr) {
+        const int64_t row = row_first + rr;
+        if (row >= m) break;
+        uint32_t w1 = 0u, w2 = 0u;
+        if (nf > 0) {
+            float v[FPW];
+            const float* src = A + row * lda + j0;
+            if (vec) {
+#pragma unroll
+                for (int i = 0; i < FPW / 4; ++i) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(src) + i);
+                    v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < FPW; ++i) v[i] = (i < nf) ? __ldg(src + i) : 0.0f;
+            }
+#pragma unroll
+            for (int pr = 0; pr < FPW / 2; ++pr) {
+                if (2 * pr >= nf) break;
+                uint32_t cell[2] = {0u, 0u};
+                float p[2] = {0.0f, 0.0f};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int i = 2 * pr + h;
+                    if (i >= nf) break;
+                    if constexpr (!TABLE) {
+                        uniform_cell(v[i], flo[i], finv[i], s, cell[h], p[h]);
+                    } else {
+                        const float* lev = levels + (j0 + i) * L;
+                        int l = 0;
+                        for (int k = 1; k <= s - 1; ++k) l = (__ldg(lev + k) <= v[i]) ? k : l;
+                        const float base = __ldg(lev + l);
+                        const float width = __fsub_rn(__ldg(lev + l + 1), base);
+                        cell[h] = (uint32_t)l;
+                        p[h] = width > 0.0f ? __fdiv_rn(__fsub_rn(v[i], base), width) : 0.0f;
+                    }
+                }
+                const bool random = (p[0] > 0.0f && p[0] < 1.0f) || (p[1] > 0.0f && p[1] < 1.0f);
+                Philox4 rnd;
+                if (random) rnd = sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr));
+                else rnd.v[0] = rnd.v[1] = rnd.v[2] = rnd.v[3] = 0u;    // decided without them: p <= 0 never up, p >= 1 always up
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int i = 2 * pr + h;
+                    if (i >= nf) break;
+                    w1 |= round_up_if(cell[h], p[h], rnd.v[2 * h]) << (i * CB);
+                    w2 |= round_up_if(cell[h], p[h], rnd.v[2 * h + 1]) << (i * CB);
+                }
+            }
+        }
+        plane1[row * row_words + q] = w1;
+        plane2[row * row_words + q] = w2;
+    }
 }
 
 int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
@@ -187,16 +212,20 @@ int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_
                     uint8_t* plane2, int64_t row_bytes) {
     const int cb = container_bits(bits);
     const int64_t row_words = row_bytes / 4;
-    const int64_t total = m * row_words;
-    const int64_t blocks = (total + 255) / 256;
-    if (blocks > 0x7fffffffLL) return ZIPML_ERR_WORKSPACE;
+    // 256 threads: as many word columns as the row has (a power of two from 8 to 256), the rest row groups
+    int tx = 8;
+    while (tx < 256 && tx < row_words) tx *= 2;
+    const int ty = 256 / tx;
+    const int64_t row_blocks = (m + (int64_t)ty * kQuantRows - 1) / ((int64_t)ty * kQuantRows);
+    const int64_t col_blocks = (row_words + tx - 1) / tx;
+    if (row_blocks > 0x7fffffffLL || col_blocks > 65535) return ZIPML_ERR_WORKSPACE;
+    const dim3 grid((unsigned)row_blocks, (unsigned)col_blocks), block((unsigned)tx, (unsigned)ty);
     const bool vec_ok = (lda % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0);
     uint32_t* p1 = reinterpret_cast<uint32_t*>(plane1);
     uint32_t* p2 = reinterpret_cast<uint32_t*>(plane2);
     const bool table = level_mode == ZIPML_LEVELS_TABLE;
-#define ZIPML_LAUNCH_Q(CB_, T_)                                                                         \
-    quantize_kernel<CB_, T_><<<(unsigned)blocks, 256, 0, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, p1, \
-                                                                        p2, row_words, vec_ok)
+#define ZIPML_LAUNCH_Q(CB_, T_) \
+    quantize_kernel<CB_, T_><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, p1, p2, row_words, vec_ok)
     if (cb == 2) { if (table) ZIPML_LAUNCH_Q(2, true); else ZIPML_LAUNCH_Q(2, false); }
     else if (cb == 4) { if (table) ZIPML_LAUNCH_Q(4, true); else ZIPML_LAUNCH_Q(4, false); }
     else { ZIPML_LAUNCH_Q(8, false); }
