@@ -291,8 +291,10 @@ int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, 
     float* dx = reinterpret_cast<float*>(s + ox);
     float* dlev = reinterpret_cast<float*>(s + olev);
     double* dloss = reinterpret_cast<double*>(s + oloss);
-    cudaError_t e = cudaMemcpy2DAsync(dA, sizeof(float) * n, A_host, sizeof(float) * lda, sizeof(float) * n, (size_t)m,
-                                      cudaMemcpyHostToDevice, ctx->stream);
+    // (contiguous rows travel as one linear copy: a pitched copy of many short rows is much slower)
+    cudaError_t e = lda == n ? cudaMemcpyAsync(dA, A_host, sizeof(float) * (size_t)m * n, cudaMemcpyHostToDevice, ctx->stream)
+                             : cudaMemcpy2DAsync(dA, sizeof(float) * n, A_host, sizeof(float) * lda, sizeof(float) * n, (size_t)m,
+                                                 cudaMemcpyHostToDevice, ctx->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(db, b_host, sizeof(float) * m, cudaMemcpyHostToDevice, ctx->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(dx, x_host, sizeof(float) * n, cudaMemcpyHostToDevice, ctx->stream);
     if (e != cudaSuccess) return cuda_status(e);
