@@ -124,22 +124,39 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
 // rows, the column extremes) needs no random numbers -- the comparison u * 2^-24 < p is decided
 // without them -- and skips its Philox block; the codes are the same.  Words past the last
 // feature are written as zero so that the planes are fully defined.
+// Level tables: the block's tables are staged in shared memory as [level][feature slot of the
+// word][word column], so that the lanes of a warp (consecutive word columns) read consecutive
+// addresses; read from global memory, where the tables of neighbouring lanes lie FPW * L floats
+// apart, every look-up took 32 cache lines per warp and the kernel ran at a tenth of this rate.
 // ---------------------------------------------------------------------------------------------
-constexpr int kQuantRows = 4;
+constexpr int kQuantRows = 4;          // rows per thread and pass
+constexpr int kQuantTableCols = 64;    // word columns per block with level tables (shared memory: L * FPW * 64 floats)
 
 template <int CB, bool TABLE>
 __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__ A, int64_t m, int64_t n, int64_t lda,
                                                        int bits, const float* __restrict__ lo,
                                                        const float* __restrict__ inv, const float* __restrict__ levels,
                                                        uint64_t seed, uint32_t* __restrict__ plane1,
-                                                       uint32_t* __restrict__ plane2, int64_t row_words, bool vec_ok) {
+                                                       uint32_t* __restrict__ plane2, int64_t row_words, bool vec_ok,
+                                                       int passes) {
     constexpr int FPW = 32 / CB;
+    extern __shared__ float lev_s[];                               // TABLE: [L][FPW][blockDim.x]
     // blockDim = (word columns, row groups); blockIdx.x runs over the rows, blockIdx.y over the columns
     const int64_t q = (int64_t)blockIdx.y * blockDim.x + threadIdx.x;
-    const int64_t row_first = ((int64_t)blockIdx.x * blockDim.y + threadIdx.y) * kQuantRows;
-    if (q >= row_words || row_first >= m) return;
-    const int64_t j0 = q * FPW;
     const int L = 1 << bits, s = L - 1;
+    if constexpr (TABLE) {
+        const int tx = blockDim.x, nthreads = blockDim.x * blockDim.y, tid = threadIdx.y * blockDim.x + threadIdx.x;
+        const int64_t jb = (int64_t)blockIdx.y * tx * FPW;         // first feature of the block
+        // consecutive threads read consecutive floats of the n x L table
+        for (int idx = tid; idx < tx * FPW * L; idx += nthreads) {
+            const int f = idx / L, k = idx - f * L;                // feature within the block, level
+            const float val = (jb + f < n) ? __ldg(levels + (jb + f) * L + k) : 0.0f;
+            lev_s[(k * FPW + (f % FPW)) * tx + f / FPW] = val;
+        }
+        __syncthreads();
+    }
+    if (q >= row_words) return;
+    const int64_t j0 = q * FPW;
     const int nf = (int)min((int64_t)FPW, n - j0);                 // real features of this word (<= 0: padding only)
     float flo[TABLE ? 1 : FPW], finv[TABLE ? 1 : FPW];
     if constexpr (!TABLE) {
@@ -150,8 +167,9 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
         }
     }
     const bool vec = vec_ok && nf == FPW;
+    const int64_t row_first = ((int64_t)blockIdx.x * blockDim.y + threadIdx.y) * kQuantRows * passes;
 #pragma unroll 2
-    for (int rr = 0; rr < kQuantRows; ++rr) {
+    for (int rr = 0; rr < kQuantRows * passes; ++rr) {
         const int64_t row = row_first + rr;
         if (row >= m) break;
         uint32_t w1 = 0u, w2 = 0u;
@@ -180,11 +198,12 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                     if constexpr (!TABLE) {
                         uniform_cell(v[i], flo[i], finv[i], s, cell[h], p[h]);
                     } else {
-                        const float* lev = levels + (j0 + i) * L;
+                        const float* lev = lev_s + i * blockDim.x + threadIdx.x;       // level k at lev[k * FPW * blockDim.x]
+                        const int ls = FPW * blockDim.x;
                         int l = 0;
-                        for (int k = 1; k <= s - 1; ++k) l = (__ldg(lev + k) <= v[i]) ? k : l;
-                        const float base = __ldg(lev + l);
-                        const float width = __fsub_rn(__ldg(lev + l + 1), base);
+                        for (int k = 1; k <= s - 1; ++k) l = (lev[k * ls] <= v[i]) ? k : l;
+                        const float base = lev[l * ls];
+                        const float width = __fsub_rn(lev[(l + 1) * ls], base);
                         cell[h] = (uint32_t)l;
                         p[h] = width > 0.0f ? __fdiv_rn(__fsub_rn(v[i], base), width) : 0.0f;
                     }
@@ -212,20 +231,24 @@ int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_
                     uint8_t* plane2, int64_t row_bytes) {
     const int cb = container_bits(bits);
     const int64_t row_words = row_bytes / 4;
-    // 256 threads: as many word columns as the row has (a power of two from 8 to 256), the rest row groups
+    const bool table = level_mode == ZIPML_LEVELS_TABLE;
+    // 256 threads: as many word columns as the row has (a power of two from 8 to 256; 64 with level tables),
+    // the rest row groups; with level tables a thread makes four passes, so that staging the tables pays
     int tx = 8;
-    while (tx < 256 && tx < row_words) tx *= 2;
+    while (tx < (table ? kQuantTableCols : 256) && tx < row_words) tx *= 2;
     const int ty = 256 / tx;
-    const int64_t row_blocks = (m + (int64_t)ty * kQuantRows - 1) / ((int64_t)ty * kQuantRows);
+    const int passes = table ? 4 : 1;
+    const size_t smem = table ? sizeof(float) * ((size_t)1 << bits) * (32 / cb) * tx : 0;
+    const int64_t rows_per_block = (int64_t)ty * kQuantRows * passes;
+    const int64_t row_blocks = (m + rows_per_block - 1) / rows_per_block;
     const int64_t col_blocks = (row_words + tx - 1) / tx;
     if (row_blocks > 0x7fffffffLL || col_blocks > 65535) return ZIPML_ERR_WORKSPACE;
     const dim3 grid((unsigned)row_blocks, (unsigned)col_blocks), block((unsigned)tx, (unsigned)ty);
     const bool vec_ok = (lda % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0);
     uint32_t* p1 = reinterpret_cast<uint32_t*>(plane1);
     uint32_t* p2 = reinterpret_cast<uint32_t*>(plane2);
-    const bool table = level_mode == ZIPML_LEVELS_TABLE;
 #define ZIPML_LAUNCH_Q(CB_, T_) \
-    quantize_kernel<CB_, T_><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, p1, p2, row_words, vec_ok)
+    quantize_kernel<CB_, T_><<<grid, block, smem, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, p1, p2, row_words, vec_ok, passes)
     if (cb == 2) { if (table) ZIPML_LAUNCH_Q(2, true); else ZIPML_LAUNCH_Q(2, false); }
     else if (cb == 4) { if (table) ZIPML_LAUNCH_Q(4, true); else ZIPML_LAUNCH_Q(4, false); }
     else { ZIPML_LAUNCH_Q(8, false); }
