@@ -91,10 +91,26 @@ __global__ void __launch_bounds__(kDpThreads) levels_dp_kernel(const uint32_t* _
     const int64_t j_feat = blockIdx.x;
     const uint32_t* cnt = counts + j_feat * M;
 
-    if (threadIdx.x == 0) {
+    // prefix sums of c, c x, c x^2: every thread sums a run of bins, the runs' totals are scanned by warp 0
+    {
+        __shared__ unsigned long long tot[3][kDpThreads];
+        const int per = (M + kDpThreads - 1) / kDpThreads;
+        const int i_begin = min(M, (int)threadIdx.x * per), i_end = min(M, i_begin + per);
         unsigned long long a0 = 0, a1 = 0, a2 = 0;
-        P0[0] = P1[0] = P2[0] = 0;
-        for (int i = 0; i < M; ++i) {
+        for (int i = i_begin; i < i_end; ++i) {
+            const unsigned long long c = cnt[i], x = 2ull * i + 1ull;
+            a0 += c; a1 += c * x; a2 += c * x * x;
+        }
+        tot[0][threadIdx.x] = a0; tot[1][threadIdx.x] = a1; tot[2][threadIdx.x] = a2;
+        __syncthreads();
+        if (threadIdx.x < 3) {                     // exclusive scan of one of the three rows (256 additions)
+            unsigned long long run = 0;
+            for (int t = 0; t < kDpThreads; ++t) { const unsigned long long v = tot[threadIdx.x][t]; tot[threadIdx.x][t] = run; run += v; }
+        }
+        __syncthreads();
+        a0 = tot[0][threadIdx.x]; a1 = tot[1][threadIdx.x]; a2 = tot[2][threadIdx.x];
+        if (threadIdx.x == 0) P0[0] = P1[0] = P2[0] = 0;
+        for (int i = i_begin; i < i_end; ++i) {
             const unsigned long long c = cnt[i], x = 2ull * i + 1ull;
             a0 += c; a1 += c * x; a2 += c * x * x;
             P0[i + 1] = a0; P1[i + 1] = a1; P2[i + 1] = a2;
@@ -109,11 +125,46 @@ __global__ void __launch_bounds__(kDpThreads) levels_dp_kernel(const uint32_t* _
     __syncthreads();
     unsigned long long* prev = Ta;
     unsigned long long* cur = Tb;
+    // The interval cost satisfies the quadrangle inequality (a point of [b,c) adds (2d-2c)(2b-2a) >= 0 to
+    // w(a,d) + w(b,c) - w(a,c) - w(b,d), points left and right of it add non-negative amounts too), so the
+    // leftmost minimiser j*(m) of prev[j] + cost(j, m) does not decrease with m.  Anchors -- every 32nd m
+    // and m = M -- are minimised over their whole range by a warp each; every other m then only scans from
+    // its lower anchor's minimiser to its upper anchor's.  The minima, and with ascending scans and strict
+    // comparisons the leftmost minimisers, are those of the full scan.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kStride = 32;
     for (int k = 2; k <= s; ++k) {
-        for (int mm = k + threadIdx.x; mm <= M; mm += kDpThreads) {
+        const int first_anchor = (k + kStride - 1) / kStride;          // anchors at kStride * a, a >= first_anchor, and at M
+        const int n_mult = M / kStride >= first_anchor ? M / kStride - first_anchor + 1 : 0;
+        const bool m_extra = (M % kStride) != 0 || n_mult == 0;         // M itself, if it is not a multiple already
+        const int n_anchor = n_mult + (m_extra ? 1 : 0);
+        for (int a = warp; a < n_anchor; a += kDpThreads / 32) {
+            const int mm = a < n_mult ? (first_anchor + a) * kStride : M;
             unsigned long long best = ~0ull;
-            int bj = k - 1;
-            for (int j = k - 1; j <= mm - 1; ++j) {
+            int bj = 0x7fffffff;
+            for (int j = k - 1 + lane; j <= mm - 1; j += 32) {
+                const unsigned long long c = prev[j] + cost(j, mm);
+                if (c < best) { best = c; bj = j; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+                if (ob < best || (ob == best && oj < bj)) { best = ob; bj = oj; }
+            }
+            if (lane == 0) { cur[mm] = best; arg[k * M1 + mm] = (unsigned short)bj; }
+        }
+        __syncthreads();
+        for (int mm = k + threadIdx.x; mm <= M; mm += kDpThreads) {
+            if (mm == M || (mm % kStride == 0 && mm / kStride >= first_anchor)) continue;      // an anchor
+            const int below = (mm / kStride) * kStride;
+            int above = below + kStride;
+            if (above > M) above = M;
+            const int j_lo = (below / kStride >= first_anchor && below >= k) ? (int)arg[k * M1 + below] : k - 1;
+            const int j_hi = min((int)arg[k * M1 + above], mm - 1);
+            unsigned long long best = ~0ull;
+            int bj = j_lo;
+            for (int j = j_lo; j <= j_hi; ++j) {
                 const unsigned long long c = prev[j] + cost(j, mm);
                 if (c < best) { best = c; bj = j; }
             }

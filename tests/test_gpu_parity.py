@@ -127,6 +127,22 @@ def test_optimal_levels_bit_exact(ctx, m, n, bits, bins):
     assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all()
 
 
+@pytest.mark.parametrize("distinct,bits,bins", [(3, 3, 1024), (6, 2, 1024), (40, 4, 512), (2, 3, 100)])
+def test_optimal_levels_bit_exact_with_many_empty_bins(ctx, distinct, bits, bins):
+    """Few distinct values: most bins are empty and many level sets cost the same, so the result hangs on the
+    tie rule (smallest index) -- which the kernel's narrowed search must keep."""
+    rng = np.random.default_rng(distinct)
+    vals = np.sort(rng.uniform(-1.0, 1.0, distinct)).astype(np.float32)
+    A = vals[rng.integers(0, distinct, size=(4000, 24))]
+    A[:, 5] = vals[0]                                              # a constant feature
+    A[:100, 7] = 1.5                                               # a far outlier: long empty stretch
+    lev, obj = oracle.optimal_levels(A, bits, bins)
+    glev, gobj = ctx.zipml_optimal_levels(to_dev(A, ctx), bits, bins, want_objective=True)
+    ctx.zipml_sync()
+    assert (gobj.cpu().numpy().astype(np.uint64) == obj).all()
+    assert (glev.cpu().numpy() == lev).all()
+
+
 # ---------------------------------------------------------------------------------------------
 # SGD: per-step gradient from identical x_t, model after an epoch, both engines, several grids
 # ---------------------------------------------------------------------------------------------
