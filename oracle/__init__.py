@@ -53,7 +53,7 @@ def _declare(L):
     L.orc_quantize_vector.argtypes = [vp, i64, i32, u64, u32, u32, u32, vp, vp]
     L.orc_quantize_vector.restype = None
     L.orc_sgd_epoch.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, i64, f32, i32, i32,
-                                u64, i64, i64, i64, vp, vp]
+                                u64, i64, i64, i64, vp, vp, i32, f32]
     L.orc_estimator_mean.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, i32, vp]
     L.orc_loss_dense.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     L.orc_loss_codes.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -176,8 +176,11 @@ def quantize_vector(v, bits, seed, epoch, step, stream):
     return out, codes
 
 
+REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
+
+
 def sgd_epoch(ds, b, x, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=None,
-              batch_order=None, want_grad=False):
+              batch_order=None, want_grad=False, reg=REG_NONE, reg_param=0.0):
     """Runs steps in place on a copy of x; returns (x_new, grad(2, n) or None)."""
     b = np.ascontiguousarray(b, dtype=np.float32)
     x = np.array(x, dtype=np.float32, copy=True)
@@ -189,7 +192,8 @@ def sgd_epoch(ds, b, x, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, f
     g = np.zeros((2, ds.n), np.float32) if want_grad else None
     _check(lib().orc_sgd_epoch(_p(ds.plane1), _p(ds.plane2), ds.row_bytes, ds.m, ds.n, ds.bits, ds.mode,
                                _p(ds.feat_lo), _p(ds.feat_step), _p(ds.levels), _p(b), _p(x), batch, lr,
-                               model_bits, grad_bits, seed, epoch, first_step, num_steps, _p(batch_order), _p(g)))
+                               model_bits, grad_bits, seed, epoch, first_step, num_steps, _p(batch_order), _p(g),
+                               int(reg), C.c_float(reg_param)))
     return x, g
 
 

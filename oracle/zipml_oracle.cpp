@@ -266,14 +266,40 @@ void orc_quantize_vector(const float* v, int64_t n, int bits, uint64_t seed, uin
 // x <- x - lr * g^ in full precision.  Batch t holds rows [t*batch, min(m, (t+1)*batch)); the
 // steps executed are batch_order[first_step .. first_step+num_steps) (identity order if null).
 // grad_out_or_null (2n): the last executed step's gradient before and after Q4.
+//
+// Regulariser (main text Eq. (proxupdate): x <- prox_{lr R}(x - lr g^), the proximal operator
+// being argmin_z 1/2 ||z - y||^2 + lr R(z)), applied coordinate by coordinate to y = x - lr g^:
+//   reg 0  R = 0                          z = y
+//   reg 1  R = c/2 ||x||_2^2              z = y * shrink,  shrink = fp32(1 / (1 + lr c))
+//   reg 2  R = lambda ||x||_1             z = sign(y) max(|y| - thr, 0),  thr = fp32(lr lambda)
+//   reg 3  R = indicator of x >= 0        z = max(y, 0)
+//   reg 4  least-squares SVM (Supplement "Least Squares Support Vector Machines": the gradient
+//          gains the term c x, kept in full precision):  z = y - fp32(lr c) * x_old
+// The constants are rounded to fp32 once per call and the coordinate arithmetic is fp32 products
+// and differences of fp32 values, evaluated in double and rounded once.
 // ---------------------------------------------------------------------------------------------
+static float orc_regularise(float y, float x_old, int reg, float cst) {
+    if (reg == 1) return (float)((double)y * (double)cst);
+    if (reg == 2) {
+        const float mag = (float)((double)std::fabs(y) - (double)cst);
+        return mag > 0.0f ? (y < 0.0f ? -mag : mag) : 0.0f;
+    }
+    if (reg == 3) return y > 0.0f ? y : 0.0f;
+    if (reg == 4) return (float)((double)y - (double)cst * (double)x_old);
+    return y;
+}
+
 int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_bytes, int64_t m, int64_t n,
                   int bits, int level_mode, const float* feat_lo, const float* feat_step,
                   const float* levels, const float* b, float* x, int64_t batch, float lr,
                   int model_bits, int grad_bits, uint64_t seed, int64_t epoch, int64_t first_step,
-                  int64_t num_steps, const int32_t* batch_order, float* grad_out_or_null) {
+                  int64_t num_steps, const int32_t* batch_order, float* grad_out_or_null, int reg, float reg_param) {
     const int cb = orc_container_bits(bits);
     if (cb == 0) return ORC_ERR_UNSUPPORTED;
+    if (reg < 0 || reg > 4 || (reg != 0 && reg != 3 && !(reg_param >= 0.0f))) return ORC_ERR_INVALID_ARG;
+    float reg_cst = 0.0f;
+    if (reg == 1) reg_cst = (float)(1.0 / (1.0 + (double)lr * (double)reg_param));
+    if (reg == 2 || reg == 4) reg_cst = (float)((double)lr * (double)reg_param);
     if (level_mode == ORC_LEVELS_TABLE && bits == 8) return ORC_ERR_UNSUPPORTED;
     if (model_bits != 0 && (model_bits < 2 || model_bits > 8)) return ORC_ERR_UNSUPPORTED;
     if (grad_bits != 0 && (grad_bits < 2 || grad_bits > 8)) return ORC_ERR_UNSUPPORTED;
@@ -305,7 +331,10 @@ int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byte
             orc_quantize_vector(g.data(), n, grad_bits, seed, (uint32_t)epoch, (uint32_t)it, 4, gq.data(), nullptr);
             gu = gq.data();
         }
-        for (int64_t j = 0; j < n; ++j) x[j] = (float)((double)x[j] - (double)lr * (double)gu[j]);
+        for (int64_t j = 0; j < n; ++j) {
+            const float y = (float)((double)x[j] - (double)lr * (double)gu[j]);
+            x[j] = orc_regularise(y, x[j], reg, reg_cst);
+        }
         if (grad_out_or_null && it == first_step + num_steps - 1) {
             std::memcpy(grad_out_or_null, g.data(), sizeof(float) * (size_t)n);
             std::memcpy(grad_out_or_null + n, gu, sizeof(float) * (size_t)n);

@@ -394,3 +394,102 @@ def test_sgd_reaches_least_squares_solution():
         x, _ = oracle.sgd_epoch(oracle.quantize(A, 4, seed=100 + ep), b, x, batch=16, lr=0.2 / ep, epoch=ep)
     assert np.linalg.norm(x - x_ls) < 0.03 * np.linalg.norm(x_ls)
     assert oracle.loss_dense(A, b, x) < 5 * oracle.loss_dense(A, b, x_ls.astype(np.float32)) + 1e-3
+
+
+# ---------------------------------------------------------------------------------------------
+# Regularisers (Eq. (proxupdate); Supplement "Least Squares Support Vector Machines").  Frozen
+# codes and full batches make the iteration deterministic proximal gradient descent on
+# f(x) = 1/2 x^T H x - c^T x with H, c as in the test above, whose fixed points are known.
+# ---------------------------------------------------------------------------------------------
+def _frozen_quadratic(seed, m=4000, n=8, labels=None):
+    rng = np.random.default_rng(seed)
+    A = rng.uniform(-1, 1, (m, n)).astype(np.float32)
+    xs = rng.standard_normal(n)
+    xs[::3] = 0.0                                       # some coordinates the l1 term can switch off
+    b = (A @ xs + 0.05 * rng.standard_normal(m)).astype(np.float32)
+    if labels == "pm1":
+        b = np.where(A @ xs >= 0, 1.0, -1.0).astype(np.float32)
+    ds = oracle.quantize(A, 4, seed=seed)
+    q1, q2 = np_dequant(ds, 1), np_dequant(ds, 2)
+    H = (q1.T @ q2 + q2.T @ q1) / (2 * m)
+    c = (q1 + q2).T @ b.astype(np.float64) / (2 * m)
+    return ds, b, H, c, m, n
+
+
+def _iterate(ds, b, m, n, steps, lr, **kw):
+    x = np.zeros(n, np.float32)
+    for _ in range(steps):
+        x, _ = oracle.sgd_epoch(ds, b, x, batch=m, lr=lr, **kw)
+    return x.astype(np.float64)
+
+
+def test_one_regularised_step_against_the_operator_written_out():
+    ds, b, H, c, m, n = _frozen_quadratic(21)
+    x0 = (np.random.default_rng(1).standard_normal(n) * 0.3).astype(np.float32)
+    lr = 0.37
+    y, _ = oracle.sgd_epoch(ds, b, x0, batch=m, lr=lr)
+    y = y.astype(np.float64)
+    # prox of lr*c/2*||.||^2, of lr*lam*||.||_1, of the indicator of the non-negative orthant; the SVM term
+    want = {(oracle.REG_L2, 0.8): y / (1 + lr * 0.8),
+            (oracle.REG_L1, 0.5): np.sign(y) * np.maximum(np.abs(y) - lr * 0.5, 0.0),
+            (oracle.REG_NONNEG, 0.0): np.maximum(y, 0.0),
+            (oracle.REG_LSSVM, 0.8): y - lr * 0.8 * x0}
+    for (reg, par), w in want.items():
+        got, _ = oracle.sgd_epoch(ds, b, x0, batch=m, lr=lr, reg=reg, reg_param=par)
+        assert np.allclose(got, w, rtol=1e-6, atol=1e-7), reg
+    # the operator minimises 1/2 ||z - y||^2 + lr R(z): no nearby point does better (l1 case)
+    z, _ = oracle.sgd_epoch(ds, b, x0, batch=m, lr=lr, reg=oracle.REG_L1, reg_param=0.5)
+    obj = lambda v: 0.5 * np.sum((v - y) ** 2) + lr * 0.5 * np.sum(np.abs(v))
+    rng = np.random.default_rng(2)
+    assert all(obj(z.astype(np.float64)) <= obj(z + 1e-3 * rng.standard_normal(n)) + 1e-12 for _ in range(200))
+    # the gradient that is reported is the data term's, with or without a regulariser
+    _, g0 = oracle.sgd_epoch(ds, b, x0, batch=m, lr=lr, want_grad=True)
+    _, g1 = oracle.sgd_epoch(ds, b, x0, batch=m, lr=lr, want_grad=True, reg=oracle.REG_L2, reg_param=0.8)
+    assert (g0[0] == g1[0]).all()
+
+
+def test_l2_and_lssvm_reach_the_ridge_solution():
+    for labels in (None, "pm1"):
+        ds, b, H, c, m, n = _frozen_quadratic(22, labels=labels)
+        cr = 0.3
+        x_ridge = np.linalg.solve(H + cr * np.eye(n), c)            # gradient of f plus cr*x vanishes
+        for reg in (oracle.REG_L2, oracle.REG_LSSVM):
+            x = _iterate(ds, b, m, n, 200, 1.0, reg=reg, reg_param=cr)
+            assert np.linalg.norm(x - x_ridge) < 2e-5 * np.linalg.norm(x_ridge), (labels, reg)
+        # and the regulariser matters: the unregularised fixed point is somewhere else
+        assert np.linalg.norm(np.linalg.solve(H, c) - x_ridge) > 0.05 * np.linalg.norm(x_ridge)
+    # with labels +-1 this is the least-squares SVM problem: 1/(2K) sum (1 - b a^T x)^2 = 1/(2K) sum (a^T x - b)^2
+
+
+def test_l1_fixed_point_satisfies_the_lasso_optimality_conditions():
+    ds, b, H, c, m, n = _frozen_quadratic(23)
+    lam = 0.08
+    x = _iterate(ds, b, m, n, 400, 1.0, reg=oracle.REG_L1, reg_param=lam)
+    grad = H @ x - c
+    on = x != 0.0
+    assert on.any() and (~on).any()                                  # some coordinates survive, some are switched off
+    assert np.allclose(grad[on], -lam * np.sign(x[on]), atol=2e-6)
+    assert (np.abs(grad[~on]) <= lam + 2e-6).all()
+    # a large enough lambda switches everything off, exactly
+    x = _iterate(ds, b, m, n, 3, 1.0, reg=oracle.REG_L1, reg_param=10.0)
+    assert (x == 0.0).all()
+
+
+def test_nonneg_fixed_point_is_the_nonnegative_least_squares_solution():
+    from scipy.optimize import nnls
+    ds, b, H, c, m, n = _frozen_quadratic(24)
+    c = c.copy()
+    # minimise 1/2 x^T H x - c^T x over x >= 0  ==  NNLS with L^T x ~ L^-1 c for H = L L^T
+    Lc = np.linalg.cholesky(H)
+    x_nnls, _ = nnls(Lc.T, np.linalg.solve(Lc, c))
+    x = _iterate(ds, b, m, n, 400, 1.0, reg=oracle.REG_NONNEG)
+    assert (x >= 0).all() and (x_nnls == 0).any()                    # the constraint is active somewhere
+    assert np.linalg.norm(x - x_nnls) < 5e-5 * np.linalg.norm(x_nnls)
+
+
+def test_regulariser_arguments():
+    ds, b, H, c, m, n = _frozen_quadratic(25, m=64)
+    with pytest.raises(Exception):
+        oracle.sgd_epoch(ds, b, np.zeros(n, np.float32), batch=m, lr=0.1, reg=7)
+    with pytest.raises(Exception):
+        oracle.sgd_epoch(ds, b, np.zeros(n, np.float32), batch=m, lr=0.1, reg=oracle.REG_L1, reg_param=-1.0)
