@@ -44,6 +44,17 @@ enum {
 
 enum { ZIPML_LEVELS_UNIFORM = 0, ZIPML_LEVELS_TABLE = 1 };
 enum { ZIPML_LOSS_DENSE = 0, ZIPML_LOSS_CODES = 1 };
+/* Regulariser of zipml_sgd_epoch (paper Eq. (proxupdate): x <- prox_{lr R}(x - lr g), the proximal
+ * operator taken coordinate by coordinate on y = x - lr g; and the Supplement's least-squares SVM,
+ * whose gradient gains the term c x).  reg_param is c or lambda; constants are rounded to fp32 once
+ * per call: shrink = 1 / (1 + lr c), thr = lr lambda, lr c. */
+enum {
+    ZIPML_REG_NONE = 0,     /* R = 0                                  x = y                          */
+    ZIPML_REG_L2 = 1,       /* R = c/2 ||x||^2                        x = y * shrink                 */
+    ZIPML_REG_L1 = 2,       /* R = lambda ||x||_1                     x = sign(y) max(|y| - thr, 0)  */
+    ZIPML_REG_NONNEG = 3,   /* R = indicator of x >= 0                x = max(y, 0)                  */
+    ZIPML_REG_LSSVM = 4     /* least-squares SVM term c x in the gradient:  x = y - (lr c) x_old     */
+};
 /* How zipml_sgd_epoch runs its minibatch chain.  Results do not depend on the choice. */
 enum {
     ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; beyond that
@@ -115,6 +126,8 @@ typedef struct zipml_sgd_params {
                                    passed, 3 residual digits ready, 4 own gradient blocks summed,
                                    5 model updated and digits published, 6 dots and labels read,
                                    7 residual scale known.  Other engines ignore the request.         */
+    int32_t reg;                /* ZIPML_REG_*                                                       */
+    float reg_param;            /* c or lambda (>= 0); ignored by ZIPML_REG_NONE and _NONNEG          */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

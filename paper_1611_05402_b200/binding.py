@@ -13,6 +13,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
+REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM = 0, 1, 2, 3, 4, 5, 6
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
@@ -43,7 +44,7 @@ class CSgdParams(C.Structure):
                 ("batch", C.c_int64), ("epoch", C.c_int64), ("first_step", C.c_int64), ("num_steps", C.c_int64),
                 ("seed", C.c_uint64), ("batch_order", C.c_void_p), ("lr", C.c_float),
                 ("grid_feature_parts", C.c_int32), ("grid_row_parts", C.c_int32), ("trace_steps", C.c_int32),
-                ("trace", C.c_void_p)]
+                ("trace", C.c_void_p), ("reg", C.c_int32), ("reg_param", C.c_float)]
 
 
 _lib = None
@@ -197,12 +198,14 @@ class Context:
         return (lev, obj) if want_objective else lev
 
     def sgd_params(self, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=-1,
-                   batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0, trace=None):
+                   batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0, trace=None,
+                   reg=REG_NONE, reg_param=0.0):
         p = CSgdParams()
         p.struct_size = C.sizeof(CSgdParams)
         p.model_bits, p.grad_bits, p.engine = model_bits, grad_bits, engine
         p.batch, p.epoch, p.first_step, p.num_steps, p.seed, p.lr = batch, epoch, first_step, num_steps, seed, lr
         p.grid_feature_parts, p.grid_row_parts = grid_feature_parts, grid_row_parts
+        p.reg, p.reg_param = reg, reg_param
         if trace is not None:      # (steps, 8) int64 device tensor
             assert trace.dtype == torch.int64 and trace.is_contiguous() and trace.shape[1] == 8
             p.trace, p.trace_steps = trace.data_ptr(), trace.shape[0]

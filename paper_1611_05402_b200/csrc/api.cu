@@ -200,6 +200,8 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
     if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_STREAM) return ZIPML_ERR_INVALID_ARG;
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
+    if (params->reg < ZIPML_REG_NONE || params->reg > ZIPML_REG_LSSVM) return ZIPML_ERR_INVALID_ARG;
+    if (params->reg != ZIPML_REG_NONE && params->reg != ZIPML_REG_NONNEG && !(params->reg_param >= 0.0f)) return ZIPML_ERR_INVALID_ARG;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
     const int64_t count = params->num_steps < 0 ? T - first : params->num_steps;

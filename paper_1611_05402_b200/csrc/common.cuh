@@ -81,6 +81,20 @@ __device__ __forceinline__ void uniform_cell(float v, float lo, float inv, int s
     p = __fsub_rn(t, fl);
 }
 
+// Regulariser applied to y = x - lr g, coordinate by coordinate (paper Eq. (proxupdate); reg 4: the
+// least-squares SVM term of the Supplement).  cst is the per-call constant in fp32: 1/(1 + lr c),
+// lr lambda or lr c.  Every operation is one IEEE fp32 rounding.
+__device__ __forceinline__ float regularise(float y, float x_old, int reg, float cst) {
+    if (reg == ZIPML_REG_L2) return __fmul_rn(y, cst);
+    if (reg == ZIPML_REG_L1) {
+        const float mag = __fsub_rn(fabsf(y), cst);
+        return mag > 0.0f ? copysignf(mag, y) : 0.0f;
+    }
+    if (reg == ZIPML_REG_NONNEG) return y > 0.0f ? y : 0.0f;
+    if (reg == ZIPML_REG_LSSVM) return __fmaf_rn(-cst, x_old, y);
+    return y;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -36,6 +36,13 @@ int cuda_status(cudaError_t e);                       // ZIPML_OK or ZIPML_ERR_C
 int ws_reserve(zipml_ctx* ctx, size_t bytes);         // grow ctx->ws to at least `bytes`
 int stage_reserve(zipml_ctx* ctx, size_t bytes);
 
+// The fp32 constant of zipml_sgd_params' regulariser for step length lr (see regularise() in common.cuh).
+inline float reg_constant(const zipml_sgd_params* p) {
+    if (p->reg == ZIPML_REG_L2) return (float)(1.0 / (1.0 + (double)p->lr * (double)p->reg_param));
+    if (p->reg == ZIPML_REG_L1 || p->reg == ZIPML_REG_LSSVM) return (float)((double)p->lr * (double)p->reg_param);
+    return 0.0f;
+}
+
 // Simple bump carving of the workspace: 256-byte aligned pieces.
 struct Carver {
     unsigned char* base;

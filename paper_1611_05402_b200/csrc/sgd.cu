@@ -464,7 +464,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_kernel(const SgdArgs a) {
                 float g = gs[f];
                 if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
                 if (last && a.grad_out && bi == 0) a.grad_out[a.n + j0 + f] = g;
-                xs[f] = fmaf(-a.lr, g, xs[f]);
+                xs[f] = regularise(fmaf(-a.lr, g, xs[f]), xs[f], a.reg, a.reg_cst);
             }
             __syncthreads();
             if (!a.persistent && bi == 0)
@@ -627,7 +627,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
     a.b = b; a.x = x; a.grad_out = grad_out;
     a.batch = p->batch < d->m ? p->batch : d->m;
     a.first_step = first_step; a.num_steps = num_steps;
-    a.lr = p->lr; a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
+    a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
     a.seed = p->seed; a.epoch = (uint32_t)p->epoch;
     a.na = plan.na; a.nb = plan.nb; a.wc = plan.wc; a.rc = plan.rc; a.stages = plan.stages;
     a.pd = reinterpret_cast<double*>(ctx->ws + sc.pd_off);

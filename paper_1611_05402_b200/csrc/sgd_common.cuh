@@ -30,6 +30,8 @@ struct SgdArgs {
     int64_t batch, first_step, num_steps;
     const int32_t* order;   // device copy of the batch order, or null
     float lr;
+    int reg;                // ZIPML_REG_* and its fp32 constant
+    float reg_cst;
     int model_bits, grad_bits;
     uint64_t seed;
     uint32_t epoch;

@@ -60,6 +60,8 @@ struct LeanArgs {
     uint64_t seed;
     uint32_t epoch;
     float lr;
+    int reg;                     // ZIPML_REG_* and its fp32 constant
+    float reg_cst;
     int n, bits, row_words, words;   // words = ceil(n / codes per word) <= row_words
     int model_bits, grad_bits;
     int nb, rc, slots;
@@ -392,7 +394,7 @@ __global__ void __launch_bounds__(kLeanThreads, 1) sgd_lean_kernel(const LeanArg
                     if (a.grad_bits > 0)
                         g = lean_quant(g, gq_M, (1 << (a.grad_bits - 1)) - 1, a.seed, a.epoch, (uint32_t)it, 4u, (uint32_t)f);
                     if (last && a.grad_out) a.grad_out[n + f] = g;
-                    xown[k] = fmaf(-a.lr, g, xown[k]);
+                    xown[k] = regularise(fmaf(-a.lr, g, xown[k]), xown[k], a.reg, a.reg_cst);
                 }
             }
         }
@@ -557,7 +559,7 @@ int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.trace_steps = p->trace ? p->trace_steps : 0;
     a.status = ctx->d_status;
     a.m = d->m; a.batch = p->batch < d->m ? p->batch : d->m;
-    a.seed = p->seed; a.epoch = (uint32_t)p->epoch; a.lr = p->lr;
+    a.seed = p->seed; a.epoch = (uint32_t)p->epoch; a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p);
     a.n = (int)d->n; a.bits = d->bits; a.row_words = (int)(d->row_bytes / 4);
     a.words = (int)((d->n + fpw - 1) / fpw);
     a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;

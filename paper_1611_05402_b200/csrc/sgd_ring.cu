@@ -971,7 +971,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                     float g = gsub[k];
                     if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
                     if (last && a.grad_out) a.grad_out[a.n + j0 + f] = g;
-                    xn = fmaf(-a.lr, g, xown[k]);
+                    xn = regularise(fmaf(-a.lr, g, xown[k]), xown[k], a.reg, a.reg_cst);
                 }
                 xown[k] = xn;
                 xsq += (double)xn * (double)xn;
@@ -1229,7 +1229,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.b = b; a.x = x; a.grad_out = grad_out;
     a.batch = B;
     a.first_step = first_step; a.num_steps = num_steps;
-    a.lr = p->lr; a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
+    a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
     a.seed = p->seed; a.epoch = (uint32_t)p->epoch;
     a.na = plan.na; a.nb = plan.nb; a.wc = plan.wc; a.rc = plan.rc; a.stages = plan.slots;
     a.cr = plan.cr; a.sub = plan.sub; a.pitch = plan.pitch;

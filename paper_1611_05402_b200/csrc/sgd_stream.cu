@@ -60,6 +60,8 @@ struct StreamArgs {
     int64_t batch, first_step, num_steps;
     const int32_t* order;
     float lr;
+    int reg;                 // ZIPML_REG_* and its fp32 constant
+    float reg_cst;
     int ca;                  // pass A: column parts of the row
     int spans;               // 64-byte spans of a row = pass B's column blocks
     int part_spans;          // most spans a part holds
@@ -411,7 +413,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             block_reduce_mms(u1, u2, rsum, shf, shd);      // its barriers publish rdig and the cleared sums
         }
         // scale of the next model's digits: a bound that writers and readers both know now
-        const float bound_next = (wm + fabsf(a.lr) * cmax * rmax) * 1.0001f;
+        // (the regularisers only pull towards zero, except the least-squares SVM term with lr c > 2)
+        const float grow = a.reg == ZIPML_REG_LSSVM ? fmaxf(1.0f, fabsf(1.0f - a.reg_cst)) : 1.0f;
+        const float bound_next = (wm * grow + fabsf(a.lr) * cmax * rmax) * 1.0001f;
         stream_mark(a, t_rel, 3);
 
         // ------------------------------------------------------------------ pass B: gradient of the own blocks
@@ -552,7 +556,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                     const float l = lo_o[idx], st = st_o[idx];
                     const float g = (float)(((double)l * lo_term + (double)st * (delta_r * (double)Sj)) * scale);
                     if (last && a.grad_out) { a.grad_out[j] = g; a.grad_out[n + j] = g; }
-                    const float xn = fmaf(-a.lr, g, x_o[idx]);
+                    const float xn = regularise(fmaf(-a.lr, g, x_o[idx]), x_o[idx], a.reg, a.reg_cst);
                     x_o[idx] = xn;
                     a.x[j] = xn;
                     const float w = st * xn;
@@ -664,7 +668,7 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     memset(&a, 0, sizeof(a));
     a.p1 = d->plane1; a.p2 = d->plane2; a.row_bytes = rb; a.m = d->m; a.n = (int)d->n; a.bits = d->bits;
     a.lo = d->feat_lo; a.step = d->feat_step; a.b = b; a.x = x; a.grad_out = grad_out;
-    a.batch = B; a.lr = p->lr;
+    a.batch = B; a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p);
     a.ca = (int)ca; a.spans = (int)spans; a.part_spans = part_spans; a.bpc = (int)bpc; a.bpad = bpad;
     a.union_bytes = (int)uni; a.vec_bytes = vec_bytes;
     // The whole next tile where two tiles fit L2 with room to spare, a quarter of it where one and a half do

@@ -337,6 +337,45 @@ def test_sgd_end_to_end_quantization(ctx, model_bits, grad_bits):
     assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
 
 
+REGS = [(binding.REG_L2, 0.5), (binding.REG_L1, 0.02), (binding.REG_NONNEG, 0.0), (binding.REG_LSSVM, 0.5)]
+
+
+@pytest.mark.parametrize("reg,param", REGS)
+@pytest.mark.parametrize("case", [SGD_CASES[1], SGD_CASES[2], SGD_CASES[4]], ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
+def test_sgd_regularised_update_parity(ctx, case, reg, param):
+    """Every engine applies the regulariser of Eq. (proxupdate) / the least-squares SVM term as the oracle does."""
+    key, m, n, bits, batch, lr = case
+    _, A, b, _ = workload(key, m, n, seed=5)
+    ods = oracle.quantize(A, bits, seed=6)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = (np.random.default_rng(7).standard_normal(n) * 0.1).astype(np.float32)
+    lr = lr * 5
+    if reg == binding.REG_L1:
+        param = 0.05 / (lr * ((m + batch - 1) // batch))            # thresholds of an epoch add up to 0.05
+    x_ref, g_ref = oracle.sgd_epoch(ods, b, x0, batch, lr, reg=reg, reg_param=param, want_grad=True)
+    if reg == binding.REG_L1:
+        assert (x_ref == 0).any() and (x_ref != 0).any()            # the threshold bites somewhere, not everywhere
+    if reg == binding.REG_NONNEG:
+        assert (x_ref >= 0).all() and ((x_ref == 0).any() or key == "c5")  # (c5's large first gradients lift every coordinate)
+    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER,
+                   binding.ENGINE_STREAM, binding.ENGINE_AUTO):
+        x = to_dev(x0, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=engine, reg=reg, reg_param=param, grad_out=g)
+        ctx.zipml_sync()
+        got = x.cpu().numpy()
+        assert rel(got, x_ref) <= MODEL_TOL, engine
+        if reg in (binding.REG_L1, binding.REG_NONNEG):
+            # the switched-off coordinates agree except where y sits within rounding of the threshold
+            assert ((got == 0) != (x_ref == 0)).sum() <= max(1, n // 200), engine
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, reg=9)
+    assert e.value.code == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, reg=binding.REG_L2, reg_param=-0.1)
+    assert e.value.code == binding.ERR_INVALID_ARG
+
+
 def test_sgd_split_calls_equal_one_call(ctx):
     _, A, b, _ = workload("c1", 640, 64, seed=9)
     ods = oracle.quantize(A, 4, seed=1)
