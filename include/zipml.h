@@ -111,7 +111,8 @@ typedef struct zipml_sgd_params {
     const int32_t* batch_order; /* HOST pointer or NULL: T = ceil(m/B) batch indices; NULL = 0..T-1  */
     float lr;                   /* step length gamma, constant within the call                       */
     int32_t grid_feature_parts; /* tuning, 0 = automatic: CTAs along the features                    */
-    int32_t grid_row_parts;     /* tuning, 0 = automatic: CTAs along the rows of a minibatch         */
+    int32_t grid_row_parts;     /* tuning, 0 = automatic: CTAs along the rows of a minibatch (stream
+                                   engine: an upper limit on its CTAs, ignored where too few)        */
     int32_t trace_steps;        /* profiling: number of steps to trace (0 = none)                    */
     uint64_t* trace;            /* profiling, DEVICE pointer or NULL: 8 uint64 per traced step; CTA 0
                                    stores its SM's cycle counter at the step's phase boundaries
