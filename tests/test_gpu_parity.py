@@ -337,6 +337,28 @@ def test_sgd_end_to_end_quantization(ctx, model_bits, grad_bits):
     assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
 
 
+def test_auto_picks_the_engine_that_fits(ctx):
+    """AUTO: cluster for small steps, stream for large uniform fp32 steps on wide rows, ring where stream declines."""
+    _, A, b, _ = workload("c5", 700, 20000, seed=2)                 # 2 x 300 rows x 10 KB: 6 MB per step, 157 column blocks
+    ods = oracle.quantize(A, 4, seed=2)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = np.zeros(20000, np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 300, 1e-4)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 300, 1e-4)
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() == binding.ENGINE_STREAM and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 300, 1e-4, grad_bits=8, seed=3)          # quantized gradient: not the stream engine's
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() == binding.ENGINE_RING
+    _, A, b, _ = workload("c2", 600, 1000, seed=2)
+    gds, db = dev_dataset(oracle.quantize(A, 8, seed=2), ctx), to_dev(b, ctx)
+    ctx.zipml_sgd_epoch(gds, db, torch.zeros(1000, device=ctx.device), 64, 1e-3)     # 0.13 MB per step
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() == binding.ENGINE_CLUSTER
+
+
 REGS = [(binding.REG_L2, 0.5), (binding.REG_L1, 0.02), (binding.REG_NONNEG, 0.0), (binding.REG_LSSVM, 0.5)]
 
 
