@@ -103,6 +103,19 @@ __device__ __forceinline__ uint64_t l2_evict_first_policy() {
 __device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, uint64_t policy) {
     asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
 }
+__device__ __forceinline__ uint64_t l2_evict_normal_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// The same copy under a predicate (no branch around it): nothing is copied where `on` is false.
+__device__ __forceinline__ void cp_async16_if(bool on, uint32_t dst, const void* src, uint64_t policy) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %0, 0;\n\t"
+        "@p cp.async.cg.shared.global.L2::cache_hint [%1], [%2], 16, %3;\n\t}"
+        ::"r"((int)on), "r"(dst), "l"(src), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
@@ -236,12 +249,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                 const uint32_t off_a = (uint32_t)(rblk * 16 + gl) * (uint32_t)rb + 16 * tl, off_h = off_a + 8 * (uint32_t)rb;
                 const int sp_end = min(s1, (int)((rb - 16 * tl + 63) / 64));      // spans whose 16 bytes of this lane lie in the row
                 const uint32_t stage0 = ring_w + lane * 16;
+                const uint64_t keep = l2_evict_normal_policy();
                 auto issue = [&](int sp) {
                     if (sp < sp_end) {
                         const uint32_t dst = stage0 + (uint32_t)((sp - s0) & (S - 1)) * kStreamStageBytes;
                         const uint32_t o = (uint32_t)sp * 64;
-                        if (ok_a) { cp_async16(dst, t1 + (off_a + o)); cp_async16(dst + 1024, t2 + (off_a + o)); }
-                        if (ok_h) { cp_async16(dst + 512, t1 + (off_h + o)); cp_async16(dst + 1536, t2 + (off_h + o)); }
+                        cp_async16_if(ok_a, dst, t1 + (off_a + o), keep);
+                        cp_async16_if(ok_a, dst + 1024, t2 + (off_a + o), keep);
+                        cp_async16_if(ok_h, dst + 512, t1 + (off_h + o), keep);
+                        cp_async16_if(ok_h, dst + 1536, t2 + (off_h + o), keep);
                     }
                     cp_async_commit();
                 };
@@ -433,6 +449,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
             const uint32_t rb32 = (uint32_t)rb;
             const uint32_t stage0 = ring_w + lane * 16;
             const uint64_t dead = l2_evict_first_policy();    // the tile is not read again: its lines may leave L2 first
+            const uint64_t keep = l2_evict_normal_policy();
             int i_ci = 0, i_rem = 0;                       // issue side: column block and position within it
             auto issue = [&]() {
                 if (i_ci < cb1 - cb0) {
@@ -444,13 +461,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                         const uint32_t o = (uint32_t)r0 * rb32;
                         // A 128-byte line holds two column blocks.  Once this CTA has read both, nobody reads the
                         // line again this step: only then may it leave L2 ahead of the rest.
-                        const bool second = i_ci > 0 && ((cb0 + i_ci) & 1);
+                        const uint64_t pol = (i_ci > 0 && ((cb0 + i_ci) & 1)) ? dead : keep;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            if (r0 + 8 * k < bt) {
-                                if (second) cp_async16_hint(dst + k * 512, tp + (o + 8 * k * rb32), dead);
-                                else cp_async16(dst + k * 512, tp + (o + 8 * k * rb32));
-                            }
+                        for (int k = 0; k < 4; ++k) cp_async16_if(r0 + 8 * k < bt, dst + k * 512, tp + (o + 8 * k * rb32), pol);
                     }
                     if (++i_rem == per_c) { i_rem = 0; ++i_ci; }
                 }
@@ -498,8 +511,10 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                     else { transpose4x4(lo4[0].y, lo4[1].y, lo4[2].y, lo4[3].y, ta); transpose4x4(hi4[0].y, hi4[1].y, hi4[2].y, hi4[3].y, th); }
 #pragma unroll
                     for (int g = 0; g < NG; ++g) {
-                        constexpr uint32_t kLow = CB == 8 ? 0xFFFFFFFFu : CB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
-                        const uint32_t mk = kLow << (g * CB);      // codes stay in place: sums 2^(g CB) times too large
+                        // Both groups of a byte meet the same residual digits, so the sums may nest: accumulator g
+                        // takes the byte with the groups below g cleared (g = 0: the byte as it is, no mask at
+                        // all), i.e. sum_{h >= g} 2^(h CB) code_h; group g is the difference of two neighbours.
+                        const uint32_t mk = 0x01010101u * (uint32_t)((0xFFu << (g * CB)) & 0xFFu);
 #pragma unroll
                         for (int u = 0; u < 2; ++u)
                             mma_u8s8(acc[g][w][u], ta[2 * u] & mk, ta[2 * u + 1] & mk, th[2 * u] & mk, th[2 * u + 1] & mk, b0, b1);
@@ -518,14 +533,22 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                                 if (tl < 2) {
                                     const int e = e0 + (g * CW + gl * 8 + 4 * w + 2 * u) * NS + 2 * tl;
                                     int* p = gacc + e + (e >> 5);
-                                    atomicAdd(p, acc[g][w][u][0] >> (g * CB));
-                                    atomicAdd(p + 1, acc[g][w][u][1] >> (g * CB));
-                                    atomicAdd(p + NS, acc[g][w][u][2] >> (g * CB));
-                                    atomicAdd(p + NS + 1, acc[g][w][u][3] >> (g * CB));
+                                    // (exact: the difference is 2^(g CB) times the group's sum)
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q) {
+                                        const int above = g + 1 < NG ? acc[g + 1 < NG ? g + 1 : g][w][u][q] : 0;
+                                        atomicAdd(p + (q >> 1) * NS + (q & 1), (acc[g][w][u][q] - above) >> (g * CB));
+                                    }
                                 }
+                            }
+#pragma unroll
+                    for (int g = 0; g < NG; ++g)
+#pragma unroll
+                        for (int w = 0; w < 2; ++w)
+#pragma unroll
+                            for (int u = 0; u < 2; ++u)
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) acc[g][w][u][e] = 0;
-                            }
                     rem = 0;
                     ++ci;
                 }
