@@ -686,9 +686,13 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
         double bpart = 0.0;
         float wm = 0.0f;
 #pragma unroll 1
-        for (int f = tid; f < Fp; f += kCluThreads) {
+        for (int idx = tid; idx < Fp; idx += kCluThreads) {
+            // level tables: consecutive threads take consecutive word columns of one feature slot, so that the L
+            // table rows they read and write are contiguous (feature-major threads hit one bank eight times when
+            // the row has a multiple of 32 words: 2 k cycles per step on 64-word rows)
+            const int q = TABLE ? idx % rw : idx >> LOGF, i = TABLE ? idx / rw : idx & (FPW - 1);
+            const int f = TABLE ? q * FPW + i : idx;
             const float xt = (f < n) ? xs[f] : 0.0f;
-            const int q = f >> LOGF, i = f & (FPW - 1);
             if constexpr (IMMA) {
                 const float w = steps[f] * xt;
                 wv[f] = w;
