@@ -6,8 +6,8 @@
 // 1/(2B) sum_k [q1_k r2_k + q2_k r1_k] (pass B), with r = dot - b between them.  Both passes feed the
 // int8 tensor cores with code bytes exactly as they lie in memory: pass A streams the tile from HBM
 // and leaves it in L2, pass B re-reads it from L2.  Every warp moves its own bytes through a private
-// ring of shared-memory stages with cp.async (each lane reads back only what it copied itself, so
-// the ring needs no barrier), several stages ahead of the arithmetic.
+// ring of shared-memory stages with cp.async, several stages ahead of the arithmetic (in pass A a
+// lane reads back only what it copied itself: no barrier; in pass B one __syncwarp per stage).
 //
 //   pass A   a CTA takes one column part of the row (a run of 64-byte spans) for 256 rows, a warp 16
 //            of them; the part's digits of w = step * x (four balanced base-128 int8 digits) are
@@ -19,8 +19,9 @@
 //            (shared memory), redundantly and identically.
 //   pass B   a CTA owns whole column blocks (64 bytes of the row = 512 / CB features) for all rows
 //            of the step, so its gradient entries never leave it.  The contraction runs over rows:
-//            a lane copies 8 bytes of 8 rows, transposes 4 x 4 byte blocks with byte permutes and
-//            feeds (features x rows) fragments; the residual digits are the B operand.
+//            a stage holds 32 rows x 64 bytes; a lane takes 8 bytes of 8 of them, transposes 4 x 4 byte
+//            blocks with byte permutes and feeds (features x rows) fragments; the residual digits are
+//            the B operand.
 //   update   the owner updates its features of x (kept in shared memory for the whole launch), turns
 //            w = step * x into digits for the next step and raises a per-block flag; pass A of the
 //            next step waits only for the flags of the blocks it reads (no second grid barrier).
@@ -42,7 +43,7 @@ constexpr int kStreamWarps = kStreamThreads / 32;
 constexpr int kStreamMaxBatch = 8192;      // residual digits of a step live in shared memory
 constexpr int kStreamMaxOwn = 4;           // column blocks per CTA
 constexpr int kStreamStages = 4;           // ring stages per warp
-constexpr int kStreamStageBytes = 2048;    // pass A: 4 x 32 lanes x 16 B; pass B: 8 x 32 lanes x 8 B
+constexpr int kStreamStageBytes = 2048;    // pass A: 4 x 32 lanes x 16 B; pass B: 32 rows x 64 B
 constexpr int kStreamRingBytes = kStreamWarps * kStreamStages * kStreamStageBytes;
 constexpr int kStreamBlock = 64;           // bytes of a column block = one span
 constexpr int kStreamMaxPartSpans = 64;    // spans of a pass-A column part
@@ -100,27 +101,19 @@ __device__ __forceinline__ uint64_t l2_evict_first_policy() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
-__device__ __forceinline__ void cp_async16_hint(uint32_t dst, const void* src, uint64_t policy) {
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
-}
 __device__ __forceinline__ uint64_t l2_evict_normal_policy() {
     uint64_t pol;
     asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
-// The same copy under a predicate (no branch around it): nothing is copied where `on` is false.
+// 16-byte global -> shared copy with an L2 policy, under a predicate (no branch around it): nothing is
+// copied where `on` is false.
 __device__ __forceinline__ void cp_async16_if(bool on, uint32_t dst, const void* src, uint64_t policy) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %0, 0;\n\t"
         "@p cp.async.cg.shared.global.L2::cache_hint [%1], [%2], 16, %3;\n\t}"
         ::"r"((int)on), "r"(dst), "l"(src), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
