@@ -57,8 +57,9 @@ enum {
 };
 /* How zipml_sgd_epoch runs its minibatch chain.  Results do not depend on the choice. */
 enum {
-    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; beyond that
-                                   stream where it applies, else ring                                 */
+    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; else stream
+                                   where it applies (wide rows, uniform grid, fp32 model and gradient),
+                                   else ring                                                          */
     ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
     ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
     ZIPML_ENGINE_RING = 3,       /* one cooperative launch; producer warp streams code chunks through a

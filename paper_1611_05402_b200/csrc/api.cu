@@ -228,10 +228,9 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
             rc = launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
             if (rc != ZIPML_ERR_WORKSPACE) return rc;
         }
-        else {
-            rc = launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, true);
-            if (rc != ZIPML_ERR_WORKSPACE) return rc;
-        }
+        // (also for small steps on rows too wide for the two above)
+        rc = launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, true);
+        if (rc != ZIPML_ERR_WORKSPACE) return rc;
         rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
         if (rc != ZIPML_ERR_WORKSPACE) return rc;
     }
