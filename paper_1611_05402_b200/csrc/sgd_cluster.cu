@@ -402,7 +402,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
 #pragma unroll
                 for (int w = 0; w < kCluWarps; ++w) { S += sh->ssum[w]; rho = fmaxf(rho, sh->fmax[w]); }
                 const float inv_r = rho > 0.0f ? QMAXF / rho : 0.0f;
-                const double delta_r = (double)rho / (double)QMAXF;
+                const float delta_rf = (float)((double)rho / (double)QMAXF), Sf = (float)S;
                 // digits of the residuals as B operands of phase B: per 32 rows and residual, per digit, 32 bytes
                 // in the row order the transposed code fragments come in (k = 16h + 4t + e <-> row 16h + 2t +
                 // (e & 1) + 8 (e >> 1)); rows past the CTA's last one count as zero
@@ -472,12 +472,14 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                         for (int g = 0; g < NG; ++g) {
 #pragma unroll
                             for (int odd = 0; odd < 2; ++odd) {
-                                const double pair = (double)acc[ti][g][2 * odd] + 128.0 * (double)acc[ti][g][2 * odd + 1];
-                                const double upper = __shfl_down_sync(0xffffffffu, pair, 1);
+                                // (the digit sums meet in 64-bit integers and are converted once: conversions to and
+                                // from double run at a sixteenth of the FMA rate and made up most of this epilogue)
+                                const long long pair = (long long)acc[ti][g][2 * odd] + 128ll * (long long)acc[ti][g][2 * odd + 1];
+                                const long long upper = __shfl_down_sync(0xffffffffu, pair, 1);
                                 const int byte_in_row = col * 16 + 2 * gl + odd;
                                 const int f = (byte_in_row >> 2) * FPW + (byte_in_row & 3) * NG + g;
                                 if (tl == 0 && f < n)
-                                    gpart[f] = (float)((double)los[f] * S + (double)steps[f] * ((pair + 16384.0 * upper) * delta_r));
+                                    gpart[f] = fmaf(steps[f], (float)(pair + 16384ll * upper) * delta_rf, los[f] * Sf);
                             }
                         }
                     }
@@ -539,6 +541,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
 #pragma unroll
                     for (int w = 0; w < kCluWarps; ++w) S += sh->ssum[w];
                 }
+                const float Sf = (float)S;
 #pragma unroll 1
                 for (int q0 = 0; q0 < nw; q0 += lanes_q) {
                     const int q = q0 + ql;
@@ -581,7 +584,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                         if (f < n) {
                             float v = gred[fl];
                             for (int g = 1; g < ngroups; ++g) v += gred[g * lanes_q * FPW + fl];
-                            if constexpr (!TABLE) v = (float)((double)los[f] * S + (double)steps[f] * (double)v);
+                            if constexpr (!TABLE) v = fmaf(steps[f], v, los[f] * Sf);      // (fp32: conversions are slow)
                             gpart[f] = v;
                         }
                     }
