@@ -110,6 +110,16 @@ __device__ __forceinline__ void cluster_sync_all() {
 // Bounded wait on a local mbarrier phase; after the first failure of this CTA every wait is skipped.
 __device__ __forceinline__ void clu_wait(unsigned long long* bar, uint32_t parity, ClusterShared* sh, DeviceStatus* status, int where) {
     if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) return;
+    // (a phase that is complete already -- a tile copied steps ahead -- answers the non-blocking test at once)
+    {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        if (done) return;
+    }
 #pragma unroll 1
     for (long long spin = 0; spin < kCopySpinLimit; ++spin)
         if (mbar_try_wait(reinterpret_cast<uint64_t*>(bar), parity)) return;
