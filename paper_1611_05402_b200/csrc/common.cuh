@@ -64,20 +64,25 @@ __device__ __forceinline__ uint32_t vector_u24(uint64_t seed, uint32_t epoch, ui
     return b.v[coord & 3u] >> 8;
 }
 
-// up <=> u24 * 2^-24 < p, both sides fp32 (the product is exact).
-__device__ __forceinline__ uint32_t round_up_if(uint32_t cell, float p, uint32_t word) {
-    const float u = __fmul_rn((float)(word >> 8), 5.9604644775390625e-08f);
-    return cell + (u < p ? 1u : 0u);
+// up <=> u24 * 2^-24 < p, both sides fp32 (the product is exact).  Since u24 is an integer below 2^24 and
+// p * 2^24 is exact in fp32, that is u24 < ceil(p * 2^24): the threshold is computed once per element (one
+// conversion; int <-> float conversions issue at a sixteenth of the FMA rate) and compared as integers for
+// both copies.  p <= 0 or NaN gives 0 (never up), p >= 1 gives at least 2^24 (always up).
+__device__ __forceinline__ uint32_t up_threshold(float p) { return __float2uint_ru(__fmul_rn(p, 16777216.0f)); }
+__device__ __forceinline__ uint32_t round_up_if(uint32_t cell, uint32_t threshold, uint32_t word) {
+    return cell + ((word >> 8) < threshold ? 1u : 0u);
 }
 
-// Cell and up-probability on a uniform grid of s intervals: t = (v - lo) * inv with every
-// operation rounded on its own (no contraction into an FMA).
+// Cell and up-probability on a uniform grid of s intervals (s < 2^22): t = (v - lo) * inv with every
+// operation rounded on its own (no contraction into an FMA), cell = clamp(floor t, 0, s-1), p = t - cell.
+// The floor needs no conversion instruction: 2^23 + t' rounded down keeps floor(t') in its mantissa.
+// A NaN lands in cell 0 with p = NaN (never up); -inf in cell 0, +inf in the last cell, always up.
 __device__ __forceinline__ void uniform_cell(float v, float lo, float inv, int s, uint32_t& cell, float& p) {
     const float t = __fmul_rn(__fsub_rn(v, lo), inv);
-    float fl = floorf(t);
-    fl = fl < 0.0f ? 0.0f : fl;                    // a NaN falls through both comparisons ...
-    fl = fl > (float)(s - 1) ? (float)(s - 1) : fl;
-    cell = (fl == fl) ? (uint32_t)fl : 0u;         // ... and lands in cell 0
+    const float tc = fmaxf(t, 0.0f);                                        // NaN -> 0
+    float fl = __fsub_rn(__fadd_rd(tc, 8388608.0f), 8388608.0f);            // floor(tc), exact for tc < 2^23
+    fl = fminf(fl, (float)(s - 1));
+    cell = __float_as_uint(__fadd_rn(fl, 8388608.0f)) & 0x7FFFFFu;
     p = __fsub_rn(t, fl);
 }
 

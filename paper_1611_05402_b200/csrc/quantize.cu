@@ -216,8 +216,9 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                 for (int h = 0; h < 2; ++h) {
                     const int i = 2 * pr + h;
                     if (i >= nf) break;
-                    w1 |= round_up_if(cell[h], p[h], rnd.v[2 * h]) << (i * CB);
-                    w2 |= round_up_if(cell[h], p[h], rnd.v[2 * h + 1]) << (i * CB);
+                    const uint32_t thr = up_threshold(p[h]);
+                    w1 |= round_up_if(cell[h], thr, rnd.v[2 * h]) << (i * CB);
+                    w2 |= round_up_if(cell[h], thr, rnd.v[2 * h + 1]) << (i * CB);
                 }
             }
         }
