@@ -186,17 +186,18 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
 #pragma unroll
                 for (int i = 0; i < FPW; ++i) v[i] = (i < nf) ? __ldg(src + i) : 0.0f;
             }
-#pragma unroll
-            for (int pr = 0; pr < FPW / 2; ++pr) {
-                if (2 * pr >= nf) break;
-                uint32_t cell[2] = {0u, 0u};
-                float p[2] = {0.0f, 0.0f};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int i = 2 * pr + h;
-                    if (i >= nf) break;
+            if constexpr (FPW <= 8) {
+                // pass 1: cells and thresholds of all features; a threshold strictly between 0 and 2^24 needs a draw
+                uint32_t thr[FPW];
+                uint32_t need = 0u;                                     // pairs with at least one such feature
+    #pragma unroll
+                for (int i = 0; i < FPW; ++i) {
+                    thr[i] = 0u;
+                    if (i >= nf) continue;
+                    uint32_t cell;
+                    float p;
                     if constexpr (!TABLE) {
-                        uniform_cell(v[i], flo[i], finv[i], s, cell[h], p[h]);
+                        uniform_cell(v[i], flo[i], finv[i], s, cell, p);
                     } else {
                         const float* lev = lev_s + i * blockDim.x + threadIdx.x;       // level k at lev[k * FPW * blockDim.x]
                         const int ls = FPW * blockDim.x;
@@ -204,21 +205,79 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                         for (int k = 1; k <= s - 1; ++k) l = (lev[k * ls] <= v[i]) ? k : l;
                         const float base = lev[l * ls];
                         const float width = __fsub_rn(lev[(l + 1) * ls], base);
-                        cell[h] = (uint32_t)l;
-                        p[h] = width > 0.0f ? __fdiv_rn(__fsub_rn(v[i], base), width) : 0.0f;
+                        cell = (uint32_t)l;
+                        p = width > 0.0f ? __fdiv_rn(__fsub_rn(v[i], base), width) : 0.0f;
+                    }
+                    const uint32_t t = up_threshold(p);
+                    const bool open = t > 0u && t < 16777216u;
+                    // decided without a draw: threshold 0 never up, 2^24 and more always up
+                    const uint32_t c = cell + (t >= 16777216u ? 1u : 0u);
+                    w1 |= c << (i * CB);
+                    w2 |= c << (i * CB);
+                    thr[i] = open ? t : 0u;                             // 0: this feature adds nothing in pass 2
+                    need |= open ? 1u << (i >> 1) : 0u;
+                }
+                // pass 2: one Philox block per pair that needs one.  Where every lane needs every pair (dense continuous
+                // data) the pairs run as independent unrolled chains; otherwise every lane walks its own short list, so
+                // a warp runs as many rounds as its busiest lane has pairs (sparse rows: about two of four).
+                auto apply = [&](int pr, const Philox4& rnd) {
+    #pragma unroll
+                    for (int i = 0; i < FPW / 2; ++i)
+                        if (i == pr) {
+                            w1 += ((rnd.v[0] >> 8) < thr[2 * i] ? 1u : 0u) << (2 * i * CB);
+                            w2 += ((rnd.v[1] >> 8) < thr[2 * i] ? 1u : 0u) << (2 * i * CB);
+                            w1 += ((rnd.v[2] >> 8) < thr[2 * i + 1] ? 1u : 0u) << ((2 * i + 1) * CB);
+                            w2 += ((rnd.v[3] >> 8) < thr[2 * i + 1] ? 1u : 0u) << ((2 * i + 1) * CB);
+                        }
+                };
+                constexpr uint32_t kAllPairs = (1u << (FPW / 2)) - 1u;
+                if (__all_sync(__activemask(), need == kAllPairs)) {
+    #pragma unroll
+                    for (int pr = 0; pr < FPW / 2; ++pr) apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr)));
+                } else {
+                    while (need) {
+                        const int pr = __ffs(need) - 1;
+                        need &= need - 1u;
+                        apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr)));
                     }
                 }
-                const bool random = (p[0] > 0.0f && p[0] < 1.0f) || (p[1] > 0.0f && p[1] < 1.0f);
-                Philox4 rnd;
-                if (random) rnd = sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr));
-                else rnd.v[0] = rnd.v[1] = rnd.v[2] = rnd.v[3] = 0u;    // decided without them: p <= 0 never up, p >= 1 always up
+        
+            } else {
+                // sixteen features per word: the thresholds of a whole word would not fit the registers; pair by pair
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int i = 2 * pr + h;
-                    if (i >= nf) break;
-                    const uint32_t thr = up_threshold(p[h]);
-                    w1 |= round_up_if(cell[h], thr, rnd.v[2 * h]) << (i * CB);
-                    w2 |= round_up_if(cell[h], thr, rnd.v[2 * h + 1]) << (i * CB);
+                for (int pr = 0; pr < FPW / 2; ++pr) {
+                    if (2 * pr >= nf) break;
+                    uint32_t cell[2] = {0u, 0u}, t[2] = {0u, 0u};
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int i = 2 * pr + h;
+                        if (i >= nf) break;
+                        float p;
+                        if constexpr (!TABLE) {
+                            uniform_cell(v[i], flo[i], finv[i], s, cell[h], p);
+                        } else {
+                            const float* lev = lev_s + i * blockDim.x + threadIdx.x;
+                            const int ls = FPW * blockDim.x;
+                            int l = 0;
+                            for (int k = 1; k <= s - 1; ++k) l = (lev[k * ls] <= v[i]) ? k : l;
+                            const float base = lev[l * ls];
+                            const float width = __fsub_rn(lev[(l + 1) * ls], base);
+                            cell[h] = (uint32_t)l;
+                            p = width > 0.0f ? __fdiv_rn(__fsub_rn(v[i], base), width) : 0.0f;
+                        }
+                        t[h] = up_threshold(p);
+                    }
+                    const bool random = (t[0] > 0u && t[0] < 16777216u) || (t[1] > 0u && t[1] < 16777216u);
+                    Philox4 rnd;
+                    if (random) rnd = sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr));
+                    else rnd.v[0] = rnd.v[1] = rnd.v[2] = rnd.v[3] = 0u;    // decided without them: 0 never up, 2^24 always up
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int i = 2 * pr + h;
+                        if (i >= nf) break;
+                        w1 |= round_up_if(cell[h], t[h], rnd.v[2 * h]) << (i * CB);
+                        w2 |= round_up_if(cell[h], t[h], rnd.v[2 * h + 1]) << (i * CB);
+                    }
                 }
             }
         }
