@@ -78,6 +78,51 @@ __global__ void __launch_bounds__(256) range_scan_kernel(const float* __restrict
     }
 }
 
+// The same scan for wide matrices: a block reads 4 KB of consecutive columns of a row at a time (256 threads x
+// float4; the narrow kernel's 512-byte pieces waste DRAM pages on rows of tens of kilobytes), a thread keeps its
+// four columns for all rows of the block's chunk, four rows' loads in flight; no meeting in shared memory.
+__global__ void __launch_bounds__(256) range_scan_wide_kernel(const float* __restrict__ A, int64_t m, int64_t n, int64_t lda,
+                                                              int64_t rows_per_block, uint32_t* lo_key, uint32_t* hi_key,
+                                                              DeviceStatus* status) {
+    const int64_t j0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+    if (j0 >= n) return;
+    const int64_t r0 = (int64_t)blockIdx.y * rows_per_block;
+    const int64_t r1 = min(m, r0 + rows_per_block);
+    const int nv = (int)min((int64_t)4, n - j0);
+    float lo[4], hi[4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v) { lo[v] = INFINITY; hi[v] = -INFINITY; }
+    bool bad = false;
+    const float* col = A + j0;
+    if (nv == 4) {
+#pragma unroll 4
+        for (int64_t r = r0; r < r1; ++r) {
+            const float4 q = __ldg(reinterpret_cast<const float4*>(col + r * lda));
+            const float val[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                bad |= !(fabsf(val[v]) <= 3.402823466e+38f);
+                lo[v] = fminf(lo[v], val[v]);
+                hi[v] = fmaxf(hi[v], val[v]);
+            }
+        }
+    } else {
+        for (int64_t r = r0; r < r1; ++r)
+            for (int v = 0; v < nv; ++v) {
+                const float val = __ldg(col + r * lda + v);
+                bad |= !(fabsf(val) <= 3.402823466e+38f);
+                lo[v] = fminf(lo[v], val);
+                hi[v] = fmaxf(hi[v], val);
+            }
+    }
+    if (bad) set_status(status, ZIPML_ERR_NONFINITE, 1);
+    for (int v = 0; v < nv; ++v)
+        if (lo[v] <= hi[v]) {  // at least one row seen
+            atomicMin(lo_key + j0 + v, float_order_key(lo[v]));
+            atomicMax(hi_key + j0 + v, float_order_key(hi[v]));
+        }
+}
+
 __global__ void range_finalize_kernel(const uint32_t* lo_key, const uint32_t* hi_key, int64_t n, int s,
                                       float* lo_out, float* hi_out, float* inv_out, float* step_out) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -97,6 +142,20 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
     const unsigned nb = (unsigned)((n + 255) / 256);
     range_init_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n);
     const bool vec = (lda % 4 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15) == 0);
+    if (vec && n >= 2048) {
+        const int64_t col_tiles = (n + 1023) / 1024;
+        int64_t chunks = (int64_t)ctx->sm_count * 8 / col_tiles;
+        chunks = chunks < 1 ? 1 : chunks;
+        int64_t rows_per_block = (m + chunks - 1) / chunks;
+        rows_per_block = rows_per_block < 64 ? 64 : rows_per_block;
+        chunks = (m + rows_per_block - 1) / rows_per_block;
+        if (chunks > 65535) { rows_per_block = (m + 65534) / 65535; chunks = (m + rows_per_block - 1) / rows_per_block; }
+        range_scan_wide_kernel<<<dim3((unsigned)col_tiles, (unsigned)chunks), 256, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key,
+                                                                                                   hi_key, ctx->d_status);
+        range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, lo_out, hi_out, inv_out, step_out);
+        ctx->launches += 3;
+        return cuda_status(cudaGetLastError());
+    }
     const int width = vec ? 128 : 32;
     const int64_t col_tiles = (n + width - 1) / width;
     // enough row chunks to give every SM a few blocks, at least 64 rows each

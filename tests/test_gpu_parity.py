@@ -93,6 +93,12 @@ def test_quantize_reports_bad_input(ctx):
     ctx.zipml_quantize(A, 4, seed=0)
     with pytest.raises(binding.ZipmlError):
         ctx.zipml_sync()
+    wide = torch.rand((70, 2052), device=ctx.device)               # wide rows take another range-scan kernel
+    wide[69, 2049] = float("nan")                                  # in the ragged last group of four columns
+    ctx.zipml_quantize(wide[:, :2050], 2, seed=0)
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sync()
+    assert e.value.code == binding.ERR_NONFINITE
     good = torch.rand((64, 16), device=ctx.device)
     for bits in (1, 5, 16):
         with pytest.raises(binding.ZipmlError) as e:
