@@ -264,6 +264,28 @@ def test_stream_engine_wide_rows(ctx, case):
     assert e.value.code == binding.ERR_WORKSPACE
 
 
+def test_stream_engine_batch_limits(ctx):
+    """The largest batch the stream engine takes (its residual digits live in shared memory), and one row more."""
+    m, n = 8300, 10240
+    _, A, b, _ = workload("c5", m, n, seed=11)
+    ods = oracle.quantize(A, 4, seed=12)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = np.zeros(n, np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 8192, 1e-4)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 8192, 1e-4, engine=binding.ENGINE_STREAM)
+    ctx.zipml_sync()
+    assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), 8193, 1e-4, engine=binding.ENGINE_STREAM)
+    assert e.value.code == binding.ERR_WORKSPACE
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 8193, 1e-4)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 8193, 1e-4)                                 # AUTO: another engine takes it
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() != binding.ENGINE_STREAM and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+
+
 def test_sgd_engines_and_grids_agree_bitwise_where_the_reduction_order_is_the_same(ctx):
     _, A, b, _ = workload("c2", 1500, 300, seed=2)
     ods = oracle.quantize(A, 8, seed=1)
