@@ -151,6 +151,11 @@ int32_t zipml_last_engine(const zipml_ctx* ctx);
  * nanoseconds (device timer) to ns_out (one uint64, DEVICE pointer).  floats_per_cta % 4 == 0.
  * ZIPML_ERR_WORKSPACE if `ctas` CTAs cannot be resident at once. */
 int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, int32_t iterations, uint64_t* ns_out);
+/* Diagnostics for the error path of the device-side waits: one thread polls a flag that nothing sets, with
+ * the engines' bounded-wait pattern and a limit of spin_limit polls (1 .. 2^24), gives up and records
+ * ZIPML_ERR_TIMEOUT, which the next zipml_sync returns (and clears); the context stays usable.  The paper
+ * has no counterpart; it exists so that the time-out route can be exercised without a hung kernel. */
+int zipml_wait_probe(zipml_ctx* ctx, int64_t spin_limit);
 /* Smallest legal row stride for n features: ceil(n*cb/8) rounded up to 16; 0 if bits is unsupported. */
 int64_t zipml_row_bytes(int64_t n, int32_t bits);
 

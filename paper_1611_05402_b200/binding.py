@@ -17,7 +17,7 @@ REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM = 0, 1, 2, 3, 4, 5, 6
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -66,6 +66,7 @@ def lib():
         L.zipml_last_engine.argtypes = [vp]
         L.zipml_last_engine.restype = C.c_int32
         L.zipml_barrier_latency.argtypes = [vp, i32, i32, i32, vp]
+        L.zipml_wait_probe.argtypes = [vp, i64]
         L.zipml_strerror.argtypes = [C.c_int]
         L.zipml_strerror.restype = C.c_char_p
         L.zipml_row_bytes.argtypes = [i64, i32]
@@ -172,6 +173,10 @@ class Context:
         _check(lib().zipml_barrier_latency(self._h, ctas, floats_per_cta, iterations, _ptr(out)), "zipml_barrier_latency")
         self.zipml_sync()
         return out.item() / iterations
+
+    def zipml_wait_probe(self, spin_limit=100000):
+        """Enqueues a bounded wait that must give up; the next zipml_sync raises ZipmlError(ERR_TIMEOUT)."""
+        _check(lib().zipml_wait_probe(self._h, spin_limit), "zipml_wait_probe")
 
     def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None):
         m, n = A.shape

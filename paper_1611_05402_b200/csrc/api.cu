@@ -62,6 +62,21 @@ constexpr int kLossPartials = 4096;
 
 using namespace zipml;
 
+namespace zipml {
+// A wait that cannot succeed, bounded like the engines' waits: lane 0 polls a zero flag `limit` times with an
+// acquire load and a pause now and then, then records the time-out (see zipml_wait_probe).
+__global__ void wait_probe_kernel(const unsigned* flag, long long limit, DeviceStatus* status) {
+    if (threadIdx.x != 0) return;
+    for (long long it = 0; it < limit; ++it) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v != 0) return;
+        if ((it & 1023) == 1023) __nanosleep(200);
+    }
+    set_status(status, ZIPML_ERR_TIMEOUT, 90);
+}
+}  // namespace zipml
+
 extern "C" {
 
 const char* zipml_strerror(int status) {
@@ -243,6 +258,19 @@ int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
     return launch_barrier_latency(ctx, ctas, floats_per_cta, iterations, reinterpret_cast<unsigned long long*>(ns_out));
+}
+
+int zipml_wait_probe(zipml_ctx* ctx, int64_t spin_limit) {
+    if (!ctx || spin_limit < 1 || spin_limit > (1 << 24)) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    int rc = ws_reserve(ctx, 256);
+    if (rc != ZIPML_OK) return rc;
+    cudaError_t e = cudaMemsetAsync(ctx->ws, 0, 256, ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    wait_probe_kernel<<<1, 32, 0, ctx->stream>>>(reinterpret_cast<const unsigned*>(ctx->ws), spin_limit, ctx->d_status);
+    ctx->launches += 1;
+    return cuda_status(cudaGetLastError());
 }
 
 int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t n, int64_t lda,

@@ -81,6 +81,27 @@ def test_quantize_strided_and_unaligned_input(ctx):
     assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all()
 
 
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(ctx):
+    """The device-side waits are bounded: one that cannot succeed (a flag that nothing sets) gives up, the next
+    zipml_sync returns ZIPML_ERR_TIMEOUT once, and the same context then works as before."""
+    ctx.zipml_sync()
+    ctx.zipml_wait_probe(50000)
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sync()
+    assert e.value.code == binding.ERR_TIMEOUT
+    ctx.zipml_sync()                                               # reported once, then cleared
+    _, A, b, _ = workload("c1", 256, 64, seed=1)
+    ods = oracle.quantize(A, 4, seed=1)
+    gds = ctx.zipml_quantize(to_dev(A, ctx), 4, seed=1)
+    x = torch.zeros(64, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, to_dev(b, ctx), x, 16, 0.01)
+    ctx.zipml_sync()
+    x_ref, _ = oracle.sgd_epoch(ods, b, np.zeros(64, np.float32), 16, 0.01)
+    assert (gds.plane1.cpu().numpy()[:, : ods.row_bytes] == ods.plane1).all() and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_wait_probe(0)
+
+
 def test_quantize_reports_bad_input(ctx):
     A = torch.rand((64, 16), device=ctx.device)
     A[5, 3] = float("nan")
