@@ -164,7 +164,7 @@ __device__ __forceinline__ void clu_mark(const ClusterArgs& a, int64_t it, int i
 
 // Shared memory after ClusterShared; Fp = row_words * FPW feature slots of a row (padding included),
 // Fs = nb * sub >= n features as the owners cut them:
-//   uniform: wv[Fp]  w = step * x~, [slot i][word q];  los[Fp], steps[Fp]  lo and step by feature
+//   uniform: wv[Fp]  w = step * x~ by feature;  los[Fp], steps[Fp]  lo and step by feature
 //   table:   tab[L*Fp] level * x~ and lev[L*Fp] levels, both [code][slot i][word q]
 //   xs[Fs]           the model this step sees (all-gather destination)
 //   gpart[Fs]        this CTA's part of the gradient (reduce-scatter source)
@@ -515,11 +515,15 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                             float c1[FPW], c2[FPW];
                             unpack_word<CB>(u1, c1);
                             unpack_word<CB>(u2, c2);
+                            // the word's FPW entries of w lie together: 16-byte loads, a quarter of the load instructions
+                            const float4* wq = reinterpret_cast<const float4*>(wv) + (size_t)q * (FPW / 4);
 #pragma unroll
-                            for (int i = 0; i < FPW; ++i) {
-                                const float w = wv[i * rw + q];
-                                acc1 = fmaf(c1[i], w, acc1);
-                                acc2 = fmaf(c2[i], w, acc2);
+                            for (int i4 = 0; i4 < FPW / 4; ++i4) {
+                                const float4 w4 = wq[i4];
+                                acc1 = fmaf(c1[4 * i4], w4.x, acc1); acc2 = fmaf(c2[4 * i4], w4.x, acc2);
+                                acc1 = fmaf(c1[4 * i4 + 1], w4.y, acc1); acc2 = fmaf(c2[4 * i4 + 1], w4.y, acc2);
+                                acc1 = fmaf(c1[4 * i4 + 2], w4.z, acc1); acc2 = fmaf(c2[4 * i4 + 2], w4.z, acc2);
+                                acc1 = fmaf(c1[4 * i4 + 3], w4.w, acc1); acc2 = fmaf(c2[4 * i4 + 3], w4.w, acc2);
                             }
                         } else {
 #pragma unroll
@@ -712,7 +716,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                 wm = fmaxf(wm, fabsf(w));
                 bpart += (double)los[f] * (double)xt;
             } else if constexpr (!TABLE) {
-                wv[i * rw + q] = steps[f] * xt;
+                wv[f] = steps[f] * xt;
                 bpart += (double)los[f] * (double)xt;
             } else {
                 for (int c = 0; c < L; ++c) tab[(c * FPW + i) * rw + q] = lev[(c * FPW + i) * rw + q] * xt;
