@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one epoch launch from the ncu capture summarised under profiles/
 # (workload, engine) -> bytes; an entry is removed when its kernel changes after the capture
 # (c5: captured on 16,384 of the 65,536 rows, 591.80 + 6.29 MB, and scaled by the rows: traffic grows with them)
-NCU_TRAFFIC_BYTES = {("c2", 5): 202.12e6 + 4.10e6, ("c5", 6): 4 * (591.80e6 + 6.29e6)}
+NCU_TRAFFIC_BYTES = {("c2", 5): 203.04e6 + 3.76e6, ("c5", 6): 4 * (591.80e6 + 6.29e6)}
 ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
                   5: "sgd_cluster_kernel", 6: "sgd_stream_kernel"}
 
