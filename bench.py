@@ -34,7 +34,7 @@ NOMINAL_HBM_GBS = 8000.0
 # (c5: captured on 16,384 of the 65,536 rows, 591.80 + 6.29 MB, and scaled by the rows: traffic grows with them)
 NCU_TRAFFIC_BYTES = {("c2", 5): 203.04e6 + 3.76e6, ("c5", 6): 4 * (591.80e6 + 6.29e6)}
 ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
-                  5: "sgd_cluster_kernel", 6: "sgd_stream_kernel"}
+                  5: "sgd_cluster_kernel", 6: "sgd_stream_kernel", 7: "sgd_column_kernel"}
 
 
 def measured_peaks():
@@ -120,7 +120,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
     ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
-    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster", "stream"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster", "stream", "column"])
+    ap.add_argument("--chunk-rows", type=int, default=0, help="column engine: rows per chunk (0 = automatic)")
     ap.add_argument("--feature-parts", type=int, default=0)
     ap.add_argument("--row-parts", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -186,13 +187,13 @@ def main():
     dev = torch.device("cuda", local_rank)
     engine = {"auto": binding.ENGINE_AUTO, "stepwise": binding.ENGINE_STEPWISE, "persistent": binding.ENGINE_PERSISTENT,
               "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN, "cluster": binding.ENGINE_CLUSTER,
-              "stream": binding.ENGINE_STREAM}[args.engine]
+              "stream": binding.ENGINE_STREAM, "column": binding.ENGINE_COLUMN}[args.engine]
 
     w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
     ctx = binding.Context(dev)
     loss_dev = torch.zeros(1, dtype=torch.float64, device=dev)
     kw = dict(model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed, engine=engine,
-              grid_feature_parts=args.feature_parts, grid_row_parts=args.row_parts)
+              grid_feature_parts=args.feature_parts, grid_row_parts=args.row_parts, column_chunk_rows=args.chunk_rows)
     epoch_events, quant_events, loss_events = [], [], []
 
     def timed(events, record, fn):

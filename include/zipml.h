@@ -57,9 +57,9 @@ enum {
 };
 /* How zipml_sgd_epoch runs its minibatch chain.  Results do not depend on the choice. */
 enum {
-    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; else stream
-                                   where it applies (wide rows, uniform grid, fp32 model and gradient),
-                                   else ring                                                          */
+    ZIPML_ENGINE_AUTO = 0,      /* cluster, else lean, for steps of at most 2 MiB of codes; else column,
+                                   else stream, where they apply (wide rows, uniform grid, fp32 model
+                                   and gradient), else ring                                           */
     ZIPML_ENGINE_STEPWISE = 1,  /* a few kernel launches per minibatch                               */
     ZIPML_ENGINE_PERSISTENT = 2, /* one cooperative launch per call, grid barriers between the phases */
     ZIPML_ENGINE_RING = 3,       /* one cooperative launch; producer warp streams code chunks through a
@@ -69,16 +69,24 @@ enum {
     ZIPML_ENGINE_CLUSTER = 5,    /* one thread-block cluster (at most 16 row parts) for small tiles:
                                     gradients and model travel between the CTAs' shared memories.
                                     Uniform grids contract in fp32 or, on taller tiles, on the int8
-                                    tensor cores; the environment variable ZIPML_CLUSTER_INT8=0/1
-                                    overrides that choice                                             */
-    ZIPML_ENGINE_STREAM = 6      /* one cooperative launch for large tiles on uniform grids with an fp32
+                                    tensor cores; zipml_sgd_params.cluster_contraction overrides that
+                                    choice                                                            */
+    ZIPML_ENGINE_STREAM = 6,     /* one cooperative launch for large tiles on uniform grids with an fp32
                                     model and gradient: both passes of a step read the codes straight
                                     from global memory into int8 tensor-core fragments (the second pass
                                     from L2), a CTA owns whole column blocks of the gradient, one grid
                                     barrier per step.  ZIPML_ERR_WORKSPACE for level tables, quantized
-                                    model or gradient, batches above 8192 rows.  The environment
-                                    variable ZIPML_STREAM_PREFETCH=0..8 overrides how many eighths of
-                                    the next step's tile are requested into L2 ahead of time           */
+                                    model or gradient, batches above 8192 rows.
+                                    zipml_sgd_params.stream_prefetch overrides how many eighths of the
+                                    next step's tile are requested into L2 ahead of time               */
+    ZIPML_ENGINE_COLUMN = 7      /* one cooperative launch for large tiles on uniform grids with an fp32
+                                    model and gradient, rows of 128 bytes .. 128 bytes x the number of
+                                    SMs: a CTA owns a 128-byte column block of the packed rows for the
+                                    whole launch; rows travel through shared memory in chunks that
+                                    serve both passes of the step, so the codes are read from HBM once
+                                    per step; CTAs exchange only the rows' dots (integer atomics and one
+                                    counter per chunk), there is no grid-wide barrier.
+                                    ZIPML_ERR_WORKSPACE for what it does not cover (as for STREAM)     */
 };
 
 typedef struct zipml_ctx zipml_ctx;
@@ -130,6 +138,18 @@ typedef struct zipml_sgd_params {
                                    7 residual scale known.  Other engines ignore the request.         */
     int32_t reg;                /* ZIPML_REG_*                                                       */
     float reg_param;            /* c or lambda (>= 0); ignored by ZIPML_REG_NONE and _NONNEG          */
+    float* model_out;           /* debug, DEVICE pointer or NULL: n floats, the model that the last
+                                   executed step's gradient saw -- Q3(x) of that step when model_bits > 0
+                                   (Supplement "Quantizing the Model"), else x as it stood before the step.
+                                   ZIPML_ERR_WORKSPACE from the stream and column engines, which keep
+                                   no such copy                                                      */
+    int32_t cluster_contraction; /* tuning, cluster engine on uniform grids: 0 = automatic, 1 = fp32,
+                                   2 = int8 tensor cores                                             */
+    int32_t stream_prefetch;    /* tuning, stream engine: 0 = automatic, 1..9 = request (value - 1)
+                                   eighths of the next step's tile into L2 ahead of time             */
+    int32_t column_chunk_rows;  /* tuning, column engine: 0 = automatic, else rows of a minibatch that
+                                   travel through shared memory together (a multiple of 32, 32..256)  */
+    int32_t reserved0;          /* must be 0                                                         */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default
@@ -228,7 +248,8 @@ int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, 
  *   - Its scratch (the table step*x or level*x and one partial sum per block) is a fixed array
  *     inside the library image, about 1 MiB, which every GPU that loads the library holds until the
  *     process exits.  Limit: n <= 262144 features for a uniform grid, 2^bits * n <= 262144 with a
- *     level table; larger problems are refused with ZIPML_ERR_WORKSPACE.
+ *     level table; larger problems are refused with ZIPML_ERR_WORKSPACE.  The dataset is checked as
+ *     by every other call (planes 16-byte aligned, stride a multiple of 16).
  *   - It calls no cudaMalloc/cudaFree and no allocating library routine.  The first call on a
  *     device looks up the array's device address (once per device); make that first call outside
  *     any stream capture.
@@ -238,8 +259,11 @@ int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, 
  *   device       ordinal of the GPU that holds the data
  *   cuda_stream  cudaStream_t as void* (NULL: the legacy default stream); the work is enqueued there
  *   data, b, x   as for zipml_loss; DEVICE pointers.   loss_out  one double, DEVICE pointer.
- * Returns like the other calls; the result equals zipml_loss(CODES) up to the order in which the
- * per-block partial sums are added. */
+ * Returns like the other calls.  It is the same estimator as zipml_loss(CODES) in other arithmetic: fp32
+ * products summed in short runs and combined in double here, where zipml_loss on a uniform grid
+ * rounds step*x once to fixed point and sums integers; the two agree to about 1e-6 relative.  The
+ * one-time address lookup is guarded by a lock, so two host threads may make a device's first call
+ * together (their kernels still must not overlap, see above). */
 int zipml_loss_codes_static(int device, void* cuda_stream, const zipml_dataset* data, const float* b,
                             const float* x, double* loss_out);
 

@@ -14,7 +14,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORK
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
 REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
-ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM = 0, 1, 2, 3, 4, 5, 6
+ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM, ENGINE_COLUMN = 0, 1, 2, 3, 4, 5, 6, 7
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
 EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
@@ -44,7 +44,9 @@ class CSgdParams(C.Structure):
                 ("batch", C.c_int64), ("epoch", C.c_int64), ("first_step", C.c_int64), ("num_steps", C.c_int64),
                 ("seed", C.c_uint64), ("batch_order", C.c_void_p), ("lr", C.c_float),
                 ("grid_feature_parts", C.c_int32), ("grid_row_parts", C.c_int32), ("trace_steps", C.c_int32),
-                ("trace", C.c_void_p), ("reg", C.c_int32), ("reg_param", C.c_float)]
+                ("trace", C.c_void_p), ("reg", C.c_int32), ("reg_param", C.c_float),
+                ("model_out", C.c_void_p), ("cluster_contraction", C.c_int32), ("stream_prefetch", C.c_int32),
+                ("column_chunk_rows", C.c_int32), ("reserved0", C.c_int32)]
 
 
 _lib = None
@@ -204,13 +206,19 @@ class Context:
 
     def sgd_params(self, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=-1,
                    batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0, trace=None,
-                   reg=REG_NONE, reg_param=0.0):
+                   reg=REG_NONE, reg_param=0.0, model_out=None, cluster_contraction=0, stream_prefetch=0,
+                   column_chunk_rows=0):
         p = CSgdParams()
         p.struct_size = C.sizeof(CSgdParams)
         p.model_bits, p.grad_bits, p.engine = model_bits, grad_bits, engine
         p.batch, p.epoch, p.first_step, p.num_steps, p.seed, p.lr = batch, epoch, first_step, num_steps, seed, lr
         p.grid_feature_parts, p.grid_row_parts = grid_feature_parts, grid_row_parts
         p.reg, p.reg_param = reg, reg_param
+        p.cluster_contraction, p.stream_prefetch = cluster_contraction, stream_prefetch
+        p.column_chunk_rows = column_chunk_rows
+        if model_out is not None:  # (n,) fp32 device tensor
+            assert model_out.dtype == torch.float32 and model_out.is_contiguous() and model_out.device == self.device
+            p.model_out = model_out.data_ptr()
         if trace is not None:      # (steps, 8) int64 device tensor
             assert trace.dtype == torch.int64 and trace.is_contiguous() and trace.shape[1] == 8
             p.trace, p.trace_steps = trace.data_ptr(), trace.shape[0]

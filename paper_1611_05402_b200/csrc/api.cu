@@ -41,7 +41,7 @@ struct DeviceGuard {
     ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
 };
 
-static int check_dataset(const zipml_dataset* d) {
+int check_dataset(const zipml_dataset* d) {
     if (!d || d->struct_size != sizeof(zipml_dataset)) return ZIPML_ERR_INVALID_ARG;
     const int cb = container_bits(d->bits);
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
@@ -213,10 +213,14 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (!b || !x || params->batch <= 0) return ZIPML_ERR_INVALID_ARG;
     if (params->model_bits != 0 && (params->model_bits < 2 || params->model_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
     if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
-    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_STREAM) return ZIPML_ERR_INVALID_ARG;
+    if (params->engine < ZIPML_ENGINE_AUTO || params->engine > ZIPML_ENGINE_COLUMN) return ZIPML_ERR_INVALID_ARG;
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
     if (params->reg < ZIPML_REG_NONE || params->reg > ZIPML_REG_LSSVM) return ZIPML_ERR_INVALID_ARG;
     if (params->reg != ZIPML_REG_NONE && params->reg != ZIPML_REG_NONNEG && !(params->reg_param >= 0.0f)) return ZIPML_ERR_INVALID_ARG;
+    if (params->cluster_contraction < 0 || params->cluster_contraction > 2) return ZIPML_ERR_INVALID_ARG;
+    if (params->stream_prefetch < 0 || params->stream_prefetch > 9) return ZIPML_ERR_INVALID_ARG;
+    if (params->column_chunk_rows < 0 || params->column_chunk_rows > 256 || params->column_chunk_rows % 32 != 0) return ZIPML_ERR_INVALID_ARG;
+    if (params->reserved0 != 0) return ZIPML_ERR_INVALID_ARG;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
     const int64_t count = params->num_steps < 0 ? T - first : params->num_steps;
@@ -231,10 +235,12 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->engine == ZIPML_ENGINE_LEAN) return launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_STREAM) return launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, false);
+    if (params->engine == ZIPML_ENGINE_COLUMN) return launch_sgd_column(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_AUTO) {
         // Small minibatch tiles are bound by the step-to-step chain, not by HBM: one cluster whose CTAs
-        // exchange through shared memory, else row parts exchanging through L2.  Larger tiles stream
-        // through the ring engine.  Each engine answers ZIPML_ERR_WORKSPACE when the shape does not fit it.
+        // exchange through shared memory, else row parts exchanging through L2.  Larger tiles go to the
+        // column engine (codes read once per step), the stream engine, then the ring engine.  Each engine
+        // answers ZIPML_ERR_WORKSPACE when the shape does not fit it.
         const int64_t B = params->batch < data->m ? params->batch : data->m;
         const int64_t step_bytes = 2 * B * data->row_bytes;
         if (step_bytes <= (2ll << 20)) {
@@ -244,6 +250,8 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
             if (rc != ZIPML_ERR_WORKSPACE) return rc;
         }
         // (also for small steps on rows too wide for the two above)
+        rc = launch_sgd_column(ctx, data, b, x, params, first, count, grad_out, true);
+        if (rc != ZIPML_ERR_WORKSPACE) return rc;
         rc = launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, true);
         if (rc != ZIPML_ERR_WORKSPACE) return rc;
         rc = launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
@@ -287,9 +295,12 @@ int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t 
     }
     int rc = check_dataset(data);
     if (rc != ZIPML_OK) return rc;
-    const size_t tab = (data->level_mode == ZIPML_LEVELS_TABLE ? ((size_t)1 << data->bits) : 1) * (size_t)data->n;
-    // (+ slack: the digit vectors of the uniform path round the row up to 64 bytes)
-    rc = ws_reserve(ctx, carve_size(sizeof(double) * (kLossPartials + 2) + sizeof(float) * tab + 2048));
+    // behind the partials: the level * x table, or (uniform grids) the digit vectors of step * x, which follow the
+    // packed row byte for byte and so take their size from the stride, not from n
+    const size_t tab = data->level_mode == ZIPML_LEVELS_TABLE
+                           ? sizeof(float) * ((size_t)1 << data->bits) * (size_t)data->n
+                           : (size_t)(8 / container_bits(data->bits)) * 4 * (((size_t)data->row_bytes + 63) / 64 * 64);
+    rc = ws_reserve(ctx, carve_size(sizeof(double) * (kLossPartials + 2) + tab + 256));
     if (rc != ZIPML_OK) return rc;
     return launch_loss_codes(ctx, data, b, x, reinterpret_cast<double*>(ctx->ws), kLossPartials, loss_out);
 }

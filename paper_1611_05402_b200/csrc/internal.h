@@ -31,6 +31,9 @@ struct zipml_ctx {
 
 namespace zipml {
 
+// Argument checks shared by every entry point that takes a dataset: ZIPML_OK, or the status to return.
+int check_dataset(const zipml_dataset* d);
+
 // Status helpers -------------------------------------------------------------------------------
 int cuda_status(cudaError_t e);                       // ZIPML_OK or ZIPML_ERR_CUDA (clears the sticky error)
 int ws_reserve(zipml_ctx* ctx, size_t bytes);         // grow ctx->ws to at least `bytes`
@@ -89,6 +92,9 @@ int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, f
 // Stream engine (uniform grids, fp32 model and gradient).  With only_if_profitable it declines
 // (ZIPML_ERR_WORKSPACE) shapes whose steps are too narrow or too short for it.
 int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
+                      int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
+// Column engine (uniform grids, fp32 model and gradient, rows of at most 128 bytes per SM).
+int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                       int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
 int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,

@@ -1,5 +1,7 @@
 // Training loss (paper Eq. (leastsquares) with l = a^T x - b) on the dense samples, its unbiased
 // estimate from the two code planes, and the allocation-free variant of the latter.
+#include <mutex>
+
 #include "common.cuh"
 #include "int_digits.cuh"
 #include "internal.h"
@@ -96,7 +98,8 @@ __global__ void __launch_bounds__(256) loss_codes_kernel(const uint32_t* __restr
 // straight from global memory (rows g and g+8 of lane group g; four lanes cover the span), and every
 // 8 bytes of a lane's 16 are one mma.sync m16n8k32 (u8 x s8) against the matching 8 bytes of each
 // digit's vector (digits in the byte order of the codes, so the operand's k order is simply the
-// lane's own byte order).  Digit sums are exact; they are combined in double.
+// lane's own byte order).  Digit sums are exact (32-bit sums moved into 64 bits before they can
+// wrap, whatever the row length); they are combined in double.
 // ---------------------------------------------------------------------------------------------
 // Digit vectors of w: wdig[group][digit][byte of the row], row_bytes rounded up to 64 per vector.
 template <int CB>
@@ -132,6 +135,8 @@ __global__ void __launch_bounds__(1024) loss_digits_kernel(const float* __restri
     }
 }
 
+constexpr int64_t kLossFlushSpans = 1024;
+
 template <int CB>
 __global__ void __launch_bounds__(512) loss_codes_imma_kernel(const unsigned char* __restrict__ p1, const unsigned char* __restrict__ p2,
                                                               int64_t row_bytes, int64_t m, int64_t vec_bytes,
@@ -152,9 +157,14 @@ __global__ void __launch_bounds__(512) loss_codes_imma_kernel(const unsigned cha
         const unsigned char* h1 = p1 + rh * row_bytes + 16 * tl;
         const unsigned char* a2 = p2 + ra * row_bytes + 16 * tl;
         const unsigned char* h2 = p2 + rh * row_bytes + 16 * tl;
+        // A span adds at most 2 * 32 * 255 * 64 to a 32-bit digit sum: they are moved into 64-bit sums every
+        // kLossFlushSpans spans (2^20 * 1024 < 2^31), so rows of any admitted length stay exact.
+        long long s1[4] = {0, 0, 0, 0}, s2[4] = {0, 0, 0, 0};
+        for (int64_t sp0 = 0; sp0 < nspans; sp0 += kLossFlushSpans) {
         int c1[4] = {0, 0, 0, 0}, c2[4] = {0, 0, 0, 0};
+        const int64_t sp1 = min(nspans, sp0 + kLossFlushSpans);
 #pragma unroll 2
-        for (int64_t sp = 0; sp < nspans; ++sp) {
+        for (int64_t sp = sp0; sp < sp1; ++sp) {
             const int64_t off = sp * 64;
             uint4 ua = make_uint4(0u, 0u, 0u, 0u), uh = ua, va = ua, vh = ua;
             if (off + 16 * tl < row_bytes) {                      // rows are whole multiples of 16 bytes
@@ -173,12 +183,15 @@ __global__ void __launch_bounds__(512) loss_codes_imma_kernel(const unsigned cha
                 mma_u8s8(c2, group_bytes<CB>(va.z, g), group_bytes<CB>(vh.z, g), group_bytes<CB>(va.w, g), group_bytes<CB>(vh.w, g), bd.z, bd.w);
             }
         }
-        // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3])
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { s1[e] += c1[e]; s2[e] += c2[e]; }
+        }
+        // lane t < 2 holds digits 2t, 2t+1 of rows g (s[0], s[1]) and g+8 (s[2], s[3])
         double v[4];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-            const double q1 = (double)c1[2 * e] + 128.0 * (double)c1[2 * e + 1];
-            const double q2 = (double)c2[2 * e] + 128.0 * (double)c2[2 * e + 1];
+            const double q1 = (double)s1[2 * e] + 128.0 * (double)s1[2 * e + 1];
+            const double q2 = (double)s2[2 * e] + 128.0 * (double)s2[2 * e + 1];
             v[2 * e] = q1 + 16384.0 * __shfl_down_sync(0xffffffffu, q1, 1);
             v[2 * e + 1] = q2 + 16384.0 * __shfl_down_sync(0xffffffffu, q2, 1);
         }
@@ -214,7 +227,7 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
     double* base = partials + max_partials;
     float* wtab = reinterpret_cast<float*>(base + 2);
     if (!table) {
-        // digit vectors take (8 / cb) * 4 * roundup64(row_bytes) bytes <= 4 n + slack: they fit the table's space
+        // digit vectors take (8 / cb) * 4 * roundup64(row_bytes) bytes (the caller reserved them from the stride)
         const int64_t vec_bytes = (d->row_bytes + 63) / 64 * 64;
         signed char* wdig = reinterpret_cast<signed char*>(wtab);
         int blocks = ctx->sm_count * 2;                            // 2 x 16 warps per SM, 16 rows per warp and turn
@@ -343,12 +356,14 @@ struct StaticLossDevice {
     int sm_count = 0;
 };
 static StaticLossDevice g_static_loss_devices[kMaxDevices];
+static std::mutex g_static_loss_lock;           // two host threads may make a device's first call together
 
 // Once per device, with that device current: in host code the array's name is only a handle, the
 // kernels need the device address, which cudaGetSymbolAddress returns.
 static int static_loss_setup(int device, StaticLossDevice** out) {
     if (device < 0 || device >= kMaxDevices) return ZIPML_ERR_INVALID_ARG;
     StaticLossDevice& d = g_static_loss_devices[device];
+    std::lock_guard<std::mutex> guard(g_static_loss_lock);
     if (!d.ready) {
         void* p = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&p, g_static_loss_scratch);
@@ -367,15 +382,11 @@ static int static_loss_setup(int device, StaticLossDevice** out) {
 extern "C" int zipml_loss_codes_static(int device, void* cuda_stream, const zipml_dataset* data, const float* b,
                                        const float* x, double* loss_out) {
     using namespace zipml;
-    if (!data || data->struct_size != sizeof(zipml_dataset) || !b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
+    if (!b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
+    const int bad = check_dataset(data);          // the same checks as every other entry point (plane alignment included)
+    if (bad != ZIPML_OK) return bad;
     const int cb = container_bits(data->bits);
-    if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
     const bool table = data->level_mode == ZIPML_LEVELS_TABLE;
-    if (!table && data->level_mode != ZIPML_LEVELS_UNIFORM) return ZIPML_ERR_INVALID_ARG;
-    if (table && data->bits == 8) return ZIPML_ERR_UNSUPPORTED;
-    if (data->m <= 0 || data->n <= 0 || !data->plane1 || !data->plane2) return ZIPML_ERR_INVALID_ARG;
-    if (data->row_bytes % 16 != 0 || data->row_bytes < zipml_row_bytes(data->n, data->bits)) return ZIPML_ERR_INVALID_ARG;
-    if (table ? !data->levels : (!data->feat_lo || !data->feat_step)) return ZIPML_ERR_INVALID_ARG;
     const int L = 1 << data->bits;
     const int64_t table_floats = (table ? (int64_t)L : 1) * data->n;
     if (table_floats > kStaticLossTableFloats) return ZIPML_ERR_WORKSPACE;   // beyond the fixed scratch

@@ -223,6 +223,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_kernel(const SgdArgs a) {
                         const int f = q * FPW + i;
                         float xv = xs[f];
                         if (a.model_bits > 0) xv = q3.apply(xv, (uint32_t)(j0 + f));
+                        if (a.model_out && last && bi == 0 && f < fcnt) a.model_out[j0 + f] = xv;
                         float sv = 0.0f, lv = 0.0f;
                         if (f < fcnt) { sv = __ldg(a.step + j0 + f); lv = __ldg(a.lo + j0 + f); }
                         tab[((i >> 2) * a.wc + q) * 4 + (i & 3)] = sv * xv;
@@ -234,6 +235,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_kernel(const SgdArgs a) {
                 for (int f = threadIdx.x; f < F; f += kSgdThreads) {
                     float xv = xs[f];
                     if (a.model_bits > 0) xv = q3.apply(xv, (uint32_t)(j0 + f));
+                    if (a.model_out && last && bi == 0 && f < fcnt) a.model_out[j0 + f] = xv;
                     const int q = f / FPW, i = f % FPW;
                     for (int c = 0; c < L; ++c) {
                         const float lv = (f < fcnt) ? __ldg(a.levels + (j0 + f) * L + c) : 0.0f;
@@ -624,7 +626,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
     a.row_words = d->row_bytes / 4;
     a.m = d->m; a.n = d->n; a.bits = d->bits;
     a.lo = d->feat_lo; a.step = d->feat_step; a.levels = d->levels;
-    a.b = b; a.x = x; a.grad_out = grad_out;
+    a.b = b; a.x = x; a.grad_out = grad_out; a.model_out = p->model_out;
     a.batch = p->batch < d->m ? p->batch : d->m;
     a.first_step = first_step; a.num_steps = num_steps;
     a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
@@ -655,7 +657,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
             chunk.first_step = s0;
             chunk.num_steps = (first_step + num_steps - s0 < max_steps) ? first_step + num_steps - s0 : max_steps;
             chunk.phases = kPhaseAll; chunk.persistent = 1;
-            if (s0 + chunk.num_steps < first_step + num_steps) chunk.grad_out = nullptr;
+            if (s0 + chunk.num_steps < first_step + num_steps) { chunk.grad_out = nullptr; chunk.model_out = nullptr; }
             void* params[] = {&chunk};
             e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kSgdThreads), params, plan.smem, ctx->stream);
             if (e != cudaSuccess) return cuda_status(e);
@@ -668,7 +670,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
     for (int64_t s = first_step; s < first_step + num_steps; ++s) {
         SgdArgs step_args = a;
         step_args.first_step = s; step_args.num_steps = 1;
-        if (s != first_step + num_steps - 1) step_args.grad_out = nullptr;
+        if (s != first_step + num_steps - 1) { step_args.grad_out = nullptr; step_args.model_out = nullptr; }
         for (int ph : {kPhaseA, kPhaseB, kPhaseC}) {
             step_args.phases = ph;
             void* params[] = {&step_args};

@@ -56,6 +56,7 @@ struct ClusterArgs {
     const float* b;
     float* x;
     float* grad_out;             // null or 2n
+    float* model_out;            // null or n: the model the last executed step's gradient saw
     const int32_t* order;        // device copy of the batch order, or null
     unsigned long long* trace;
     DeviceStatus* status;
@@ -681,6 +682,7 @@ __global__ void __launch_bounds__(kCluThreads, 1) sgd_cluster_kernel(const Clust
                 float xt = (f < n) ? xown[k] : 0.0f;
                 if (a.model_bits > 0 && f < n)
                     xt = clu_quant(xt, xq_M, (1 << (a.model_bits - 1)) - 1, a.seed, a.epoch, (uint32_t)(it + 1), 3u, (uint32_t)f);
+                if (a.model_out && it + 2 == step_end && f < n) a.model_out[f] = xt;
                 xpub[k] = xt;
             }
         }
@@ -807,9 +809,8 @@ static int make_cluster_plan(const zipml_ctx* ctx, const zipml_dataset* d, const
     if (nb < 1) nb = 1;
     const size_t cap = (size_t)ctx->smem_optin;
     const int64_t nb_max = B < kCluMaxCtas ? B : kCluMaxCtas;
-    // ZIPML_CLUSTER_INT8=0/1 overrides the choice of the contraction for uniform grids (tests, tuning)
-    const char* env = getenv("ZIPML_CLUSTER_INT8");
-    const int force_int8 = (env && (env[0] == '0' || env[0] == '1') && env[1] == 0) ? env[0] - '0' : -1;
+    // the caller may fix the contraction for uniform grids (tests, tuning): 1 = fp32, 2 = int8 tensor cores
+    const int force_int8 = p->cluster_contraction == 1 ? 0 : p->cluster_contraction == 2 ? 1 : -1;
     // the requested number of row parts is a hint: more parts are used when a tile does not fit
     for (;; ++nb) {
         if (nb > nb_max) return ZIPML_ERR_WORKSPACE;
@@ -882,7 +883,7 @@ int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, f
     a.p1 = reinterpret_cast<const uint32_t*>(d->plane1);
     a.p2 = reinterpret_cast<const uint32_t*>(d->plane2);
     a.lo = d->feat_lo; a.step = d->feat_step; a.levels = d->levels;
-    a.b = b; a.x = x; a.grad_out = grad_out;
+    a.b = b; a.x = x; a.grad_out = grad_out; a.model_out = p->model_out;
     a.trace = reinterpret_cast<unsigned long long*>(p->trace);
     a.trace_steps = p->trace ? p->trace_steps : 0;
     a.status = ctx->d_status;

@@ -27,6 +27,7 @@ struct SgdArgs {
     const float* b;
     float* x;
     float* grad_out;        // null or 2n
+    float* model_out;       // null or n: the model the last executed step's gradient saw (Q3(x) or x)
     int64_t batch, first_step, num_steps;
     const int32_t* order;   // device copy of the batch order, or null
     float lr;

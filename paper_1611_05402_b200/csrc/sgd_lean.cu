@@ -49,6 +49,7 @@ struct LeanArgs {
     const float* b;
     float* x;
     float* grad_out;             // null or 2n
+    float* model_out;            // null or n: the model the last executed step's gradient saw
     const int32_t* order;        // device copy of the batch order, or null
     unsigned long long* rs;      // [n][nb]   partial gradients, per feature the nb writers
     unsigned long long* ag;      // [n]       the model the next step sees
@@ -418,6 +419,7 @@ __global__ void __launch_bounds__(kLeanThreads, 1) sgd_lean_kernel(const LeanArg
                 float xt = xown[k];
                 if (a.model_bits > 0)
                     xt = lean_quant(xt, xq_M, (1 << (a.model_bits - 1)) - 1, a.seed, a.epoch, (uint32_t)(it + 1), 3u, (uint32_t)f);
+                if (a.model_out && it + 2 == step_end) a.model_out[f] = xt;
                 lean_store(a.ag + f, xt, tag);
             }
         }
@@ -550,7 +552,7 @@ int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.p1 = reinterpret_cast<const uint32_t*>(d->plane1);
     a.p2 = reinterpret_cast<const uint32_t*>(d->plane2);
     a.lo = d->feat_lo; a.step = d->feat_step; a.levels = d->levels;
-    a.b = b; a.x = x; a.grad_out = grad_out;
+    a.b = b; a.x = x; a.grad_out = grad_out; a.model_out = p->model_out;
     a.rs = reinterpret_cast<unsigned long long*>(ctx->ws + o_ll);
     a.ag = a.rs + n_rs;
     a.gn = a.ag + n_ag;
@@ -579,7 +581,7 @@ int launch_sgd_lean(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         LeanArgs chunk = a;
         chunk.first_step = s0;
         chunk.num_steps = (first_step + num_steps - s0 < max_steps) ? first_step + num_steps - s0 : max_steps;
-        if (s0 + chunk.num_steps < first_step + num_steps) chunk.grad_out = nullptr;
+        if (s0 + chunk.num_steps < first_step + num_steps) { chunk.grad_out = nullptr; chunk.model_out = nullptr; }
         void* params[] = {&chunk};
         e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)plan.nb), dim3(kLeanThreads), params, plan.smem, ctx->stream);
         if (e != cudaSuccess) return cuda_status(e);

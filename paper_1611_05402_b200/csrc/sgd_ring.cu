@@ -444,6 +444,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 const int f = q * FPW + i;
                 xt[i] = (have && f < fcnt) ? a.x[j0 + f] : 0.0f;
                 if (a.model_bits > 0 && have) xt[i] = q3.apply(xt[i], (uint32_t)(j0 + f));
+                if (a.model_out && a.num_steps == 1 && bi == 0 && have && f < fcnt) a.model_out[j0 + f] = xt[i];
             }
             delta_w = word_stage(have, q, xt);
         }
@@ -998,6 +999,7 @@ __global__ void __launch_bounds__(kRingThreads, 1) sgd_ring_kernel(const SgdArgs
                 const int f = sub0 + k;
                 float xt = xown[k];
                 if (a.model_bits > 0 && f < fcnt) xt = q3.apply(xt, (uint32_t)(j0 + f));
+                if (a.model_out && it + 2 == a.first_step + a.num_steps && f < fcnt) a.model_out[j0 + f] = xt;
                 ll_store(ag_part + f, xt, tag);
             }
         }
@@ -1226,7 +1228,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
     a.row_words = d->row_bytes / 4;
     a.m = d->m; a.n = d->n; a.bits = d->bits;
     a.lo = d->feat_lo; a.step = d->feat_step; a.levels = d->levels;
-    a.b = b; a.x = x; a.grad_out = grad_out;
+    a.b = b; a.x = x; a.grad_out = grad_out; a.model_out = p->model_out;
     a.batch = B;
     a.first_step = first_step; a.num_steps = num_steps;
     a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
@@ -1268,7 +1270,7 @@ int launch_sgd_ring(zipml_ctx* ctx, const zipml_dataset* d, const float* b, floa
         SgdArgs chunk = a;
         chunk.first_step = s0;
         chunk.num_steps = (first_step + num_steps - s0 < max_steps) ? first_step + num_steps - s0 : max_steps;
-        if (s0 + chunk.num_steps < first_step + num_steps) chunk.grad_out = nullptr;
+        if (s0 + chunk.num_steps < first_step + num_steps) { chunk.grad_out = nullptr; chunk.model_out = nullptr; }
         void* params[] = {&chunk, &tmaps[0], &tmaps[1]};
         e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kRingThreads), params, plan.smem, ctx->stream);
         if (e != cudaSuccess) return cuda_status(e);

@@ -627,6 +627,9 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     if (d->n > (1 << 30) / 8) return ZIPML_ERR_WORKSPACE;
     const int cb = container_bits(d->bits);
     const int ng = 8 / cb, cw = kStreamBlock;
+    // (model_out: with an fp32 model the last step's gradient saw the model as it stood before that step; this
+    // engine keeps no copy of it, so the request is declined like the quantized model itself)
+    if (p->model_out) return ZIPML_ERR_WORKSPACE;
     const int64_t T = (d->m + p->batch - 1) / p->batch;
     const int64_t B = p->batch < d->m ? p->batch : d->m;
     if (B > kStreamMaxBatch) return ZIPML_ERR_WORKSPACE;
@@ -689,12 +692,12 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     a.ca = (int)ca; a.spans = (int)spans; a.part_spans = part_spans; a.bpc = (int)bpc; a.bpad = bpad;
     a.union_bytes = (int)uni; a.vec_bytes = vec_bytes;
     // The whole next tile where two tiles fit L2 with room to spare, a quarter of it where one and a half do
-    // (measured on 64 MB tiles in a 126 MB L2: 2/8 gains 3 %, 8/8 loses 6 %); ZIPML_STREAM_PREFETCH=0..8 overrides
+    // (measured on 64 MB tiles in a 126 MB L2: 2/8 gains 3 %, 8/8 loses 6 %); zipml_sgd_params.stream_prefetch overrides
     int l2_bytes = 0;
     cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, ctx->device);
     const int64_t step_bytes = 2 * B * rb;
     a.l2_prefetch = 9 * step_bytes <= 4 * (int64_t)l2_bytes ? 8 : 3 * step_bytes <= 2 * (int64_t)l2_bytes ? 2 : 0;
-    if (const char* env = getenv("ZIPML_STREAM_PREFETCH")) { a.l2_prefetch = atoi(env); if (a.l2_prefetch < 0 || a.l2_prefetch > 8) a.l2_prefetch = 0; }
+    if (p->stream_prefetch >= 1 && p->stream_prefetch <= 9) a.l2_prefetch = p->stream_prefetch - 1;    // the caller's choice
     a.barrier = reinterpret_cast<unsigned*>(ctx->ws + o_bar);
     a.ready = reinterpret_cast<unsigned*>(ctx->ws + o_ready);
     a.dots = reinterpret_cast<long long*>(ctx->ws + o_dots);

@@ -34,7 +34,7 @@ def test_host_only_helpers(lib):
     assert lib.zipml_row_bytes(10, 5) == 0 and lib.zipml_row_bytes(0, 4) == 0
     assert lib.zipml_strerror(0) == b"ok"
     assert b"non-finite" in lib.zipml_strerror(binding.ERR_NONFINITE)
-    assert C.sizeof(binding.CDataset) == 80 and C.sizeof(binding.CSgdParams) == 96
+    assert C.sizeof(binding.CDataset) == 80 and C.sizeof(binding.CSgdParams) == 120
 
 
 def test_no_device_is_an_error_not_a_fallback(lib):

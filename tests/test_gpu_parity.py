@@ -219,11 +219,10 @@ def test_sgd_epoch_parity(ctx, case, engine):
         assert rel(xb.cpu().numpy(), x_ref) <= MODEL_TOL
 
 
-@pytest.mark.parametrize("int8", ["0", "1"])
+@pytest.mark.parametrize("contraction", [1, 2], ids=["fp32", "int8"])
 @pytest.mark.parametrize("case", SGD_CASES[:5], ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}")
-def test_cluster_engine_both_contractions(ctx, case, int8, monkeypatch):
+def test_cluster_engine_both_contractions(ctx, case, contraction):
     """The cluster engine's fp32 and int8 tensor-core contractions, forced, against the oracle."""
-    monkeypatch.setenv("ZIPML_CLUSTER_INT8", int8)
     key, m, n, bits, batch, lr = case
     _, A, b, _ = workload(key, m, n, seed=3)
     ods = oracle.quantize(A, bits, seed=5)
@@ -235,13 +234,14 @@ def test_cluster_engine_both_contractions(ctx, case, int8, monkeypatch):
     _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=T - 1, num_steps=1, want_grad=True)
     for fb in (0, 3, 16):
         x = to_dev(x0, ctx)
-        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=binding.ENGINE_CLUSTER, grid_row_parts=fb)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=binding.ENGINE_CLUSTER, grid_row_parts=fb,
+                            cluster_contraction=contraction)
         ctx.zipml_sync()
         assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL, fb
         xb = to_dev(x_before, ctx)
         g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
         ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=T - 1, num_steps=1, engine=binding.ENGINE_CLUSTER,
-                            grid_row_parts=fb, grad_out=g)
+                            grid_row_parts=fb, grad_out=g, cluster_contraction=contraction)
         ctx.zipml_sync()
         assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL, fb
 
@@ -282,6 +282,79 @@ def test_stream_engine_wide_rows(ctx, case):
     # what it does not cover is declined, not approximated
     with pytest.raises(binding.ZipmlError) as e:
         ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=binding.ENGINE_STREAM, model_bits=8)
+    assert e.value.code == binding.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("case", [
+    # key, m, n, bits, batch, lr, chunk rows (0 = automatic)
+    ("c5", 700, 20000, 4, 300, 1e-4, 0),          # 79 column blocks, the last one partly past the row; ragged batches
+    ("c5", 1500, 30001, 4, 640, 1e-4, 64),        # several chunks per step, n odd
+    ("c2", 1300, 9001, 8, 520, 1e-3, 0),
+    ("c3", 1100, 40000, 2, 500, 5e-4, 96),
+    ("c4u", 900, 12345, 3, 333, 1e-3, 256),
+    ("c2", 400, 300, 8, 100, 1e-3, 32),           # three CTAs only
+], ids=lambda c: f"{c[0]}-{c[1]}x{c[2]}-b{c[3]}-B{c[4]}-R{c[6]}")
+def test_column_engine(ctx, case):
+    """The column engine (a CTA per 128-byte column block, codes read once per step): model after an epoch in a
+    permuted batch order from a zero and a non-zero model, bit-identical repeats, last-step gradient, split calls."""
+    key, m, n, bits, batch, lr, chunk = case
+    _, A, b, _ = workload(key, m, n, seed=8)
+    ods = oracle.quantize(A, bits, seed=9)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    T = (m + batch - 1) // batch
+    order = np.random.default_rng(5).permutation(T).astype(np.int32)
+    kw = dict(engine=binding.ENGINE_COLUMN, column_chunk_rows=chunk, batch_order=order)
+    for x0 in (np.zeros(n, np.float32), (np.random.default_rng(4).standard_normal(n) * 0.05).astype(np.float32)):
+        x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order)
+        x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order, num_steps=T - 1)
+        _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, batch_order=order, first_step=T - 1, num_steps=1, want_grad=True)
+        runs = []
+        for _ in range(2):
+            x = to_dev(x0, ctx)
+            ctx.zipml_sgd_epoch(gds, db, x, batch, lr, **kw)
+            ctx.zipml_sync()
+            assert ctx.zipml_last_engine() == binding.ENGINE_COLUMN
+            runs.append(x.cpu().numpy())
+            assert rel(runs[-1], x_ref) <= MODEL_TOL
+        assert (runs[0] == runs[1]).all()                 # integer sums and fixed orders: the same bits run to run
+        xb = to_dev(x_before, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=T - 1, num_steps=1, grad_out=g, **kw)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL and (g[0] == g[1]).all()
+        assert rel(xb.cpu().numpy(), x_ref) <= MODEL_TOL
+        if T >= 3:                                        # an epoch in two calls
+            x = to_dev(x0, ctx)
+            ctx.zipml_sgd_epoch(gds, db, x, batch, lr, first_step=0, num_steps=2, **kw)
+            ctx.zipml_sgd_epoch(gds, db, x, batch, lr, first_step=2, **kw)
+            ctx.zipml_sync()
+            assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    # what it does not cover is declined, not approximated
+    for bad in (dict(model_bits=8), dict(grad_bits=8), dict(model_out=torch.zeros(n, device=ctx.device))):
+        with pytest.raises(binding.ZipmlError) as e:
+            ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=binding.ENGINE_COLUMN, **bad)
+        assert e.value.code == binding.ERR_WORKSPACE
+
+
+def test_column_engine_limits(ctx):
+    """Rows narrower than one column block, rows wider than one block per SM and batches above 8,192 are declined."""
+    _, A, b, _ = workload("c1", 200, 64, seed=1)
+    gds, db = dev_dataset(oracle.quantize(A, 4, seed=1), ctx), to_dev(b, ctx)
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, torch.zeros(64, device=ctx.device), 16, 0.01, engine=binding.ENGINE_COLUMN)
+    assert e.value.code == binding.ERR_WORKSPACE
+    m, n = 8300, 10240
+    _, A, b, _ = workload("c5", m, n, seed=11)
+    ods = oracle.quantize(A, 4, seed=12)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = np.zeros(n, np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 8192, 1e-4)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 8192, 1e-4, engine=binding.ENGINE_COLUMN)
+    ctx.zipml_sync()
+    assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), 8193, 1e-4, engine=binding.ENGINE_COLUMN)
     assert e.value.code == binding.ERR_WORKSPACE
 
 
@@ -349,45 +422,122 @@ def test_sgd_table_levels_parity(ctx):
     assert rel(g[0].cpu().numpy(), g1[0]) <= GRAD_TOL
 
 
+def q3_margins(x, bits, seed, epoch, step):
+    """|u 2^-24 - p| of every coordinate's Q3 rounding decision (Supplement Eq. (quant2) with M = ||x||_2), from
+    the oracle's own random integers; the arithmetic mirrors the quantizer's fp32 steps only to *classify*
+    coordinates (which ones a sub-ulp difference in M could flip), never to produce an expected value."""
+    sm = np.float32((1 << (bits - 1)) - 1)
+    M = np.float32(np.sqrt(np.sum(x.astype(np.float64) ** 2)))
+    t = (np.abs(x) / M).astype(np.float32) * sm
+    fl = np.minimum(np.floor(t), sm - 1).astype(np.float32)
+    p = (t - fl).astype(np.float32)
+    u = np.array([oracle.u24_vector(seed, epoch, step, j, 3) for j in range(x.shape[0])], np.float64) * 2.0 ** -24
+    return np.abs(u - p.astype(np.float64)), float(M / sm)
+
+
+E2E_ENGINES = [
+    # engine, cluster_contraction, id
+    (binding.ENGINE_STEPWISE, 0), (binding.ENGINE_PERSISTENT, 0), (binding.ENGINE_RING, 0), (binding.ENGINE_LEAN, 0),
+    (binding.ENGINE_CLUSTER, 1), (binding.ENGINE_CLUSTER, 2), (binding.ENGINE_AUTO, 0),
+]
+
+
 @pytest.mark.parametrize("model_bits,grad_bits", [(8, 0), (0, 8), (8, 8), (4, 4)])
-def test_sgd_end_to_end_quantization(ctx, model_bits, grad_bits):
-    _, A, b, _ = workload("c3", 3000, 512, seed=6)
+@pytest.mark.parametrize("shape", [(3000, 512), (3000, 2048)], ids=["n512", "c3-n2048"])
+def test_sgd_end_to_end_quantization(ctx, shape, model_bits, grad_bits):
+    """Q3 / Q4 (Supplement "Quantizing the Model", "Quantizing the Gradients", "End-to-end Quantization") on 2-bit
+    data with B = 1024; the second shape is config 3's own step (n = 2,048: 64 rows x 512 B per CTA, where AUTO
+    runs the cluster engine's int8 contraction) and both contractions of the cluster engine are forced."""
+    m, n = shape
+    _, A, b, _ = workload("c3", m, n, seed=6)
     ods = oracle.quantize(A, 2, seed=2)
     gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
-    x0 = (np.random.default_rng(3).standard_normal(512) * 0.05).astype(np.float32)
-    # one step from identical x: the pre-Q4 gradient must agree to GRAD_TOL; the quantized
-    # quantities must agree exactly except where a stochastic rounding sits within 1e-4 of its
-    # threshold (a sub-ulp difference in the norm may flip those)
-    _, g_ref = oracle.sgd_epoch(ods, b, x0, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
-                                first_step=1, num_steps=1, want_grad=True)
-    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER):
+    x0 = (np.random.default_rng(3).standard_normal(n) * 0.05).astype(np.float32)
+    seed, epoch, step = 11, 2, 1
+    # what the model quantizer must produce from x0, and how close each of its decisions is to its threshold
+    if model_bits:
+        xq_ref, _ = oracle.quantize_vector(x0, model_bits, seed, epoch, step, 3)
+        margin, unit_x = q3_margins(x0, model_bits, seed, epoch, step)
+    else:
+        xq_ref = x0
+    for engine, contraction in E2E_ENGINES:
         x = to_dev(x0, ctx)
-        g = torch.zeros((2, 512), dtype=torch.float32, device=ctx.device)
-        ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
-                            first_step=1, num_steps=1, engine=engine, grad_out=g)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        xq = torch.zeros(n, dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=seed, epoch=epoch,
+                            first_step=step, num_steps=1, engine=engine, grad_out=g, model_out=xq,
+                            cluster_contraction=contraction)
         ctx.zipml_sync()
-        gg = g.cpu().numpy()
-        if model_bits == 0:
-            assert rel(gg[0], g_ref[0]) <= GRAD_TOL
+        if engine == binding.ENGINE_AUTO and n == 2048:
+            assert ctx.zipml_last_engine() == binding.ENGINE_CLUSTER
+        gg, xq = g.cpu().numpy(), xq.cpu().numpy()
+        # Q3: the quantized model agrees exactly, except where a rounding sits within 1e-4 of its threshold
+        # (a last-bit difference in ||x||_2 may flip those: by one quantization unit, and only a few)
+        differs = xq != xq_ref
+        if model_bits:
+            assert not (differs & (margin >= 1e-4)).any(), (engine, contraction)
+            assert differs.sum() <= 3 and (np.abs(xq - xq_ref)[differs] <= 1.001 * unit_x).all()
         else:
-            # a flipped model coordinate changes the gradient by about |a_j|*|step|: allow a few
-            assert rel(gg[0], g_ref[0]) <= 5e-3
+            assert not differs.any()
+        # the gradient before Q4, held to the plain bar against the oracle run from the very model the kernel used
+        _, g_ref = oracle.sgd_epoch(ods, b, xq, 1024, 5e-4, model_bits=0, grad_bits=grad_bits, seed=seed, epoch=epoch,
+                                    first_step=step, num_steps=1, want_grad=True)
+        assert rel(gg[0], g_ref[0]) <= GRAD_TOL, (engine, contraction)
         if grad_bits:
             sm = (1 << (grad_bits - 1)) - 1
             unit = np.linalg.norm(g_ref[0]) / sm
             flips = np.abs(gg[1] - g_ref[1]) > 0.5 * unit
             assert flips.sum() <= 3
             assert np.abs(gg[1] - g_ref[1])[~flips].max() <= 1e-5 * unit + 1e-12
-    # whole epoch: the trajectories stay together within the model tolerance
+        else:
+            assert (gg[0] == gg[1]).all()
+    # whole epoch: the trajectories stay together (a rare flipped rounding moves one coordinate by one unit)
     x_ref, _ = oracle.sgd_epoch(ods, b, x0, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2)
+    for contraction in (1, 2):
+        x = to_dev(x0, ctx)
+        ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2,
+                            cluster_contraction=contraction)
+        ctx.zipml_sync()
+        assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
+
+
+def test_ring_engine_int8_path_with_quantized_model_and_gradient(ctx):
+    """The ring engine's tensor-core contraction (uniform grid, tiles of 32-row chunks) under Q3 and Q4, on a
+    step too large for one cluster: 2-bit codes, n = 8,192 (2 KB rows), B = 2,048."""
+    m, n, batch = 4200, 8192, 2048
+    _, A, b, _ = workload("c3", m, n, seed=7)
+    ods = oracle.quantize(A, 2, seed=4)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = (np.random.default_rng(5).standard_normal(n) * 0.02).astype(np.float32)
+    seed, epoch, step = 21, 1, 1
+    xq_ref, _ = oracle.quantize_vector(x0, 8, seed, epoch, step, 3)
+    margin, unit_x = q3_margins(x0, 8, seed, epoch, step)
+    for engine in (binding.ENGINE_RING, binding.ENGINE_AUTO):
+        x = to_dev(x0, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        xq = torch.zeros(n, dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, 5e-4, model_bits=8, grad_bits=8, seed=seed, epoch=epoch, first_step=step,
+                            num_steps=1, engine=engine, grad_out=g, model_out=xq)
+        ctx.zipml_sync()
+        assert ctx.zipml_last_engine() == binding.ENGINE_RING
+        gg, xq = g.cpu().numpy(), xq.cpu().numpy()
+        differs = xq != xq_ref
+        assert not (differs & (margin >= 1e-4)).any() and differs.sum() <= 3
+        _, g_ref = oracle.sgd_epoch(ods, b, xq, batch, 5e-4, model_bits=0, grad_bits=8, seed=seed, epoch=epoch,
+                                    first_step=step, num_steps=1, want_grad=True)
+        assert rel(gg[0], g_ref[0]) <= GRAD_TOL
+        unit = np.linalg.norm(g_ref[0]) / 127
+        flips = np.abs(gg[1] - g_ref[1]) > 0.5 * unit
+        assert flips.sum() <= 3 and np.abs(gg[1] - g_ref[1])[~flips].max() <= 1e-5 * unit + 1e-12
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, 5e-4, model_bits=8, grad_bits=8, seed=seed, epoch=epoch)
     x = to_dev(x0, ctx)
-    ctx.zipml_sgd_epoch(gds, db, x, 1024, 5e-4, model_bits=model_bits, grad_bits=grad_bits, seed=11, epoch=2)
+    ctx.zipml_sgd_epoch(gds, db, x, batch, 5e-4, model_bits=8, grad_bits=8, seed=seed, epoch=epoch, engine=binding.ENGINE_RING)
     ctx.zipml_sync()
     assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
 
 
 def test_auto_picks_the_engine_that_fits(ctx):
-    """AUTO: cluster for small steps, stream for large uniform fp32 steps on wide rows, ring where stream declines."""
+    """AUTO: cluster for small steps, column (else stream) for large uniform fp32 steps on wide rows, ring where they decline."""
     _, A, b, _ = workload("c5", 700, 20000, seed=2)                 # 2 x 300 rows x 10 KB: 6 MB per step, 157 column blocks
     ods = oracle.quantize(A, 4, seed=2)
     gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
@@ -396,7 +546,12 @@ def test_auto_picks_the_engine_that_fits(ctx):
     x = to_dev(x0, ctx)
     ctx.zipml_sgd_epoch(gds, db, x, 300, 1e-4)
     ctx.zipml_sync()
-    assert ctx.zipml_last_engine() == binding.ENGINE_STREAM and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    assert ctx.zipml_last_engine() == binding.ENGINE_COLUMN and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    x_small, _ = oracle.sgd_epoch(ods, b, x0, 100, 1e-4)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, 100, 1e-4)                               # short steps: the stream engine's
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() == binding.ENGINE_STREAM and rel(x.cpu().numpy(), x_small) <= MODEL_TOL
     x = to_dev(x0, ctx)
     ctx.zipml_sgd_epoch(gds, db, x, 300, 1e-4, grad_bits=8, seed=3)          # quantized gradient: not the stream engine's
     ctx.zipml_sync()
@@ -428,8 +583,11 @@ def test_sgd_regularised_update_parity(ctx, case, reg, param):
         assert (x_ref == 0).any() and (x_ref != 0).any()            # the threshold bites somewhere, not everywhere
     if reg == binding.REG_NONNEG:
         assert (x_ref >= 0).all() and ((x_ref == 0).any() or key == "c5")  # (c5's large first gradients lift every coordinate)
-    for engine in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER,
-                   binding.ENGINE_STREAM, binding.ENGINE_AUTO):
+    engines = [binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT, binding.ENGINE_RING, binding.ENGINE_LEAN, binding.ENGINE_CLUSTER,
+               binding.ENGINE_STREAM, binding.ENGINE_AUTO]
+    if gds.row_bytes >= 128:
+        engines.append(binding.ENGINE_COLUMN)
+    for engine in engines:
         x = to_dev(x0, ctx)
         g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
         ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=engine, reg=reg, reg_param=param, grad_out=g)
@@ -497,6 +655,120 @@ def test_loss_codes_with_level_table_and_strided_dense(ctx):
     ctx.zipml_sync()
     assert abs(got_c.item() - want_c) <= LOSS_TOL * abs(want_c)
     assert abs(got.item() - oracle.loss_dense(A, b, xs)) <= LOSS_TOL * oracle.loss_dense(A, b, xs)
+
+
+def test_loss_codes_with_a_stride_far_above_the_minimum(ctx):
+    """Planes that are column slices of a wider packed matrix: the row stride, not n, sizes what the loss stages."""
+    _, A, b, xs = workload("c3", 200, 100, seed=5)
+    ods = oracle.quantize(A, 2, seed=6)
+    want_c = oracle.loss_codes(ods, b, xs)
+    stride = 80 * 1024
+    wide1 = torch.zeros((200, stride), dtype=torch.uint8, device=ctx.device)
+    wide2 = torch.zeros((200, stride), dtype=torch.uint8, device=ctx.device)
+    wide1[:, : ods.row_bytes] = to_dev(ods.plane1, ctx)
+    wide2[:, : ods.row_bytes] = to_dev(ods.plane2, ctx)
+    gds = binding.Dataset(wide1, wide2, 200, 100, 2, binding.LEVELS_UNIFORM, to_dev(ods.feat_lo, ctx), to_dev(ods.feat_step, ctx), None)
+    with binding.Context(ctx.device) as fresh:                     # a context whose workspace has not grown yet
+        got_c = fresh.zipml_loss(binding.LOSS_CODES, to_dev(b, ctx), to_dev(xs, ctx), data=gds)
+        fresh.zipml_sync()
+    assert abs(got_c.item() - want_c) <= LOSS_TOL * abs(want_c)
+
+
+# ---------------------------------------------------------------------------------------------
+# the configurations at their own step shapes (a few minibatches of rows)
+# ---------------------------------------------------------------------------------------------
+def test_config5_step_shape(ctx):
+    """Config 5 as it runs: n = 32,768 (16 KB packed rows), 4-bit, B = 2,048; two full minibatches and a ragged one.
+    Planes bit-exact, then the engine AUTO picks for this shape: model after the epoch and the last step's gradient."""
+    m, n, batch, lr = 2 * 2048 + 1000, 32768, 2048, 1e-4
+    _, A, b, _ = workload("c5", m, n, seed=0)
+    ods = oracle.quantize(A, 4, seed=0)
+    dA = to_dev(A, ctx)
+    gds = ctx.zipml_quantize(dA, 4, seed=0)
+    ctx.zipml_sync()
+    del dA
+    assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all() and (gds.feat_step.cpu().numpy() == ods.feat_step).all()
+    assert (gds.plane1.cpu().numpy() == ods.plane1).all() and (gds.plane2.cpu().numpy() == ods.plane2).all()
+    db = to_dev(b, ctx)
+    x0 = np.zeros(n, np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr)
+    x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, num_steps=2)
+    _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=2, num_steps=1, want_grad=True)
+    for engine in (binding.ENGINE_AUTO, binding.ENGINE_STREAM, binding.ENGINE_COLUMN):
+        x = to_dev(x0, ctx)
+        ctx.zipml_sgd_epoch(gds, db, x, batch, lr, engine=engine)
+        ctx.zipml_sync()
+        if engine == binding.ENGINE_AUTO:
+            assert ctx.zipml_last_engine() == binding.ENGINE_COLUMN
+        assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL, engine
+        xb = to_dev(x_before, ctx)
+        g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=2, num_steps=1, grad_out=g, engine=engine)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL, engine
+        # the full step before it too (2,048 rows)
+        _, g_full = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=1, num_steps=1, want_grad=True)
+        xb = to_dev(x_before, ctx)
+        ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=1, num_steps=1, grad_out=g, engine=engine)
+        ctx.zipml_sync()
+        assert rel(g[0].cpu().numpy(), g_full[0]) <= GRAD_TOL, engine
+    want = oracle.loss_codes(ods, b, x_ref)
+    got = ctx.zipml_loss(binding.LOSS_CODES, db, to_dev(x_ref, ctx), data=gds)
+    ctx.zipml_sync()
+    assert abs(got.item() - want) <= LOSS_TOL * max(abs(want), oracle.loss_dense(A, b, x_ref))
+
+
+def test_config4_step_shape_with_level_table(ctx):
+    """Config 4 as it runs: n = 512, 3-bit variance-optimal levels from a 1,024-bin histogram, B = 512."""
+    m, n, batch, lr = 3 * 512 + 100, 512, 512, 1e-3
+    _, A, b, _ = workload("c4", m, n, seed=0)
+    lev, obj = oracle.optimal_levels(A, 3, 1024)
+    ods = oracle.quantize(A, 3, seed=0, mode=oracle.TABLE, levels=lev)
+    dA = to_dev(A, ctx)
+    glev, gobj = ctx.zipml_optimal_levels(dA, 3, 1024, want_objective=True)
+    gds = ctx.zipml_quantize(dA, 3, seed=0, level_mode=binding.LEVELS_TABLE, levels=glev)
+    ctx.zipml_sync()
+    assert (glev.cpu().numpy() == lev).all() and (gobj.cpu().numpy().astype(np.uint64) == obj).all()
+    assert (gds.plane1.cpu().numpy() == ods.plane1).all() and (gds.plane2.cpu().numpy() == ods.plane2).all()
+    db = to_dev(b, ctx)
+    x0 = np.zeros(n, np.float32)
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr)
+    x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, num_steps=2)
+    _, g_ref = oracle.sgd_epoch(ods, b, x_before, batch, lr, first_step=2, num_steps=1, want_grad=True)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, batch, lr)
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() == binding.ENGINE_CLUSTER and rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    xb = to_dev(x_before, ctx)
+    g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=2, num_steps=1, grad_out=g)
+    ctx.zipml_sync()
+    assert rel(g[0].cpu().numpy(), g_ref[0]) <= GRAD_TOL
+    want = oracle.loss_codes(ods, b, x_ref)
+    got = ctx.zipml_loss(binding.LOSS_CODES, db, to_dev(x_ref, ctx), data=gds)
+    ctx.zipml_sync()
+    assert abs(got.item() - want) <= LOSS_TOL * max(abs(want), oracle.loss_dense(A, b, x_ref))
+
+
+def test_quantize_rows_more_than_2_to_31_elements_apart(ctx):
+    """A strided view whose last row starts beyond element 2^31 of its buffer: row * lda must be 64-bit arithmetic."""
+    m, n, lda = 4, 300, 800_000_000
+    _, A, _, _ = workload("c2", m, n, seed=4)
+    big = torch.empty((m - 1) * lda + n, dtype=torch.float32, device=ctx.device)     # 9.6 GB, touched only at the rows
+    view = big.as_strided((m, n), (lda, 1))
+    view.copy_(to_dev(A, ctx))
+    ods = oracle.quantize(A, 8, seed=77)
+    gds = ctx.zipml_quantize(view, 8, seed=77)
+    ctx.zipml_sync()
+    assert (gds.feat_lo.cpu().numpy() == ods.feat_lo).all() and (gds.feat_step.cpu().numpy() == ods.feat_step).all()
+    assert (gds.plane1.cpu().numpy() == ods.plane1).all() and (gds.plane2.cpu().numpy() == ods.plane2).all()
+    lev, _ = oracle.optimal_levels(A, 2, 64)
+    glev = ctx.zipml_optimal_levels(view, 2, 64)
+    want = oracle.loss_dense(A, np.ones(m, np.float32), np.ones(n, np.float32))
+    got = ctx.zipml_loss(binding.LOSS_DENSE, torch.ones(m, device=ctx.device), torch.ones(n, device=ctx.device), A=view)
+    ctx.zipml_sync()
+    assert (glev.cpu().numpy() == lev).all() and abs(got.item() - want) <= LOSS_TOL * want
+    del big, view
 
 
 # ---------------------------------------------------------------------------------------------
