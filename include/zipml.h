@@ -43,6 +43,13 @@ enum {
 };
 
 enum { ZIPML_LEVELS_UNIFORM = 0, ZIPML_LEVELS_TABLE = 1 };
+/* How a plane lies in memory.  ROWS is the layout described above and the one every call produces and
+ * accepts.  COLUMN_BLOCKS is a rearrangement for zipml_sgd_epoch's column engine (made and undone by
+ * zipml_convert_layout, bit for bit): the plane is cut into blocks of 128 bytes of the row, block j
+ * (bytes 128 j .. 128 j + 127 of every row, zero where the row has ended) stored as m consecutive
+ * pieces of 128 bytes: piece (j, k) of row k at byte (j * m + k) * 128.  A plane then takes
+ * zipml_column_blocks_bytes(m, row_bytes) bytes; row_bytes still names the row-major stride it came from. */
+enum { ZIPML_LAYOUT_ROWS = 0, ZIPML_LAYOUT_COLUMN_BLOCKS = 1 };
 enum { ZIPML_LOSS_DENSE = 0, ZIPML_LOSS_CODES = 1 };
 /* Regulariser of zipml_sgd_epoch (paper Eq. (proxupdate): x <- prox_{lr R}(x - lr g), the proximal
  * operator taken coordinate by coordinate on y = x - lr g; and the Supplement's least-squares SVM,
@@ -82,10 +89,12 @@ enum {
     ZIPML_ENGINE_COLUMN = 7      /* one cooperative launch for large tiles on uniform grids with an fp32
                                     model and gradient, rows of 128 bytes .. 128 bytes x the number of
                                     SMs: a CTA owns a 128-byte column block of the packed rows for the
-                                    whole launch; rows travel through shared memory in chunks that
-                                    serve both passes of the step, so the codes are read from HBM once
-                                    per step; CTAs exchange only the rows' dots (integer atomics and one
-                                    counter per chunk), there is no grid-wide barrier.
+                                    whole launch; chunks of rows visit shared memory once for the dots
+                                    and once more, out of L2, for the gradient, so the codes are read
+                                    from HBM once per step; CTAs exchange only the rows' dots (integer
+                                    atomics that count their own completion), there is no grid-wide
+                                    barrier.  The only engine that takes ZIPML_LAYOUT_COLUMN_BLOCKS
+                                    (where its copies are contiguous; AUTO picks it for such data).
                                     ZIPML_ERR_WORKSPACE for what it does not cover (as for STREAM)     */
 };
 
@@ -96,7 +105,7 @@ typedef struct zipml_dataset {
     uint32_t struct_size;   /* sizeof(zipml_dataset), for ABI evolution                              */
     int32_t bits;           /* 2, 3, 4 or 8                                                          */
     int32_t level_mode;     /* ZIPML_LEVELS_UNIFORM or ZIPML_LEVELS_TABLE                            */
-    int32_t reserved;
+    int32_t layout;         /* ZIPML_LAYOUT_ROWS, or ZIPML_LAYOUT_COLUMN_BLOCKS (zipml_sgd_epoch only)         */
     int64_t m, n;           /* samples, features                                                     */
     int64_t row_bytes;      /* stride of both planes                                                 */
     const uint8_t* plane1;  /* m * row_bytes bytes, 16-byte aligned                                  */
@@ -135,7 +144,13 @@ typedef struct zipml_sgd_params {
                                    mark 4.  Stream engine: 0 step start, 1 own dots added, 2 barrier
                                    passed, 3 residual digits ready, 4 own gradient blocks summed,
                                    5 model updated and digits published, 6 dots and labels read,
-                                   7 residual scale known.  Other engines ignore the request.         */
+                                   7 residual scale known.  Column engine (the buffer must be zeroed):
+                                   0 clock at the step's first dots, 7 clock when the next w is out;
+                                   cycles that warp 0 of a role spent waiting in the step: 1 A warp
+                                   for first-visit copies, 2 R warp for complete dots (of its chunks),
+                                   3 R warp for its digit buffer, 4 B warp for digits, 5 B warp for
+                                   second-visit copies; 6 cycles of the step-end update.  Other engines
+                                   ignore the request.                                               */
     int32_t reg;                /* ZIPML_REG_*                                                       */
     float reg_param;            /* c or lambda (>= 0); ignored by ZIPML_REG_NONE and _NONNEG          */
     float* model_out;           /* debug, DEVICE pointer or NULL: n floats, the model that the last
@@ -148,7 +163,8 @@ typedef struct zipml_sgd_params {
     int32_t stream_prefetch;    /* tuning, stream engine: 0 = automatic, 1..9 = request (value - 1)
                                    eighths of the next step's tile into L2 ahead of time             */
     int32_t column_chunk_rows;  /* tuning, column engine: 0 = automatic, else rows of a minibatch that
-                                   travel through shared memory together (a multiple of 32, 32..256)  */
+                                   travel through shared memory together (a multiple of 32; values
+                                   above 128 count as 128)                                            */
     int32_t reserved0;          /* must be 0                                                         */
 } zipml_sgd_params;
 
@@ -178,6 +194,16 @@ int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, 
 int zipml_wait_probe(zipml_ctx* ctx, int64_t spin_limit);
 /* Smallest legal row stride for n features: ceil(n*cb/8) rounded up to 16; 0 if bits is unsupported. */
 int64_t zipml_row_bytes(int64_t n, int32_t bits);
+/* Bytes of one plane of m rows with row stride row_bytes in the ZIPML_LAYOUT_COLUMN_BLOCKS layout. */
+int64_t zipml_column_blocks_bytes(int64_t m, int64_t row_bytes);
+
+/* Rearranges both planes of `data` into the other layout (the packed layout is not fixed by the paper: the
+ * Supplement's FPGA section only says that the pipeline consumes 64-byte lines; a column engine wants each
+ * CTA's share of a minibatch contiguous in memory).  `data` is in the layout its `layout` field names; out1
+ * and out2 (16-byte aligned, m * row_bytes bytes for ROWS, zipml_column_blocks_bytes for COLUMN_BLOCKS, not
+ * overlapping the inputs) receive planes 1 and 2 in `to_layout`.  Converting there and back gives the
+ * original bytes. */
+int zipml_convert_layout(zipml_ctx* ctx, const zipml_dataset* data, int32_t to_layout, uint8_t* out1, uint8_t* out2);
 
 /* Stochastic quantization with double sampling (paper Section 2.1, Eq. (double); Supplement
  * "Randomized Quantization", "Column Scaling").

@@ -13,11 +13,12 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
+LAYOUT_ROWS, LAYOUT_COLUMN_BLOCKS = 0, 1
 REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM, ENGINE_COLUMN = 0, 1, 2, 3, 4, 5, 6, 7
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -33,7 +34,7 @@ class ZipmlError(RuntimeError):
 
 
 class CDataset(C.Structure):
-    _fields_ = [("struct_size", C.c_uint32), ("bits", C.c_int32), ("level_mode", C.c_int32), ("reserved", C.c_int32),
+    _fields_ = [("struct_size", C.c_uint32), ("bits", C.c_int32), ("level_mode", C.c_int32), ("layout", C.c_int32),
                 ("m", C.c_int64), ("n", C.c_int64), ("row_bytes", C.c_int64),
                 ("plane1", C.c_void_p), ("plane2", C.c_void_p),
                 ("feat_lo", C.c_void_p), ("feat_step", C.c_void_p), ("levels", C.c_void_p)]
@@ -73,6 +74,9 @@ def lib():
         L.zipml_strerror.restype = C.c_char_p
         L.zipml_row_bytes.argtypes = [i64, i32]
         L.zipml_row_bytes.restype = i64
+        L.zipml_column_blocks_bytes.argtypes = [i64, i64]
+        L.zipml_column_blocks_bytes.restype = i64
+        L.zipml_convert_layout.argtypes = [vp, C.POINTER(CDataset), i32, vp, vp]
         L.zipml_quantize.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
         L.zipml_optimal_levels.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp]
         L.zipml_sgd_epoch.argtypes = [vp, C.POINTER(CDataset), vp, vp, C.POINTER(CSgdParams), vp]
@@ -103,16 +107,18 @@ def _ptr(t, dtype=None, device=None):
 class Dataset:
     """Two packed planes plus scales/levels, all torch tensors on the context's device."""
 
-    def __init__(self, plane1, plane2, m, n, bits, level_mode, feat_lo, feat_step, levels):
+    def __init__(self, plane1, plane2, m, n, bits, level_mode, feat_lo, feat_step, levels, layout=LAYOUT_ROWS,
+                 row_bytes=None):
         self.plane1, self.plane2 = plane1, plane2
-        self.m, self.n, self.bits, self.level_mode = m, n, bits, level_mode
-        self.row_bytes = plane1.shape[1]
+        self.m, self.n, self.bits, self.level_mode, self.layout = m, n, bits, level_mode, layout
+        self.row_bytes = plane1.shape[1] if row_bytes is None else row_bytes
         self.feat_lo, self.feat_step, self.levels = feat_lo, feat_step, levels
 
     def c_struct(self):
         d = CDataset()
         d.struct_size = C.sizeof(CDataset)
         d.bits, d.level_mode, d.m, d.n, d.row_bytes = self.bits, self.level_mode, self.m, self.n, self.row_bytes
+        d.layout = self.layout
         d.plane1, d.plane2 = self.plane1.data_ptr(), self.plane2.data_ptr()
         d.feat_lo = self.feat_lo.data_ptr() if self.feat_lo is not None else None
         d.feat_step = self.feat_step.data_ptr() if self.feat_step is not None else None
@@ -194,6 +200,20 @@ class Context:
                                     _ptr(levels, torch.float32, self.device), seed, _ptr(p1), _ptr(p2), rb, _ptr(lo),
                                     _ptr(step)), "zipml_quantize")
         return Dataset(p1, p2, m, n, bits, level_mode, lo, step, levels)
+
+    def zipml_convert_layout(self, data, to_layout):
+        """A new Dataset with both planes in `to_layout` (scales and levels are shared with `data`)."""
+        if to_layout == LAYOUT_COLUMN_BLOCKS:
+            nbytes = int(lib().zipml_column_blocks_bytes(data.m, data.row_bytes))
+            p1 = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            p2 = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        else:
+            p1 = torch.empty((data.m, data.row_bytes), dtype=torch.uint8, device=self.device)
+            p2 = torch.empty((data.m, data.row_bytes), dtype=torch.uint8, device=self.device)
+        d = data.c_struct()
+        _check(lib().zipml_convert_layout(self._h, C.byref(d), to_layout, _ptr(p1), _ptr(p2)), "zipml_convert_layout")
+        return Dataset(p1, p2, data.m, data.n, data.bits, data.level_mode, data.feat_lo, data.feat_step, data.levels,
+                       layout=to_layout, row_bytes=data.row_bytes)
 
     def zipml_optimal_levels(self, A, bits, hist_bins=1024, want_objective=False):
         m, n = A.shape

@@ -46,6 +46,7 @@ int check_dataset(const zipml_dataset* d) {
     const int cb = container_bits(d->bits);
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
     if (d->level_mode != ZIPML_LEVELS_UNIFORM && d->level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
+    if (d->layout != ZIPML_LAYOUT_ROWS && d->layout != ZIPML_LAYOUT_COLUMN_BLOCKS) return ZIPML_ERR_INVALID_ARG;
     if (d->level_mode == ZIPML_LEVELS_TABLE && d->bits == 8) return ZIPML_ERR_UNSUPPORTED;
     if (d->m <= 0 || d->n <= 0) return ZIPML_ERR_INVALID_ARG;
     if (d->n > 0x7fffffffLL / 8) return ZIPML_ERR_WORKSPACE;
@@ -90,6 +91,25 @@ const char* zipml_strerror(int status) {
         case ZIPML_ERR_WORKSPACE: return "problem does not fit the kernels' shared memory or scratch limits";
         default: return "unknown status";
     }
+}
+
+int64_t zipml_column_blocks_bytes(int64_t m, int64_t row_bytes) {
+    if (m <= 0 || row_bytes <= 0) return 0;
+    return (row_bytes + 127) / 128 * m * 128;
+}
+
+int zipml_convert_layout(zipml_ctx* ctx, const zipml_dataset* data, int32_t to_layout, uint8_t* out1, uint8_t* out2) {
+    if (!ctx) return ZIPML_ERR_INVALID_ARG;
+    int rc = check_dataset(data);
+    if (rc != ZIPML_OK) return rc;
+    if (to_layout != ZIPML_LAYOUT_ROWS && to_layout != ZIPML_LAYOUT_COLUMN_BLOCKS) return ZIPML_ERR_INVALID_ARG;
+    if (to_layout == data->layout) return ZIPML_ERR_INVALID_ARG;
+    if (!out1 || !out2 || !aligned16(out1) || !aligned16(out2)) return ZIPML_ERR_INVALID_ARG;
+    if (out1 == data->plane1 || out1 == data->plane2 || out2 == data->plane1 || out2 == data->plane2 || out1 == out2)
+        return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    return launch_convert_layout(ctx, data, to_layout, out1, out2);
 }
 
 int64_t zipml_row_bytes(int64_t n, int32_t bits) {
@@ -231,6 +251,11 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (count == 0) return ZIPML_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
+    if (data->layout == ZIPML_LAYOUT_COLUMN_BLOCKS) {                 // the column engine's own layout
+        if (params->engine != ZIPML_ENGINE_AUTO && params->engine != ZIPML_ENGINE_COLUMN) return ZIPML_ERR_UNSUPPORTED;
+        rc = launch_sgd_column(ctx, data, b, x, params, first, count, grad_out, false);
+        return rc == ZIPML_ERR_WORKSPACE ? ZIPML_ERR_UNSUPPORTED : rc;
+    }
     if (params->engine == ZIPML_ENGINE_RING) return launch_sgd_ring(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_LEAN) return launch_sgd_lean(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
@@ -295,6 +320,7 @@ int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t 
     }
     int rc = check_dataset(data);
     if (rc != ZIPML_OK) return rc;
+    if (data->layout != ZIPML_LAYOUT_ROWS) return ZIPML_ERR_UNSUPPORTED;
     // behind the partials: the level * x table, or (uniform grids) the digit vectors of step * x, which follow the
     // packed row byte for byte and so take their size from the stride, not from n
     const size_t tab = data->level_mode == ZIPML_LEVELS_TABLE

@@ -96,6 +96,8 @@ int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
 // Column engine (uniform grids, fp32 model and gradient, rows of at most 128 bytes per SM).
 int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                       int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
+// Both planes of d into the other layout (see ZIPML_LAYOUT_* in zipml.h).
+int launch_convert_layout(zipml_ctx* ctx, const zipml_dataset* d, int to_layout, uint8_t* out1, uint8_t* out2);
 int launch_barrier_latency(zipml_ctx* ctx, int ctas, int floats, int iterations, unsigned long long* ns_out_dev);
 int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                      int64_t first_step, int64_t num_steps, float* grad_out);

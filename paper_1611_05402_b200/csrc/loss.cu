@@ -385,6 +385,7 @@ extern "C" int zipml_loss_codes_static(int device, void* cuda_stream, const zipm
     if (!b || !x || !loss_out) return ZIPML_ERR_INVALID_ARG;
     const int bad = check_dataset(data);          // the same checks as every other entry point (plane alignment included)
     if (bad != ZIPML_OK) return bad;
+    if (data->layout != ZIPML_LAYOUT_ROWS) return ZIPML_ERR_UNSUPPORTED;
     const int cb = container_bits(data->bits);
     const bool table = data->level_mode == ZIPML_LEVELS_TABLE;
     const int L = 1 << data->bits;

@@ -376,4 +376,43 @@ int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_
     return cuda_status(cudaGetLastError());
 }
 
+// ---------------------------------------------------------------------------------------------
+// Layout conversion: row-major planes <-> 128-byte column blocks ([block][row][128 B]).  One thread moves
+// 16 bytes; a warp covers four 128-byte pieces (four consecutive rows of one block): 512 contiguous bytes
+// on the blocked side, four runs of 128 bytes on the row-major side.  Bytes of a block past the end of
+// the row are written as zero (to blocks) or skipped (to rows).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) convert_layout_kernel(const uint4* __restrict__ in1, const uint4* __restrict__ in2,
+                                                             uint4* __restrict__ out1, uint4* __restrict__ out2, int64_t m,
+                                                             int64_t row_bytes, int64_t nblk, bool to_blocks) {
+    const int64_t pieces = nblk * m;                      // 128-byte pieces of a plane
+    const int64_t row16 = row_bytes / 16;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pieces * 8; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t piece = i >> 3, blk = piece / m, row = piece - blk * m;
+        const int64_t c16 = blk * 8 + (i & 7);            // 16-byte column of the row
+        const bool inside = c16 < row16;
+        const int64_t r_idx = row * row16 + c16;
+        if (to_blocks) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            out1[i] = inside ? __ldg(in1 + r_idx) : z;
+            out2[i] = inside ? __ldg(in2 + r_idx) : z;
+        } else if (inside) {
+            out1[r_idx] = __ldg(in1 + i);
+            out2[r_idx] = __ldg(in2 + i);
+        }
+    }
+}
+
+int launch_convert_layout(zipml_ctx* ctx, const zipml_dataset* d, int to_layout, uint8_t* out1, uint8_t* out2) {
+    const int64_t nblk = (d->row_bytes + 127) / 128;
+    const int64_t units = nblk * d->m * 8;
+    int64_t blocks = (units + 255) / 256;
+    if (blocks > (int64_t)ctx->sm_count * 32) blocks = (int64_t)ctx->sm_count * 32;
+    convert_layout_kernel<<<(unsigned)blocks, 256, 0, ctx->stream>>>(
+        reinterpret_cast<const uint4*>(d->plane1), reinterpret_cast<const uint4*>(d->plane2), reinterpret_cast<uint4*>(out1),
+        reinterpret_cast<uint4*>(out2), d->m, d->row_bytes, nblk, to_layout == ZIPML_LAYOUT_COLUMN_BLOCKS);
+    ctx->launches += 1;
+    return cuda_status(cudaGetLastError());
+}
+
 }  // namespace zipml

@@ -1,5 +1,5 @@
 // Column engine of zipml_sgd_epoch: large minibatch tiles on uniform grids, fp32 model and gradient,
-// every code byte read from HBM exactly once per step.
+// every code byte read from HBM exactly once per step, no grid-wide barrier.
 //
 // A step of the double-sampled minibatch SGD (paper Eq. (double) in its symmetrised form, footnote of
 // "Double Sampling"; update in full precision, "End-to-end Quantization") needs the step's code tile
@@ -8,35 +8,54 @@
 // the 128-byte column block j of the packed rows (1024 / CB features) for all rows and the whole
 // launch, so its slice of the model, of w = step * x and of the gradient never leave the CTA, and the
 // only thing CTAs exchange is the rows' dots.  Rows travel in chunks of R rows (both planes, R x 128
-// bytes each, one 2-D tensor copy per plane with the 128-byte swizzle) through a ring of shared-memory
-// slots, and a chunk stays in its slot until both of its uses are over:
+// bytes each, one 2-D tensor copy per plane with the 128-byte swizzle).  A chunk comes into shared memory
+// twice: from HBM for its dots, and again -- out of L2, where the first copy left it a few microseconds
+// earlier -- when its residuals are known.  Between the two visits it occupies no shared memory, so the
+// exchange of its dots (several L2 round trips under load) may take as long as it likes without holding
+// the stream up:
 //
-//   producer  (1 warp)   tensor copies of the coming chunks, across step boundaries (codes do not depend
-//                        on the model); publishes "this CTA's dots of chunk q are added" to a counter
-//   A warps   (8)        partial dots of the chunk from shared memory on the int8 tensor cores
-//                        (mma.sync m16n8k32, u8 codes x s8 digits of w), converted to a fixed-point unit
-//                        common to all CTAs and added to dots[row] with 64-bit integer atomics
-//   R warps   (4)        wait until all CTAs' parts of the chunk have arrived (counter), read the chunk's
-//                        dots and labels, turn the residuals into eight balanced base-128 int8 digits
-//   B warps   (8)        gradient of the CTA's own features from the same slot (transposing ldmatrix,
-//                        residual digits as the other operand), accumulated in registers over the step;
-//                        at the step's end: update of the own slice of x, digits of the next w
+//   service   (1 warp)   lane 0: tensor copies into two rings of slots, "A" (first visit, ahead of the A
+//                        warps, across step boundaries: codes do not depend on the model) and "B" (second
+//                        visit, in the same order, as far ahead of the B warps as that ring allows)
+//   A warps   (8)        partial dots of the chunk on the int8 tensor cores (mma.sync m16n8k32, u8 codes x
+//                        s8 digits of w), converted to a fixed-point unit common to all CTAs and added to
+//                        the row's word with one 64-bit integer atomic, whose low byte counts the CTAs
+//   R warps   (4)        poll a chunk's words until their counts are complete, read the labels, turn the
+//                        residuals into eight balanced base-128 int8 digits; each warp takes every fourth
+//                        chunk, so four exchanges are in flight at a time
+//   B warps   (8)        gradient of the CTA's own features (transposing ldmatrix, residual digits as the
+//                        other operand), accumulated in registers over the step; at the step's end: update
+//                        of the own slice of x, digits of the next w
 //
-// There is no grid-wide barrier: while the exchange of chunk q settles (about one L2 round trip plus
-// the slowest CTA's lag) the CTA streams and processes the chunks behind it.  At a step's end the
-// pipeline drains (the next dots need the whole new w of the CTA), while the producer keeps filling
-// free slots with the next step's first chunks.
+// A word is its own flag (sum in the upper 56 bits, count below), so there is no counter and no barrier
+// between CTAs.  At a step's end the pipeline drains (the next dots need the whole new w of the CTA) while
+// the A ring fills with the next step's first chunks.  The CTAs may be split into groups with a word each per
+// row (same-address atomics are served one after the other), but one word for all measured fastest.
 //
-// Fixed point.  w of the own features: four digits relative to the CTA's own max |w| (27 bits).  Dots:
-// each CTA rounds its part (own part of lo^T x + delta * digit sums) to a multiple of U = 2^e / 2^61
-// where 2^e >= D, and D bounds every |dot| of the step: D(0) = sum_j |x_j| amax_j from the caller's
-// model, D(t+1) = grow * D(t) + lr * rmax(t) * sum_j amax_j^2 (amax_j the largest |value| of feature
-// j, rmax(t) the step's largest |residual|, which every CTA reads off the same dots): every CTA
-// derives the same U without asking anyone, 64-bit sums of multiples of U are exact and order-free,
-// and the bound may be loose by 2^30 before 2^-31 relative precision is touched.  Residuals: eight
-// digits (55 bits) relative to D(t) + max |b| of the step, for the same reason; all eight columns of
-// the tensor-core tile carry a digit.  Results do not depend on timing: every sum is an integer sum or
-// has a fixed order.
+// Fixed point.  Dots: every CTA adds its part as a multiple of U = 2^e / 2^52 where 2^e > D, and D bounds
+// every |dot| of the step: D(0) = sum_j |x_j| amax_j from the caller's model, D(t+1) = grow * D(t) +
+// lr * rmax(t) * sum_j amax_j^2 (amax_j the largest |value| of feature j, rmax(t) the step's largest
+// |residual|, which every CTA reads off the same words): every CTA derives the same U without asking
+// anyone, sums of multiples of U are exact and order-free, and the bound may be loose by 2^21 before 2^-31
+// relative precision is touched.  w of the own features: four digits (27 bits) whose unit is U times a power
+// of two, at most twice what the CTA's own max |w| needs, so that a digit sum becomes a multiple of U by a
+// shift; the own part of lo^T x is rounded to a multiple of U once per step: the path from the tensor-core
+// sums to the atomic is integer arithmetic only.  Residuals: eight digits (55 bits) relative to D(t) +
+// max |b| of the step; all eight columns of the tensor-core tile carry a digit.  Digits are balanced
+// (-64..63) and found without a carry chain: with 64 added to every digit the number is plain base 128.
+// Results do not depend on timing: every sum is an integer sum or has a fixed order.
+//
+// The machine code is kept small on purpose (four roles share the instruction cache): 32-bit counters kept up
+// step by step instead of 64-bit divisions, waits as functions with one copy, loops unrolled only where
+// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 26.2 us per step (stream engine:
+// 29.8), DRAM reads 1.00 x the packed bytes; the R warps (an L2 round trip or two and the digits per chunk)
+// and the instruction issue rate of the SM, not HBM, bound it.
+//
+// Memory order.  A buffer of dot words serves every third step and is cleared in between by the R warp that
+// has just seen the first chunk of step t complete (then every CTA has left step t-1, the buffer's last
+// use, behind: hence its fence before the stores); the A warps fence once per step before their first
+// addition, so that whoever sees a CTA's additions of step t+1 -- which every adder of step t+2 has -- also
+// sees its cleared share.
 #include <cuda.h>
 #include <string.h>
 
@@ -45,16 +64,20 @@
 
 namespace zipml {
 
-constexpr int kColAWarps = 8, kColBWarps = 8, kColRWarps = 4;
+constexpr int kColAWarps = 8, kColBWarps = 8, kColRWarps = 4, kColRShift = 2;     // (kColRWarps = 2^kColRShift)
 constexpr int kColWarpA0 = 1, kColWarpB0 = kColWarpA0 + kColAWarps, kColWarpR0 = kColWarpB0 + kColBWarps;
 constexpr int kColThreads = 32 * (kColWarpR0 + kColRWarps);
 constexpr int kColRThreads = 32 * kColRWarps;
 constexpr int kColBThreads = 32 * kColBWarps;
 constexpr int kColBlockBytes = 128;         // bytes of a packed row that a CTA owns
 constexpr int kColMaxBatch = 8192;
-constexpr int kColMaxSlots = 8;
+constexpr int kColMaxSlots = 16;            // per ring
+constexpr int kColMaxChunkRows = 128;       // a lane of an R warp takes four rows of a chunk
+constexpr int kColMaxGroups = 4;            // words per row and plane
 constexpr int kColRDigits = 8;              // digits of a residual
 constexpr long long kColQmaxR = 35000000000000000LL;     // below 63 * (128^8 - 1) / 127
+constexpr long long kColBiasR = 64ll * 567382630219905ll;    // 64 * (128^8 - 1) / 127: digit s of W + bias is balanced digit s of W, plus 64
+constexpr int kColBiasW = 64 * 2113665;                      // 64 * (128^4 - 1) / 127
 constexpr long long kColWaitCycles = 6000000000LL;       // a wait gives up after about three seconds
 constexpr int kColNamedR = 1, kColNamedB = 2;            // named barriers of the R and B warps
 
@@ -68,14 +91,15 @@ struct ColumnArgs {
     float* grad_out;
     int n, bits;
     int R;                   // rows of a chunk (multiple of 32)
-    int slots;               // ring slots
-    int bpad;                // rows of a dots buffer: chunks of the largest step * R
-    int ring;                // entries of the counter ring (a power of two)
+    int slots_a, slots_b;    // slots of the two rings
+    int bpad;                // rows of a buffer of dot words: chunks of the largest step * R
+    int ngrp, gsize;         // groups of CTAs with a dot word each per row and plane; CTAs per group
+    int blocked;             // the planes are in the column-block layout: a CTA's pieces of consecutive rows are contiguous
     float lr;
     int reg;
     float reg_cst;
-    long long* dots;         // [3][2][bpad] fixed-point dots (three steps in rotation), zeroed before the launch
-    unsigned* count;         // [ring][32] one counter per chunk in flight (128 bytes apart), zeroed before the launch
+    long long* dots;         // [3][ngrp][2][bpad] three steps in rotation, zeroed before the launch; a word holds the
+                             // fixed-point sum in its upper 56 bits and the number of CTAs that added in its low byte
     DeviceStatus* status;
     unsigned long long* trace;
     int trace_steps;
@@ -83,17 +107,17 @@ struct ColumnArgs {
 
 struct ColStepParams {       // by step parity
     double U, invU;          // fixed-point unit of the dots                     (R warps -> A, R warps)
-    double delta_w, base;    // unit of the w digits, own part of lo^T x        (B warps -> A warps)
+    long long bint;          // own part of lo^T x in units of U                 (B warps -> A warps)
+    int kshift;              // the unit of the own w digits is U * 2^kshift     (B warps -> A warps)
     double inv_r, delta_r;   // fixed point of the residuals                     (R warps -> B warps)
     double rsum;             // sum of all fixed-point residuals of the step     (R warps -> B warps)
 };
 
 struct ColShared {
-    unsigned long long full[kColMaxSlots];     // the slot's tensor copies have landed
-    unsigned long long empty[kColMaxSlots];    // the B warps are done with the slot
-    unsigned long long adone[kColMaxSlots];    // the A warps have added the slot's dots
-    unsigned long long rfull[2], rempty[2];    // residual digits of a chunk: written / consumed
-    unsigned long long wready;                 // digits of the next w are in place
+    unsigned long long full_a[kColMaxSlots], empty_a[kColMaxSlots];     // A ring: copies landed / the A warps are done
+    unsigned long long full_b[kColMaxSlots], empty_b[kColMaxSlots];     // B ring: copies landed / the B warps are done
+    unsigned long long rfull[kColRWarps], rempty[kColRWarps];   // residual digits of a chunk (one buffer per R warp): written / consumed
+    int w_version;                             // steps (+1) whose digits of w are in place
     ColStepParams sp[2];
     double red_d[2][32];
     float red_f[2][32];
@@ -113,14 +137,27 @@ __device__ __forceinline__ bool mbar_test_wait(unsigned long long* bar, uint32_t
     return done != 0;
 }
 
-// Bounded wait on a local mbarrier phase.  False once this CTA has given up anywhere.
-__device__ __forceinline__ bool col_wait(unsigned long long* bar, uint32_t parity, ColShared* sh, DeviceStatus* status, int where) {
+// try_wait that lets the hardware park the thread for up to about a microsecond: a warp that waits should not
+// take issue slots from the warps that work.
+__device__ __forceinline__ bool mbar_try_wait_parked(unsigned long long* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_u32(bar)), "r"(parity), "r"(1000u) : "memory");
+    return done != 0;
+}
+
+// Bounded wait on a local mbarrier phase.  False once this CTA has given up anywhere.  (Not inlined: one copy.)
+__device__ __noinline__ bool col_wait(unsigned long long* bar, uint32_t parity, ColShared* sh, DeviceStatus* status, int where) {
     if (mbar_test_wait(bar, parity)) return true;
     if (col_aborted(sh)) return false;
     const long long t0 = clock64();
 #pragma unroll 1
     for (int spin = 0;; ++spin) {
-        if (mbar_try_wait(reinterpret_cast<uint64_t*>(bar), parity)) return true;
+        if (mbar_try_wait_parked(bar, parity)) return true;
+        if (spin >= 4) __nanosleep(spin < 16 ? 100 : 400);       // a warp that waits long should stay out of the others' way
         if ((spin & 15) == 15) {
             if (col_aborted(sh)) return false;
             if (clock64() - t0 > kColWaitCycles) break;
@@ -131,15 +168,70 @@ __device__ __forceinline__ bool col_wait(unsigned long long* bar, uint32_t parit
     return false;
 }
 
+// Addition to a word in global memory that returns nothing: fire and forget.  (atomicAdd on a generic pointer
+// compiled to an atomic that brings the old value back, and the warp waited an L2 round trip for a register
+// it never read: 5.6 k cycles per 32-row task instead of a few hundred.)
+__device__ __forceinline__ void red_add_u64(long long* p, unsigned long long v) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "l"(v) : "memory");
+}
+
+// Polling load of two neighbouring words straight from L2 (16-byte aligned).
+__device__ __forceinline__ void ld_l2_v2(const long long* p, long long& v0, long long& v1) {
+    asm volatile("ld.global.cg.v2.s64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(p) : "memory");
+}
+
+__device__ __forceinline__ void st_release_cta(int* p, int v) {
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const int* p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+
+// Bounded wait until a version count in shared memory has reached `want`.
+__device__ __noinline__ bool col_wait_version(const int* version, int want, ColShared* sh, DeviceStatus* status, int where) {
+    const long long t0 = clock64();
+#pragma unroll 1
+    for (int spin = 0; ld_acquire_cta(version) < want; ++spin) {
+        __nanosleep(100);
+        if ((spin & 15) == 15) {
+            if (col_aborted(sh)) return false;
+            if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(status, ZIPML_ERR_TIMEOUT, where); return false; }
+        }
+    }
+    return true;
+}
+
+// Powers of two by their exponent fields (no library call: the code must stay small).
+__device__ __forceinline__ int col_exponent(double v) { return (int)((__double_as_longlong(v) >> 52) & 0x7FF) - 1023; }     // v < 2^(e + 1)
+__device__ __forceinline__ double col_pow2(int e) { return __longlong_as_double((long long)(min(1000, max(-1000, e)) + 1023) << 52); }
+
+// The fixed-point unit of the dots for a bound of their size: 2^e / 2^52 with bound < 2^e.
+__device__ __forceinline__ void col_unit_of(double bound, double& U, double& invU) {
+    const int ex = max(-900, min(900, col_exponent(bound) + 1));
+    U = col_pow2(ex - 52);
+    invU = col_pow2(52 - ex);
+}
+
 __device__ __forceinline__ void named_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
 
 __device__ __forceinline__ void tensor_load_2d(void* dst_smem, const CUtensorMap* tm, int x, int y, unsigned long long* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(smem_u32(dst_smem)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// The same with an L2 eviction policy for the lines it reads.
+__device__ __forceinline__ void tensor_load_2d_hint(void* dst_smem, const CUtensorMap* tm, int x, int y, unsigned long long* bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(smem_u32(dst_smem)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
 
 __device__ __forceinline__ void col_mark(const ColumnArgs& a, int64_t t_rel, int k) {
     if (a.trace && blockIdx.x == 0 && t_rel < a.trace_steps) a.trace[t_rel * 8 + k] = (unsigned long long)clock64();
+}
+// Adds `cycles` to slot k of the step's trace record (one writer per slot).
+__device__ __forceinline__ void col_tally(const ColumnArgs& a, int64_t t_rel, int k, long long cycles) {
+    if (a.trace && blockIdx.x == 0 && t_rel < a.trace_steps) a.trace[t_rel * 8 + k] += (unsigned long long)cycles;
 }
 
 // Rows of step position `it`.
@@ -156,6 +248,17 @@ __device__ __forceinline__ ColStep col_step(const ColumnArgs& a, int64_t it) {
     return s;
 }
 
+// A position in a ring of slots: slot index and the parity of the number of times the ring has wrapped.
+struct ColRing {
+    int slot;
+    uint32_t phase;
+    __device__ __forceinline__ void next(int slots) { if (++slot == slots) { slot = 0; phase ^= 1u; } }
+};
+
+// The kernel's machine code must stay small: four roles run side by side, and once their loops do not fit the
+// instruction cache together every warp waits for its next instructions (a first version of 96 KB spent more
+// time there than anywhere else).  Hence: 32-bit counters kept up step by step instead of 64-bit divisions,
+// waits and helpers as functions with one copy, loops unrolled only where registers demand it.
 template <int CB>
 __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const ColumnArgs a, const __grid_constant__ CUtensorMap tm1,
                                                                     const __grid_constant__ CUtensorMap tm2) {
@@ -166,38 +269,44 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     constexpr int NRD = kColRDigits;
     static_assert(NS == 4, "four digits of w");
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    // [slots][2 planes][R rows][128 B] (1024-byte aligned), then the digit operands, then the bookkeeping
+    // [A slots + B slots][2 planes][R rows][128 B] (1024-byte aligned), then the digit operands, then the bookkeeping
     unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int R = a.R;
     const uint32_t plane_bytes = (uint32_t)R * kColBlockBytes, slot_bytes = 2u * plane_bytes;
+    unsigned char* tiles_b = tiles + (size_t)a.slots_a * slot_bytes;
     const int rstride = R + 32;                        // bytes between the residual digit vectors
-    signed char* rdig = reinterpret_cast<signed char*>(tiles + (size_t)a.slots * slot_bytes);     // [2 buffers][2 operands][8 digits][rstride]
-    signed char* wdig = rdig + (size_t)2 * 2 * NRD * rstride;                                      // [NG][4 k-blocks][4 digits][32 B]
+    signed char* rdig = reinterpret_cast<signed char*>(tiles_b + (size_t)a.slots_b * slot_bytes);  // [R warps][2 operands][8 digits][rstride]
+    signed char* wdig = rdig + (size_t)kColRWarps * 2 * NRD * rstride;                             // [NG][4 k-blocks][4 digits][32 B]
     ColShared* sh = reinterpret_cast<ColShared*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * NS * 32) + 15) & ~(uintptr_t)15);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gl = lane >> 2, tl = lane & 3;
     const int cta = blockIdx.x, G = gridDim.x;
     const int n = a.n;
-    const int64_t steps = a.num_steps;
+    const int steps = (int)a.num_steps;
     const int64_t byte0 = (int64_t)cta * kColBlockBytes;          // first byte of the own column block
+    // tensor-copy coordinates of row 0 of the own block (rows past the step's last one come along and meet zero digits)
+    const int x_own = a.blocked ? 0 : (int)byte0;
+    const int64_t y_own = a.blocked ? (int64_t)cta * a.m : 0;
 
     if (tid == 0) {
-        for (int s = 0; s < a.slots; ++s) {
-            mbar_init(reinterpret_cast<uint64_t*>(sh->full + s), 1);
-            mbar_init(reinterpret_cast<uint64_t*>(sh->empty + s), kColBWarps);
-            mbar_init(reinterpret_cast<uint64_t*>(sh->adone + s), kColAWarps);
+        for (int s = 0; s < kColMaxSlots; ++s) {
+            mbar_init(reinterpret_cast<uint64_t*>(sh->full_a + s), 1);
+            mbar_init(reinterpret_cast<uint64_t*>(sh->empty_a + s), a.R / 32);     // one arrival per 32-row task
+            mbar_init(reinterpret_cast<uint64_t*>(sh->full_b + s), 1);
+            mbar_init(reinterpret_cast<uint64_t*>(sh->empty_b + s), kColBWarps);
         }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(reinterpret_cast<uint64_t*>(sh->rfull + s), kColRWarps);
+        for (int s = 0; s < kColRWarps; ++s) {
+            mbar_init(reinterpret_cast<uint64_t*>(sh->rfull + s), 1);
             mbar_init(reinterpret_cast<uint64_t*>(sh->rempty + s), kColBWarps);
         }
-        mbar_init(reinterpret_cast<uint64_t*>(&sh->wready), kColBWarps);
+        sh->w_version = 0;
         sh->abort_flag = 0;
         mbar_fence_init();
     }
     // ---- every CTA scans the model once, with the same arithmetic: the bound of the dots and its growth rate
     const float smax = (float)((1 << a.bits) - 1);
     double dsum = 0.0, csum = 0.0;
+#pragma unroll 1
     for (int j = tid; j < n; j += kColThreads) {
         const float l = a.lo[j], s = a.step[j];
         const double am = (double)fmaxf(fabsf(l), fabsf(l + s * smax));
@@ -209,146 +318,185 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     if (lane == 0) { sh->red_d[0][warp] = dsum; sh->red_d[1][warp] = csum; }
     __syncthreads();
     double dbound = 0.0, c2 = 0.0;
+#pragma unroll 1
     for (int w = 0; w < kColThreads / 32; ++w) { dbound += sh->red_d[0][w]; c2 += sh->red_d[1][w]; }
     dbound *= 1.0001;
-    auto unit_of = [](double bound, double& U, double& invU) {
-        int ex = 0;
-        if (bound > 0.0) (void)frexp(bound, &ex);        // bound <= 2^ex
-        U = ldexp(1.0, ex - 61);
-        invU = ldexp(1.0, 61 - ex);
-    };
-    if (tid == 0) unit_of(dbound, sh->sp[0].U, sh->sp[0].invU);
+    if (tid == 0) col_unit_of(dbound, sh->sp[0].U, sh->sp[0].invU);
     __syncthreads();                                      // barriers initialised, sums read, U(0) in place
 
-    // =================================================================================== producer
+    // =================================================================================== service warp
     if (warp == 0) {
         if (lane == 0) {
-            int64_t tL = 0, tP = 0;                       // steps of the next chunk to load / to publish
-            int cL = 0, cP = 0;
-            int64_t qL = 0, qP = 0;                       // their positions in the launch's chunk sequence
-            ColStep sL = col_step(a, a.first_step), sP = sL;
+            // first visits: the next chunk as soon as a slot of the A ring is free; second visits: the next chunk that
+            // has had its first copy issued (it is in L2 or on its way there), as soon as a slot of the B ring is free
+            int qA = 0, tA = 0, cA = 0, qB = 0, tB = 0, cB = 0;
+            ColRing ra{0, 0u}, rb{0, 0u};
+            ColStep sA = col_step(a, a.first_step), sB = sA;
+            uint64_t evict_first;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
             long long idle0 = clock64();
+            int idle = 0;
             bool ok = true;
-            while (tP < steps && ok) {
+#pragma unroll 1
+            while (ok && tB < steps) {
                 bool progress = false;
-                if (tL < steps) {
-                    const int slot = (int)(qL % a.slots);
-                    const int64_t use = qL / a.slots;
-                    if (use == 0 || mbar_test_wait(sh->empty + slot, (uint32_t)((use - 1) & 1))) {
-                        unsigned char* dst = tiles + (size_t)slot * slot_bytes;
-                        mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(sh->full + slot), slot_bytes);
-                        const int y = (int)(sL.row0 + (int64_t)cL * R);
-                        tensor_load_2d(dst, &tm1, (int)byte0, y, sh->full + slot);
-                        tensor_load_2d(dst + plane_bytes, &tm2, (int)byte0, y, sh->full + slot);
-                        ++qL;
-                        if (++cL == sL.nch) { cL = 0; if (++tL < steps) sL = col_step(a, a.first_step + tL); }
-                        progress = true;
-                    }
+                if (tA < steps && (qA < a.slots_a || mbar_test_wait(sh->empty_a + ra.slot, ra.phase ^ 1u))) {
+                    unsigned char* dst = tiles + (size_t)ra.slot * slot_bytes;
+                    mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(sh->full_a + ra.slot), slot_bytes);
+                    const int y = (int)(y_own + sA.row0 + (int64_t)cA * R);
+                    tensor_load_2d(dst, &tm1, x_own, y, sh->full_a + ra.slot);
+                    tensor_load_2d(dst + plane_bytes, &tm2, x_own, y, sh->full_a + ra.slot);
+                    ++qA;
+                    ra.next(a.slots_a);
+                    if (++cA == sA.nch) { cA = 0; if (++tA < steps) sA = col_step(a, a.first_step + tA); }
+                    progress = true;
                 }
-                if (qP < qL) {
-                    const int slot = (int)(qP % a.slots);
-                    if (mbar_test_wait(sh->adone + slot, (uint32_t)((qP / a.slots) & 1))) {
-                        // every A warp's additions come before its arrival, this thread's fence after its wait:
-                        // whoever sees the count sees the sums
-                        __threadfence();
-                        atomicAdd(a.count + (size_t)(qP & (a.ring - 1)) * 32, 1u);
-                        ++qP;
-                        if (++cP == sP.nch) {
-                            if (blockIdx.x == 0 && a.trace && tP < a.trace_steps) a.trace[tP * 8 + 6] = (unsigned long long)clock64();
-                            cP = 0;
-                            if (++tP < steps) sP = col_step(a, a.first_step + tP);
-                        }
-                        progress = true;
-                    }
+                if (qB < qA && (qB < a.slots_b || mbar_test_wait(sh->empty_b + rb.slot, rb.phase ^ 1u))) {
+                    unsigned char* dst = tiles_b + (size_t)rb.slot * slot_bytes;
+                    mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(sh->full_b + rb.slot), slot_bytes);
+                    const int y = (int)(y_own + sB.row0 + (int64_t)cB * R);
+                    // (nobody reads these lines again this epoch: they may leave L2 ahead of the rest)
+                    tensor_load_2d_hint(dst, &tm1, x_own, y, sh->full_b + rb.slot, evict_first);
+                    tensor_load_2d_hint(dst + plane_bytes, &tm2, x_own, y, sh->full_b + rb.slot, evict_first);
+                    ++qB;
+                    rb.next(a.slots_b);
+                    if (++cB == sB.nch) { cB = 0; if (++tB < steps) sB = col_step(a, a.first_step + tB); }
+                    progress = true;
                 }
-                if (progress) idle0 = clock64();
+                if (progress) { idle0 = clock64(); idle = 0; }
                 else {
-                    if (col_aborted(sh)) ok = false;
-                    else if (clock64() - idle0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 70); ok = false; }
+                    __nanosleep(idle < 8 ? 100 : 300);
+                    if ((++idle & 15) == 15) {
+                        if (col_aborted(sh)) ok = false;
+                        else if (clock64() - idle0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 70); ok = false; }
+                    }
                 }
             }
             if (!ok) {
                 // leaving early: the copies in flight must land before the CTA's shared memory goes away
-                for (int64_t q = (qL > a.slots ? qL - a.slots : 0); q < qL; ++q) {
-                    const long long t0 = clock64();
-                    while (!mbar_test_wait(sh->full + (q % a.slots), (uint32_t)((q / a.slots) & 1)) && clock64() - t0 < kColWaitCycles) {}
+                const long long t0 = clock64();
+#pragma unroll 1
+                for (int s = 0; s < kColMaxSlots; ++s) {
+                    if (s < a.slots_a && s < qA) {
+                        const uint32_t par = (uint32_t)((((qA - 1 - ((qA - 1 - s + a.slots_a) % a.slots_a)) / a.slots_a)) & 1);
+                        while (!mbar_test_wait(sh->full_a + s, par) && clock64() - t0 < kColWaitCycles) {}
+                    }
+                    if (s < a.slots_b && s < qB) {
+                        const uint32_t par = (uint32_t)((((qB - 1 - ((qB - 1 - s + a.slots_b) % a.slots_b)) / a.slots_b)) & 1);
+                        while (!mbar_test_wait(sh->full_b + s, par) && clock64() - t0 < kColWaitCycles) {}
+                    }
                 }
             }
         }
     }
     // =================================================================================== A warps: dots
     else if (warp < kColWarpB0) {
+        // A task is 32 rows of a chunk (two 16-row tiles, interleaved); the tasks of the launch's chunk sequence are
+        // dealt to the eight warps in turn, so that several chunks are worked on at a time.
         const int aw = warp - kColWarpA0;
-        int64_t q = 0;
         constexpr uint32_t kLow = CB == 8 ? 0xFFFFFFFFu : CB == 4 ? 0x0F0F0F0Fu : 0x03030303u;
         // ldmatrix row addresses: lane l gives row (l & 7) + 8 * ((l >> 3) & 1) of the 16-row block and the
         // 16-byte piece (l >> 4) of a 32-byte k-block; the 128-byte swizzle moves piece c of row r to c ^ (r & 7)
         const uint32_t a_row = (uint32_t)((lane & 7) + 8 * ((lane >> 3) & 1)), a_piece = (uint32_t)(lane >> 4), a_x = (uint32_t)(lane & 7);
         const uint32_t wdig_lane = smem_u32(wdig) + (uint32_t)(gl * 32 + tl * 8);          // lanes with gl < 4 read digit gl
-        bool ok = true;
-        for (int64_t t_rel = 0; t_rel < steps && ok; ++t_rel) {
-            const ColStep st = col_step(a, a.first_step + t_rel);
-            ok = __all_sync(0xffffffffu, col_wait(&sh->wready, (uint32_t)(t_rel & 1), sh, a.status, 71));     // (the warp acts as one)
-            if (!ok) break;
-            if (aw == 0 && lane == 0) col_mark(a, t_rel, 0);
-            const ColStepParams& sp = sh->sp[t_rel & 1];
-            const double invU = sp.invU, delta_w = sp.delta_w, base = sp.base;
-            long long* dots = a.dots + (size_t)(t_rel % 3) * 2 * a.bpad;
-            for (int c = 0; c < st.nch; ++c, ++q) {
-                const int slot = (int)(q % a.slots);
-                ok = __all_sync(0xffffffffu, col_wait(sh->full + slot, (uint32_t)((q / a.slots) & 1), sh, a.status, 72));
+        const int grp = cta / a.gsize;
+        const int tpc = R / 32;                          // tasks per chunk
+        int t_rel = 0, c = 0, j = aw;                    // the current task: step, chunk of the step, task of the chunk
+        ColRing ring{0, 0u};                             // the chunk's slot
+        ColStep st = col_step(a, a.first_step);
+        bool fresh = true, ok = true;                    // fresh: the step's parameters are still to be fetched
+        int kshift = 0;
+        long long bint = 0;
+        long long* dots = a.dots;
+#pragma unroll 1
+        while (ok) {
+#pragma unroll 1
+            while (j >= tpc && t_rel < steps) {          // on to the task's chunk
+                j -= tpc;
+                ring.next(a.slots_a);
+                if (++c == st.nch) {
+                    c = 0;
+                    fresh = true;
+                    if (++t_rel < steps) st = col_step(a, a.first_step + t_rel);
+                }
+            }
+            if (t_rel >= steps) break;
+            if (fresh) {
+                // the digits of this step's w (a version count, not a phase: a warp without a task in some step
+                // never looks at that step's digits)
+                ok = __all_sync(0xffffffffu, col_wait_version(&sh->w_version, t_rel + 1, sh, a.status, 71));     // (the warp acts as one)
                 if (!ok) break;
-                const uint32_t tile = smem_u32(tiles) + (uint32_t)slot * slot_bytes;
-                for (int rb = aw; rb < R / 16; rb += kColAWarps) {
-                    const int k0 = c * R + rb * 16;                      // first row of the block within the step
-                    if (k0 >= st.bt) break;
-                    int c1[NG][4], c2[NG][4];
+                __threadfence();        // (see "Memory order" above: the cleared words before this step's additions)
+                const ColStepParams& sp = sh->sp[t_rel & 1];
+                kshift = sp.kshift; bint = sp.bint;
+                dots = a.dots + ((size_t)(t_rel % 3) * a.ngrp + grp) * 2 * a.bpad;
+                fresh = false;
+                if (lane == 0 && c == 0 && j == 0) col_mark(a, t_rel, 0);
+            }
+            const long long w0c = (a.trace && aw == 0) ? clock64() : 0;
+            ok = __all_sync(0xffffffffu, col_wait(sh->full_a + ring.slot, ring.phase, sh, a.status, 72));
+            if (!ok) break;
+            if (a.trace && aw == 0 && lane == 0) col_tally(a, t_rel, 1, clock64() - w0c);
+            const uint32_t tile = smem_u32(tiles) + (uint32_t)ring.slot * slot_bytes;
+            const int k0 = c * R + j * 32;                                // first row of the task within the step
+            if (k0 < st.bt) {
+                int c1[2][NG][4], c2[2][NG][4];                          // [tile][group][fragment]: plane 1, plane 2
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
 #pragma unroll
                     for (int g = 0; g < NG; ++g)
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) { c1[g][e] = 0; c2[g][e] = 0; }
-                    const uint32_t row_addr = tile + (uint32_t)(rb * 16 + a_row) * kColBlockBytes;
+                        for (int e = 0; e < 4; ++e) { c1[h][g][e] = 0; c2[h][g][e] = 0; }
+                const uint32_t row_addr = tile + (uint32_t)(j * 32 + a_row) * kColBlockBytes;
+#pragma unroll 1
+                for (int kb = 0; kb < 4; ++kb) {
+                    uint32_t f1[2][4], f2[2][4];
+                    const uint32_t off = row_addr + (((uint32_t)(2 * kb) + a_piece) ^ a_x) * 16u;
 #pragma unroll
-                    for (int kb = 0; kb < 4; ++kb) {
-                        uint32_t f1[4], f2[4];
-                        const uint32_t off = row_addr + (((uint32_t)(2 * kb) + a_piece) ^ a_x) * 16u;
-                        ldsm_x4(f1, off);
-                        ldsm_x4(f2, off + plane_bytes);
-#pragma unroll
-                        for (int g = 0; g < NG; ++g) {
-                            uint32_t b0 = 0u, b1 = 0u;
-                            if (gl < NS) asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(wdig_lane + (uint32_t)((g * 4 + kb) * NS * 32)));
-                            // group g's codes stay where they are in the byte: its sums come out 2^(g CB) times too large
-                            const uint32_t mk = kLow << (g * CB);
-                            mma_u8s8(c1[g], f1[0] & mk, f1[1] & mk, f1[2] & mk, f1[3] & mk, b0, b1);
-                            mma_u8s8(c2[g], f2[0] & mk, f2[1] & mk, f2[2] & mk, f2[3] & mk, b0, b1);
-                        }
+                    for (int h = 0; h < 2; ++h) {
+                        ldsm_x4(f1[h], off + (uint32_t)h * 16u * kColBlockBytes);
+                        ldsm_x4(f2[h], off + (uint32_t)h * 16u * kColBlockBytes + plane_bytes);
                     }
-                    // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3])
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        long long q1 = 0, q2 = 0;
+                    for (int g = 0; g < NG; ++g) {
+                        uint32_t b0 = 0u, b1 = 0u;
+                        if (gl < NS) asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(wdig_lane + (uint32_t)((g * 4 + kb) * NS * 32)));
+                        // group g's codes stay where they are in the byte: its sums come out 2^(g CB) times too large
+                        const uint32_t mk = kLow << (g * CB);
 #pragma unroll
-                        for (int g = 0; g < NG; ++g) {                   // exact: the sums are multiples of 2^(g CB)
-                            q1 += (long long)(c1[g][2 * e] >> (g * CB)) + 128ll * (long long)(c1[g][2 * e + 1] >> (g * CB));
-                            q2 += (long long)(c2[g][2 * e] >> (g * CB)) + 128ll * (long long)(c2[g][2 * e + 1] >> (g * CB));
-                        }
-                        const long long v1 = q1 + 16384ll * __shfl_down_sync(0xffffffffu, q1, 1);
-                        const long long v2 = q2 + 16384ll * __shfl_down_sync(0xffffffffu, q2, 1);
-                        const int k = k0 + gl + 8 * e;
-                        if (tl == 0 && k < st.bt) {
-                            // this CTA's part of the dot, as a multiple of the unit every CTA uses this step
-                            const long long P1 = __double2ll_rn(((double)v1 * delta_w + base) * invU);
-                            const long long P2 = __double2ll_rn(((double)v2 * delta_w + base) * invU);
-                            atomicAdd(reinterpret_cast<unsigned long long*>(dots + k), (unsigned long long)P1);
-                            atomicAdd(reinterpret_cast<unsigned long long*>(dots + a.bpad + k), (unsigned long long)P2);
+                        for (int h = 0; h < 2; ++h) {
+                            mma_u8s8(c1[h][g], f1[h][0] & mk, f1[h][1] & mk, f1[h][2] & mk, f1[h][3] & mk, b0, b1);
+                            mma_u8s8(c2[h][g], f2[h][0] & mk, f2[h][1] & mk, f2[h][2] & mk, f2[h][3] & mk, b0, b1);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->adone + slot));
+                // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3]) of each tile.  Integers all
+                // the way: the groups' sums (multiples of 2^(g CB), shifted back exactly) in 32 bits, two digits per
+                // lane and then the neighbour's two in 64, the shift into the dots' unit, the own part of lo^T x.
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        int x10 = 0, x11 = 0, x20 = 0, x21 = 0;
+#pragma unroll
+                        for (int g = 0; g < NG; ++g) {
+                            x10 += c1[h][g][2 * e] >> (g * CB); x11 += c1[h][g][2 * e + 1] >> (g * CB);
+                            x20 += c2[h][g][2 * e] >> (g * CB); x21 += c2[h][g][2 * e + 1] >> (g * CB);
+                        }
+                        const long long q1 = (long long)x10 + ((long long)x11 << 7), q2 = (long long)x20 + ((long long)x21 << 7);
+                        const long long v1 = q1 + (__shfl_down_sync(0xffffffffu, q1, 1) << 14);
+                        const long long v2 = q2 + (__shfl_down_sync(0xffffffffu, q2, 1) << 14);
+                        const int k = k0 + 16 * h + gl + 8 * e;
+                        if (tl == 0 && k < st.bt) {
+                            // the word's upper 56 bits take the sum, its low byte counts this CTA in
+                            red_add_u64(dots + k, ((unsigned long long)((v1 << kshift) + bint) << 8) + 1ull);
+                            red_add_u64(dots + a.bpad + k, ((unsigned long long)((v2 << kshift) + bint) << 8) + 1ull);
+                        }
+                    }
             }
-            if (aw == 0 && lane == 0) col_mark(a, t_rel, 1);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty_a + ring.slot));
+            j += kColAWarps;
         }
     }
     // =================================================================================== B warps: gradient, update
@@ -369,94 +517,118 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             lo_o[e] = have[e] ? a.lo[jo[e]] : 0.0f;
             st_o[e] = have[e] ? a.step[jo[e]] : 0.0f;
         }
-        // digits of w = step * x of the own features for the step at parity `par`, and the own part of lo^T x
-        auto publish_w = [&](int par) {
-            float wm = 0.0f;
-            double bs = 0.0;
-#pragma unroll
-            for (int e = 0; e < NF; ++e) { wm = fmaxf(wm, fabsf(st_o[e] * xo[e])); bs += (double)lo_o[e] * (double)xo[e]; }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
-            bs = warp_sum(bs);
-            if (lane == 0) { sh->red_f[0][p] = wm; sh->red_d[0][p] = bs; }
-            named_barrier(kColNamedB, kColBThreads);
-            float wmax = 0.0f;
-            double bsum = 0.0;
-#pragma unroll
-            for (int w = 0; w < kColBWarps; ++w) { wmax = fmaxf(wmax, sh->red_f[0][w]); bsum += sh->red_d[0][w]; }
-            const float inv = wmax > 0.0f ? (float)QMAXW / wmax : 0.0f;
-            if (btid == 0) { sh->sp[par].delta_w = (double)wmax / (double)QMAXW; sh->sp[par].base = bsum; }
-#pragma unroll
-            for (int e = 0; e < NF; ++e) {
-                const int fi = tl + 4 * e, h = fi / NG, gi = fi - h * NG;
-                if (fi < 2 * NG) {
-                    const int byte = 16 * p + 2 * gl + h, kb = byte >> 5, bb = byte & 31;
-                    int d[NS];
-                    balanced_digits<NS>(have[e] ? max(-QMAXW, min(QMAXW, __float2int_rn(st_o[e] * xo[e] * inv))) : 0, d);
-                    signed char* dst = wdig + (size_t)((gi * 4 + kb) * NS) * 32 + ((bb & 15) >> 2) * 8 + (bb >> 4) * 4 + (bb & 3);
-#pragma unroll
-                    for (int s = 0; s < NS; ++s) dst[s * 32] = (signed char)d[s];
-                }
-            }
-            named_barrier(kColNamedB, kColBThreads);     // (also: nobody re-enters with red_* still being read)
-            __syncwarp();
-            if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(&sh->wready));
-        };
-        publish_w(0);
-
         const uint32_t b_x = (uint32_t)(lane & 7);
         const uint32_t b_off = (uint32_t)lane * kColBlockBytes + (((uint32_t)p ^ b_x) << 4);
         const uint32_t rdig_lane = smem_u32(rdig) + (uint32_t)(gl * rstride + tl * 8);
-        int64_t q = 0;
+        int q = 0;                                       // chunks so far
+        ColRing ring{0, 0u};
         // After a wait has given up the warp stays in step with the others (the named barriers below need every
         // B thread) but waits for nothing and skips the arithmetic.
         bool ok = true;
-        for (int64_t t_rel = 0; t_rel < steps; ++t_rel) {
+#pragma unroll 1
+        for (int t_rel = 0; t_rel < steps; ++t_rel) {
             const ColStep st = col_step(a, a.first_step + t_rel);
             const bool last = t_rel + 1 == steps;
-            int acc[NG][4];
+            // ---- digits of w = step * x of the own features for this step, and the own part of lo^T x
+            {
+                const int par = t_rel & 1;
+                float wm = 0.0f;
+                double bs = 0.0;
 #pragma unroll
-            for (int g = 0; g < NG; ++g)
+                for (int e = 0; e < NF; ++e) { wm = fmaxf(wm, fabsf(st_o[e] * xo[e])); bs += (double)lo_o[e] * (double)xo[e]; }
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[g][e] = 0;
-            for (int c = 0; c < st.nch; ++c, ++q) {
-                const int slot = (int)(q % a.slots), rbuf = (int)(q & 1);
-                ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> 1) & 1), sh, a.status, 73);
-                ok = ok && col_wait(sh->full + slot, (uint32_t)((q / a.slots) & 1), sh, a.status, 74);     // (landed long ago: makes the copy's bytes visible here)
-                ok = __all_sync(0xffffffffu, ok);                      // the warp acts as one
-                const uint32_t tile = smem_u32(tiles) + (uint32_t)slot * slot_bytes + b_off;
-                const int nrb = ok ? (min(R, st.bt - c * R) + 31) >> 5 : 0;
+                for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+                bs = warp_sum(bs);
+                if (lane == 0) { sh->red_f[0][p] = wm; sh->red_d[0][p] = bs; }
+                named_barrier(kColNamedB, kColBThreads);
+                float wmax = 0.0f;
+                double bsum = 0.0;
+#pragma unroll
+                for (int w = 0; w < kColBWarps; ++w) { wmax = fmaxf(wmax, sh->red_f[0][w]); bsum += sh->red_d[0][w]; }
+                // the unit of the digits is the dots' unit times a power of two (at most twice what max |w| needs), so
+                // that a digit sum turns into the dots' unit by a shift
+                const double U = sh->sp[par].U, need = (double)wmax * (1.0 / (double)QMAXW);
+                const int eu = col_exponent(U);                           // U = 2^eu
+                const int ks = need > U ? col_exponent(need) + 1 - eu : 0;   // need < U * 2^ks
+                const float inv = (float)col_pow2(-(eu + ks));
+                if (btid == 0) { sh->sp[par].kshift = ks; sh->sp[par].bint = __double2ll_rn(bsum * sh->sp[par].invU); }
+#pragma unroll
+                for (int e = 0; e < NF; ++e) {
+                    const int fi = tl + 4 * e, h = fi / NG, gi = fi - h * NG;
+                    if (fi < 2 * NG) {
+                        const int byte = 16 * p + 2 * gl + h, kb = byte >> 5, bb = byte & 31;
+                        // balanced digits without a carry chain: with 64 added to every digit the number is plain base 128
+                        const uint32_t u = (uint32_t)((have[e] ? max(-QMAXW, min(QMAXW, __float2int_rn(st_o[e] * xo[e] * inv))) : 0) + kColBiasW);
+                        signed char* dst = wdig + (size_t)((gi * 4 + kb) * NS) * 32 + ((bb & 15) >> 2) * 8 + (bb >> 4) * 4 + (bb & 3);
+#pragma unroll
+                        for (int s = 0; s < NS; ++s) dst[s * 32] = (signed char)((int)((u >> (7 * s)) & 127u) - 64);
+                    }
+                }
+                named_barrier(kColNamedB, kColBThreads);     // every digit is written (also: red_* may be reused)
+                if (btid == 0) st_release_cta(&sh->w_version, t_rel + 1);
+                if (t_rel > 0 && p == 0 && lane == 0) col_mark(a, t_rel - 1, 7);
+            }
+            int acc2[2][NG][4];                                  // two sets, for alternate 32-row blocks: shorter dependency chains
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int g = 0; g < NG; ++g)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc2[h][g][e] = 0;
 #pragma unroll 1
-                for (int rb = 0; rb < nrb; ++rb) {
+            for (int c = 0; c < st.nch; ++c, ++q) {
+                const int rbuf = q & (kColRWarps - 1);
+                const long long w0c = (a.trace && p == 0) ? clock64() : 0;
+                ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1), sh, a.status, 73);
+                const long long w1c = (a.trace && p == 0) ? clock64() : 0;
+                ok = ok && col_wait(sh->full_b + ring.slot, ring.phase, sh, a.status, 74);
+                if (a.trace && p == 0 && lane == 0) { col_tally(a, t_rel, 4, w1c - w0c); col_tally(a, t_rel, 5, clock64() - w1c); }
+                ok = __all_sync(0xffffffffu, ok);                      // the warp acts as one
+                const uint32_t tile = smem_u32(tiles_b) + (uint32_t)ring.slot * slot_bytes + b_off;
+                const int nrb = ok ? (min(R, st.bt - c * R) + 31) >> 5 : 0;
 #pragma unroll
-                    for (int pl = 0; pl < 2; ++pl) {
-                        uint32_t r4[4], b0, b1;
-                        ldsm_x4_trans(r4, tile + (uint32_t)pl * plane_bytes + (uint32_t)rb * 32u * kColBlockBytes);
-                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1)
-                                     : "r"(rdig_lane + (uint32_t)(((rbuf * 2 + pl) * NRD) * rstride + rb * 32)));
-                        // bytes {2g, 2g+1} of rows {2t, 2t+1} of the four 8-row groups -> byte 2g (and 2g+1) of rows
-                        // {2t, 2t+1, 8+2t, 9+2t} (+16): features x rows, in the row order of the residual digits
-                        const uint32_t e0 = __byte_perm(r4[0], r4[1], 0x6420), o0 = __byte_perm(r4[0], r4[1], 0x7531);
-                        const uint32_t e1 = __byte_perm(r4[2], r4[3], 0x6420), o1 = __byte_perm(r4[2], r4[3], 0x7531);
+                for (int rb2 = 0; rb2 < kColMaxChunkRows / 32; rb2 += 2) {
 #pragma unroll
-                        for (int g = 0; g < NG; ++g) {
-                            // All groups of a byte meet the same residual digits, so the sums may nest: accumulator g
-                            // takes the byte with the groups below g cleared (g = 0: the byte as it is), i.e.
-                            // sum_{h >= g} 2^(h CB) code_h; group g is the difference of two neighbours.
-                            const uint32_t mk = 0x01010101u * (uint32_t)((0xFFu << (g * CB)) & 0xFFu);
-                            mma_u8s8(acc[g], e0 & mk, o0 & mk, e1 & mk, o1 & mk, b0, b1);
+                    for (int h = 0; h < 2; ++h) {
+                        const int rb = rb2 + h;
+                        if (rb < nrb) {
+#pragma unroll
+                            for (int pl = 0; pl < 2; ++pl) {
+                                uint32_t r4[4], b0, b1;
+                                ldsm_x4_trans(r4, tile + (uint32_t)pl * plane_bytes + (uint32_t)rb * 32u * kColBlockBytes);
+                                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1)
+                                             : "r"(rdig_lane + (uint32_t)(((rbuf * 2 + pl) * NRD) * rstride + rb * 32)));
+                                // bytes {2g, 2g+1} of rows {2t, 2t+1} of the four 8-row groups -> byte 2g (and 2g+1) of rows
+                                // {2t, 2t+1, 8+2t, 9+2t} (+16): features x rows, in the row order of the residual digits
+                                const uint32_t e0 = __byte_perm(r4[0], r4[1], 0x6420), o0 = __byte_perm(r4[0], r4[1], 0x7531);
+                                const uint32_t e1 = __byte_perm(r4[2], r4[3], 0x6420), o1 = __byte_perm(r4[2], r4[3], 0x7531);
+#pragma unroll
+                                for (int g = 0; g < NG; ++g) {
+                                    // All groups of a byte meet the same residual digits, so the sums may nest: accumulator g
+                                    // takes the byte with the groups below g cleared (g = 0: the byte as it is), i.e.
+                                    // sum_{h >= g} 2^(h CB) code_h; group g is the difference of two neighbours.
+                                    const uint32_t mk = 0x01010101u * (uint32_t)((0xFFu << (g * CB)) & 0xFFu);
+                                    mma_u8s8(acc2[h][g], e0 & mk, o0 & mk, e1 & mk, o1 & mk, b0, b1);
+                                }
+                            }
                         }
                     }
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty + slot));
+                    mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty_b + ring.slot));
                     mbar_arrive(reinterpret_cast<uint64_t*>(sh->rempty + rbuf));
                 }
+                ring.next(a.slots_b);
             }
-            if (p == 0 && lane == 0) col_mark(a, t_rel, 4);
-            // ---- the step's gradient of the own features; update; digits of the next w
+            const long long u0c = (a.trace && p == 0) ? clock64() : 0;
+            // ---- the step's gradient of the own features; update
             // lane (g, t): acc[gi][0..1] = digits 2t, 2t+1 of byte 2g, acc[gi][2..3] of byte 2g+1
+            int acc[NG][4];
+#pragma unroll
+            for (int g = 0; g < NG; ++g)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[g][e] = acc2[0][g][e] + acc2[1][g][e];
             const ColStepParams& sp = sh->sp[t_rel & 1];
             const double delta_r = sp.delta_r, lo_term = sp.delta_r * sp.rsum, scale = 1.0 / (2.0 * (double)st.bt);
             const double w0 = (tl == 0) ? 1.0 : (tl == 1) ? 16384.0 : (tl == 2) ? 268435456.0 : 4398046511104.0;     // 128^(2t)
@@ -483,120 +655,194 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     if (last) a.x[jo[e]] = xo[e];
                 }
             }
-            if (last) break;
-            publish_w((int)((t_rel + 1) & 1));
-            if (p == 0 && lane == 0) col_mark(a, t_rel, 5);
+            if (p == 0 && lane == 0) col_tally(a, t_rel, 6, clock64() - u0c);
         }
     }
     // =================================================================================== R warps: residual digits
     else {
+        // Each R warp works alone on the chunks q = rw (mod kColRWarps) of the launch's sequence, with a digit buffer
+        // of its own: that many exchanges are in flight at a time.  The warps meet twice per step: for the largest
+        // |label| and for the step's sums.
         const int rt = tid - 32 * kColWarpR0, rw = rt >> 5;
-        int64_t q = 0;
+        int q0 = 0;                                      // the step's first chunk in the launch's sequence
         bool ok = true;                                  // (after a failure: as for the B warps)
         const double grow = a.reg == ZIPML_REG_LSSVM ? fmax(1.0, fabs(1.0 - (double)a.reg_cst)) : 1.0;
-        const int zper = (a.bpad + G - 1) / G;           // rows of a dots buffer that this CTA clears
-        for (int64_t t_rel = 0; t_rel < steps; ++t_rel) {
+        const int zper = (a.bpad + G - 1) / G;           // rows of a buffer of dot words that this CTA clears
+        const int ngrp = a.ngrp;
+        const int last_size = G - (ngrp - 1) * a.gsize;  // CTAs of the last group
+        signed char* rd = rdig + (size_t)rw * 2 * NRD * rstride;
+#pragma unroll 1
+        for (int t_rel = 0; t_rel < steps; ++t_rel) {
             const ColStep st = col_step(a, a.first_step + t_rel);
             const ColStepParams& sp = sh->sp[t_rel & 1];
-            const long long* dots = a.dots + (size_t)(t_rel % 3) * 2 * a.bpad;
+            const long long* dots = a.dots + (size_t)(t_rel % 3) * ngrp * 2 * a.bpad;
             // the step's largest |label| completes the bound of its residuals
             float bm = 0.0f;
+#pragma unroll 1
             for (int k = rt; k < st.bt; k += kColRThreads) bm = fmaxf(bm, fabsf(__ldg(a.b + st.row0 + k)));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
             if (lane == 0) sh->red_f[1][rw] = bm;
             named_barrier(kColNamedR, kColRThreads);
-            bm = fmaxf(fmaxf(sh->red_f[1][0], sh->red_f[1][1]), fmaxf(sh->red_f[1][2], sh->red_f[1][3]));
+            bm = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kColRWarps; ++w) bm = fmaxf(bm, sh->red_f[1][w]);
             const double rbound = (dbound + (double)bm) * 1.0001;
             const double inv_r = rbound > 0.0 ? (double)kColQmaxR / rbound : 0.0;
             const double U = sp.U;
             double rmax = 0.0;
             long long rs_hi = 0, rs_lo = 0;              // sum of the fixed-point residuals: high parts and low 28 bits
-            for (int c = 0; c < st.nch; ++c, ++q) {
-                const int rbuf = (int)(q & 1);
-                // ---- all CTAs' parts of the chunk's dots have arrived
-                if (rt == 0 && ok) {
-                    const unsigned* cnt = a.count + (size_t)(q & (a.ring - 1)) * 32;
-                    const unsigned target = (unsigned)((q / a.ring + 1) * G);
-                    const long long t0 = clock64();
-                    for (int spin = 0;; ++spin) {
-                        unsigned v;
-                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(cnt) : "memory");
-                        if (v >= target) break;
-                        if ((spin & 31) == 31) {
-                            if (col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0) { sh->abort_flag = 1; break; }
-                            if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 75); break; }
+            const int c_last = st.nch - 1;
+#pragma unroll 1
+            for (int c = (rw - q0) & (kColRWarps - 1); c < st.nch; c += kColRWarps) {
+                const int q = q0 + c;
+                // A lane takes the four rows whose digits make one 32-bit word of pass B's operand: rows 2t, 2t+1, 8+2t,
+                // 9+2t of half `hf` of the 32-row block `blk` (k index 4t + i <-> row 2t + (i & 1) + 8 (i >> 1)).
+                const int blk = lane >> 3, hf = (lane >> 2) & 1;
+                const int kkA = blk * 32 + 16 * hf + 2 * tl;           // the first of them within the chunk
+                const int kA = c * R + kkA;                              // and within the step
+                const bool mine = kkA < R && kA < st.bt;
+                float bk[4];                                             // the labels wait for nobody
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int k = kA + (i & 1) + 8 * (i >> 1);
+                    bk[i] = (mine && k < st.bt) ? __ldg(a.b + st.row0 + k) : 0.0f;
+                }
+                // ---- the chunk's dots.  First a few lanes watch the last row of each 32-row task and group (one request
+                // per look, with a pause: five hundred warps looking at L2 as fast as it answers would take a good part
+                // of its bandwidth), then every lane reads its own rows' words until their counts are complete too.
+                const long long t0 = clock64();
+                if (lane < 4 * ngrp && ok) {
+                    const int g = lane >> 2, first = c * R + 32 * (lane & 3);
+                    if (first < st.bt && 32 * (lane & 3) < R) {
+                        const long long* wl = dots + ((size_t)g * 2 + 1) * a.bpad + min(st.bt, first + 32) - 1;
+                        const int want = g == ngrp - 1 ? last_size : a.gsize;
+#pragma unroll 1
+                        for (int spin = 0;; ++spin) {
+                            long long v0;
+                            asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(v0) : "l"(wl) : "memory");
+                            if ((int)(v0 & 0xFF) >= want) break;
+                            if ((spin & 15) == 15) {
+                                if (col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0) { sh->abort_flag = 1; break; }
+                                if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 75); break; }
+                            }
+                            __nanosleep(200);
                         }
                     }
-                    if (c == 0) col_mark(a, t_rel, 7);
-                    if (c == st.nch - 1) col_mark(a, t_rel, 2);
-                }
-                named_barrier(kColNamedR, kColRThreads);
-                ok = ok && !col_aborted(sh);
-                // every CTA has left step t - 1 behind: its dots buffer is cleared for step t + 2 (this CTA's
-                // share; the stores precede this CTA's counter arrivals of step t + 1, which every adder waits for)
-                if (c == 0 && ok) {
-                    long long* z = a.dots + (size_t)((t_rel + 2) % 3) * 2 * a.bpad;
-                    const int z0 = cta * zper, z1 = min(a.bpad, z0 + zper);
-                    for (int i = z0 + rt; i < z1; i += kColRThreads) { z[i] = 0; z[a.bpad + i] = 0; }
-                }
-                if (ok && q >= 2) ok = col_wait(sh->rempty + rbuf, (uint32_t)(((q >> 1) - 1) & 1), sh, a.status, 76);
-                signed char* rd = rdig + (size_t)rbuf * 2 * NRD * rstride;
-                for (int kk = rt; kk < R && ok; kk += kColRThreads) {
-                    const int k = c * R + kk;
-                    long long R1 = 0, R2 = 0;
-                    if (k < st.bt) {
-                        const double bk = (double)__ldg(a.b + st.row0 + k);
-                        const double r1 = (double)__ldcg(dots + k) * U - bk, r2 = (double)__ldcg(dots + a.bpad + k) * U - bk;
-                        rmax = fmax(rmax, fmax(fabs(r1), fabs(r2)));
-                        R1 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r1 * inv_r)));
-                        R2 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r2 * inv_r)));
-                        rs_hi += (R1 >> 28) + (R2 >> 28);
-                        rs_lo += (R1 & 0xFFFFFFFll) + (R2 & 0xFFFFFFFll);
-                    }
-                    // row rho of a 32-row block sits where the transposed code fragments look for it:
-                    // k index 4t + i <-> row 2t + (i & 1) + 8 (i >> 1), second half 16 rows further
-                    const int rho = kk & 31, r16 = rho & 15;
-                    signed char* dst = rd + (kk >> 5) * 32 + ((r16 & 7) >> 1) * 8 + (rho >> 4) * 4 + (r16 & 1) + 2 * (r16 >> 3);
-                    long long W1 = R1, W2 = R2;
-#pragma unroll
-                    for (int s = 0; s < NRD; ++s) {
-                        int d1, d2;
-                        if (s < NRD - 1) {
-                            d1 = (int)((W1 + 64) & 127) - 64; W1 = (W1 - d1) >> 7;
-                            d2 = (int)((W2 + 64) & 127) - 64; W2 = (W2 - d2) >> 7;
-                        } else { d1 = (int)W1; d2 = (int)W2; }
-                        dst[(size_t)s * rstride] = (signed char)d2;                    // plane 1 meets r2
-                        dst[(size_t)(NRD + s) * rstride] = (signed char)d1;            // plane 2 meets r1
-                    }
-                }
-                if (c == st.nch - 1) {
-                    // ---- the step's residuals are all known: their sum for the B warps, the next step's bound and unit
-                    rmax = fmax(rmax, __shfl_xor_sync(0xffffffffu, rmax, 16));
-#pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) rmax = fmax(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) { rs_hi += __shfl_xor_sync(0xffffffffu, rs_hi, o); rs_lo += __shfl_xor_sync(0xffffffffu, rs_lo, o); }
-                    if (lane == 0) { sh->red_d[1][rw] = rmax; sh->red_l[0][rw] = rs_hi; sh->red_l[1][rw] = rs_lo; }
-                    named_barrier(kColNamedR, kColRThreads);
-                    double rm = 0.0;
-                    long long hi = 0, lo = 0;
-#pragma unroll
-                    for (int w = 0; w < kColRWarps; ++w) { rm = fmax(rm, sh->red_d[1][w]); hi += sh->red_l[0][w]; lo += sh->red_l[1][w]; }
-                    dbound = (dbound * grow + fabs((double)a.lr) * rm * c2) * 1.0001;
-                    if (rt == 0) {
-                        ColStepParams& cur = sh->sp[t_rel & 1];
-                        cur.inv_r = inv_r;
-                        cur.delta_r = rbound / (double)kColQmaxR;
-                        cur.rsum = (double)hi * 268435456.0 + (double)lo;
-                        unit_of(dbound, sh->sp[(t_rel + 1) & 1].U, sh->sp[(t_rel + 1) & 1].invU);
-                    }
-                    named_barrier(kColNamedR, kColRThreads);       // (red_* free again; the parameters precede the arrivals)
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rbuf));
-                if (rt == 0 && c == st.nch - 1) col_mark(a, t_rel, 3);
+                ok = __all_sync(0xffffffffu, ok && !col_aborted(sh));          // (the warp acts as one)
+                if (a.trace && rw == 0 && lane == 0) col_tally(a, t_rel, 2, clock64() - t0);
+                long long D1[4], D2[4];                                  // the rows' dots: sums over the groups' words
+#pragma unroll 1
+                for (int spin = 0;; ++spin) {
+                    bool done = true;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { D1[i] = 0; D2[i] = 0; }
+                    if (mine && ok) {
+#pragma unroll 1
+                        for (int g = 0; g < ngrp; ++g) {
+                            const long long* s1 = dots + (size_t)g * 2 * a.bpad + kA;
+                            const int want = g == ngrp - 1 ? last_size : a.gsize;
+                            long long w1[4], w2[4];
+                            ld_l2_v2(s1, w1[0], w1[1]);
+                            ld_l2_v2(s1 + 8, w1[2], w1[3]);
+                            ld_l2_v2(s1 + a.bpad, w2[0], w2[1]);
+                            ld_l2_v2(s1 + a.bpad + 8, w2[2], w2[3]);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                if (kA + (i & 1) + 8 * (i >> 1) < st.bt) done = done && (int)(w1[i] & 0xFF) >= want && (int)(w2[i] & 0xFF) >= want;
+                                D1[i] += w1[i] >> 8;
+                                D2[i] += w2[i] >> 8;
+                            }
+                        }
+                    }
+                    if (__all_sync(0xffffffffu, done) || !ok) break;
+                    __nanosleep(100);
+                    if ((spin & 7) == 7) {
+                        bool give_up = col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0;
+                        if (clock64() - t0 > kColWaitCycles) { set_status(a.status, ZIPML_ERR_TIMEOUT, 77); give_up = true; }
+                        if (__any_sync(0xffffffffu, give_up)) { sh->abort_flag = 1; ok = false; }
+                    }
+                }
+                // every CTA has left step t - 1 behind: its buffer of dot words is cleared for step t + 2 (this CTA's share)
+                if (c == 0 && ok) {
+                    __threadfence();        // (see "Memory order" above: the others' reads of that buffer before these stores)
+                    long long* z = a.dots + (size_t)((t_rel + 2) % 3) * ngrp * 2 * a.bpad;
+                    const int z0 = cta * zper, z1 = min(a.bpad, z0 + zper);
+#pragma unroll 1
+                    for (int g = 0; g < 2 * ngrp; ++g)
+#pragma unroll 1
+                        for (int i = z0 + lane; i < z1; i += 32) z[(size_t)g * a.bpad + i] = 0;
+                }
+                const long long e0c = (a.trace && rw == 0) ? clock64() : 0;
+                if (ok && q >= kColRWarps) ok = col_wait(sh->rempty + rw, (uint32_t)(((q >> kColRShift) - 1) & 1), sh, a.status, 76);
+                ok = __all_sync(0xffffffffu, ok);
+                if (a.trace && rw == 0 && lane == 0) col_tally(a, t_rel, 3, clock64() - e0c);
+                if (kkA < R && ok) {
+                    // residuals r = U * dot - label in fixed point, then their digits: with 64 added to every digit the
+                    // number is plain base 128 (no carry chain); four rows' digits make a word
+                    unsigned long long u1[4], u2[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        long long R1 = 0, R2 = 0;
+                        if (kA + (i & 1) + 8 * (i >> 1) < st.bt) {
+                            const double r1 = (double)D1[i] * U - (double)bk[i], r2 = (double)D2[i] * U - (double)bk[i];
+                            rmax = fmax(rmax, fmax(fabs(r1), fabs(r2)));
+                            R1 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r1 * inv_r)));
+                            R2 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r2 * inv_r)));
+                            rs_hi += (R1 >> 28) + (R2 >> 28);
+                            rs_lo += (R1 & 0xFFFFFFFll) + (R2 & 0xFFFFFFFll);
+                        }
+                        u1[i] = (unsigned long long)(R1 + kColBiasR);
+                        u2[i] = (unsigned long long)(R2 + kColBiasR);
+                    }
+                    signed char* dst = rd + blk * 32 + tl * 8 + hf * 4;
+#pragma unroll
+                    for (int s = 0; s < NRD; ++s) {
+                        uint32_t wa = 0u, wb = 0u;                       // digit s of r2 (meets plane 1) and of r1 (meets plane 2)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            wa |= (uint32_t)((u2[i] >> (7 * s)) & 127ull) << (8 * i);
+                            wb |= (uint32_t)((u1[i] >> (7 * s)) & 127ull) << (8 * i);
+                        }
+                        wa ^= 0x40404040u; wa |= (wa & 0x40404040u) << 1;      // every byte minus 64, as a signed byte
+                        wb ^= 0x40404040u; wb |= (wb & 0x40404040u) << 1;
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)s * rstride) = wa;
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)(NRD + s) * rstride) = wb;
+                    }
+                }
+                if (c != c_last) {                       // (the step's last chunk is released below, after the step's sums)
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rw));
+                }
             }
+            // ---- the step's residuals are all known: their sum for the B warps, the next step's bound and unit
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                rmax = fmax(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+                rs_hi += __shfl_xor_sync(0xffffffffu, rs_hi, o);
+                rs_lo += __shfl_xor_sync(0xffffffffu, rs_lo, o);
+            }
+            if (lane == 0) { sh->red_d[1][rw] = rmax; sh->red_l[0][rw] = rs_hi; sh->red_l[1][rw] = rs_lo; }
+            named_barrier(kColNamedR, kColRThreads);     // (the next step's barrier keeps these slots from being rewritten early)
+            double rm = 0.0;
+            long long hi = 0, lo = 0;
+#pragma unroll
+            for (int w = 0; w < kColRWarps; ++w) { rm = fmax(rm, sh->red_d[1][w]); hi += sh->red_l[0][w]; lo += sh->red_l[1][w]; }
+            dbound = (dbound * grow + fabs((double)a.lr) * rm * c2) * 1.0001;
+            if (((q0 + c_last) & (kColRWarps - 1)) == rw) {      // the warp that holds the step's last chunk
+                if (lane == 0) {
+                    ColStepParams& cur = sh->sp[t_rel & 1];
+                    cur.inv_r = inv_r;
+                    cur.delta_r = rbound / (double)kColQmaxR;
+                    cur.rsum = (double)hi * 268435456.0 + (double)lo;
+                    col_unit_of(dbound, sh->sp[(t_rel + 1) & 1].U, sh->sp[(t_rel + 1) & 1].invU);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rw));
+            }
+            q0 += st.nch;
         }
     }
     __syncthreads();
@@ -611,8 +857,8 @@ static const void* column_kernel_ptr(int cb) {
     return reinterpret_cast<const void*>(&sgd_column_kernel<8>);
 }
 
-// Tensor maps over the two planes as m x row_bytes byte matrices: boxes of 128 bytes x R rows with the
-// 128-byte swizzle, bytes past the row or the last row read as zero.  The encoder is a driver entry
+// Tensor maps over the two planes as byte matrices: boxes of 128 bytes x R rows with the 128-byte swizzle,
+// bytes past the row or the matrix's last row read as zero.  The encoder is a driver entry
 // point looked up through the runtime (no link against the driver library).
 static int encode_column_maps(zipml_ctx* ctx, const zipml_dataset* d, int R, CUtensorMap* out) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -628,8 +874,11 @@ static int encode_column_maps(zipml_ctx* ctx, const zipml_dataset* d, int R, CUt
         }
         ctx->tmap_encode = fn;
     }
-    const cuuint64_t gdim[2] = {(cuuint64_t)d->row_bytes, (cuuint64_t)d->m};
-    const cuuint64_t gstride[1] = {(cuuint64_t)d->row_bytes};
+    // row-major: m x row_bytes; column blocks: (blocks * m) pieces of 128 bytes, a CTA's rows one after the other
+    const bool blocks = d->layout == ZIPML_LAYOUT_COLUMN_BLOCKS;
+    const cuuint64_t nblk = (cuuint64_t)((d->row_bytes + kColBlockBytes - 1) / kColBlockBytes);
+    const cuuint64_t gdim[2] = {blocks ? (cuuint64_t)kColBlockBytes : (cuuint64_t)d->row_bytes, blocks ? nblk * (cuuint64_t)d->m : (cuuint64_t)d->m};
+    const cuuint64_t gstride[1] = {blocks ? (cuuint64_t)kColBlockBytes : (cuuint64_t)d->row_bytes};
     const cuuint32_t box[2] = {(cuuint32_t)kColBlockBytes, (cuuint32_t)R};
     const cuuint32_t estr[2] = {1, 1};
     const void* planes[2] = {d->plane1, d->plane2};
@@ -648,6 +897,7 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     if (!ctx->cooperative) return ZIPML_ERR_WORKSPACE;
     if (d->level_mode != ZIPML_LEVELS_UNIFORM || p->model_bits != 0 || p->grad_bits != 0 || p->model_out) return ZIPML_ERR_WORKSPACE;
     if (d->m > 0x7fffffffLL || d->row_bytes < kColBlockBytes) return ZIPML_ERR_WORKSPACE;
+    if ((d->row_bytes + kColBlockBytes - 1) / kColBlockBytes * d->m > 0x7fffffffLL) return ZIPML_ERR_WORKSPACE;     // (32-bit copy coordinates)
     const int cb = container_bits(d->bits);
     const int ng = 8 / cb;
     const int64_t T = (d->m + p->batch - 1) / p->batch;
@@ -658,17 +908,31 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     // worth it where the rows occupy most of the device and a step holds several chunks
     if (only_if_profitable && (G < ctx->sm_count / 2 || B < 256)) return ZIPML_ERR_WORKSPACE;
     int R = p->column_chunk_rows > 0 ? p->column_chunk_rows : 128;
+    if (R > kColMaxChunkRows) R = kColMaxChunkRows;
     if (R > (B + 31) / 32 * 32) R = (int)((B + 31) / 32 * 32);
     const int nch_max = (int)((B + R - 1) / R);
     const int bpad = nch_max * R;
-    int ring = 16;
-    while (ring < 2 * nch_max + 2 * kColMaxSlots) ring *= 2;
+    // One dot word per row and plane for all CTAs (tuning: grid_feature_parts = words, each shared by a group of
+    // CTAs).  Same-address atomics are served one after the other, but more words cost the readers more than the
+    // shorter queues give back: measured on 128 CTAs, 16 KB rows: 26.3 / 27.8 / 30.8 us per step with 1 / 2 / 4 words.
+    int ngrp = p->grid_feature_parts > 0 ? p->grid_feature_parts : 1;
+    if (ngrp > kColMaxGroups) ngrp = kColMaxGroups;
+    if (ngrp > G) ngrp = (int)G;
+    int gsize = (int)((G + ngrp - 1) / ngrp);
+    while (ngrp > 1 && (int64_t)(ngrp - 1) * gsize >= G) --ngrp;       // no empty group
 
     const size_t slot_bytes = (size_t)2 * R * kColBlockBytes;
-    const size_t fixed = 1024 + (size_t)2 * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 4 * 32 + 16 + sizeof(ColShared);
-    if (fixed + 2 * slot_bytes > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
+    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 4 * 32 + 16 + sizeof(ColShared);
+    if (fixed + 4 * slot_bytes > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
     int slots = (int)(((size_t)ctx->smem_optin - fixed) / slot_bytes);
-    if (slots > kColMaxSlots) slots = kColMaxSlots;
+    if (slots > 2 * kColMaxSlots) slots = 2 * kColMaxSlots;
+    // the first visits come from HBM and need the deeper ring (tuning: grid_row_parts = slots of the B ring)
+    int slots_b = p->grid_row_parts > 0 ? p->grid_row_parts : slots / 3;
+    if (slots_b < 2) slots_b = 2;
+    if (slots_b > slots - 2) slots_b = slots - 2;
+    if (slots_b > kColMaxSlots) slots_b = kColMaxSlots;
+    int slots_a = slots - slots_b;
+    if (slots_a > kColMaxSlots) slots_a = kColMaxSlots;
     const size_t smem = fixed + (size_t)slots * slot_bytes;
     const void* kernel = column_kernel_ptr(cb);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -684,8 +948,7 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
 
     size_t off = 0;
     auto piece = [&](size_t bytes) { const size_t o = off; off += carve_size(bytes); return o; };
-    const size_t o_count = piece(sizeof(unsigned) * 32 * (size_t)ring);
-    const size_t o_dots = piece(sizeof(long long) * 3 * 2 * (size_t)bpad);
+    const size_t o_dots = piece(sizeof(long long) * 3 * 2 * (size_t)bpad * ngrp);
     const size_t zero_bytes = off;
     const size_t o_ord = piece(sizeof(int32_t) * (size_t)(p->batch_order ? T : 0));
     rc = ws_reserve(ctx, off);
@@ -694,34 +957,27 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     ColumnArgs a;
     memset(&a, 0, sizeof(a));
     a.m = d->m; a.batch = B; a.lo = d->feat_lo; a.step = d->feat_step; a.b = b; a.x = x; a.grad_out = grad_out;
-    a.n = (int)d->n; a.bits = d->bits; a.R = R; a.slots = slots; a.bpad = bpad; a.ring = ring;
+    a.n = (int)d->n; a.bits = d->bits; a.R = R; a.slots_a = slots_a; a.slots_b = slots_b; a.bpad = bpad;
+    a.ngrp = ngrp; a.gsize = gsize; a.blocked = d->layout == ZIPML_LAYOUT_COLUMN_BLOCKS;
     a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p);
-    a.count = reinterpret_cast<unsigned*>(ctx->ws + o_count);
     a.dots = reinterpret_cast<long long*>(ctx->ws + o_dots);
     a.status = ctx->d_status;
     a.trace = reinterpret_cast<unsigned long long*>(p->trace);
     a.trace_steps = p->trace ? p->trace_steps : 0;
+    a.first_step = first_step;
+    a.num_steps = num_steps;
     if (p->batch_order) {
         int32_t* dev_order = reinterpret_cast<int32_t*>(ctx->ws + o_ord);
         e = cudaMemcpyAsync(dev_order, p->batch_order, sizeof(int32_t) * (size_t)T, cudaMemcpyHostToDevice, ctx->stream);
         if (e != cudaSuccess) return cuda_status(e);
         a.order = dev_order;
     }
-    // the chunk counters are 32-bit: (chunks of a launch / ring + 1) * G must stay below 2^31
-    const int64_t max_steps = ((int64_t)(0x7fffffff / G) - 2) * ring / nch_max;
-    for (int64_t s0 = first_step; s0 < first_step + num_steps; s0 += max_steps) {
-        e = cudaMemsetAsync(ctx->ws, 0, zero_bytes, ctx->stream);
-        if (e != cudaSuccess) return cuda_status(e);
-        ColumnArgs chunk = a;
-        chunk.first_step = s0;
-        chunk.num_steps = (first_step + num_steps - s0 < max_steps) ? first_step + num_steps - s0 : max_steps;
-        if (s0 + chunk.num_steps < first_step + num_steps) chunk.grad_out = nullptr;
-        if (s0 > first_step) { chunk.trace = nullptr; chunk.trace_steps = 0; }
-        void* params[] = {&chunk, &tmaps[0], &tmaps[1]};
-        e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kColThreads), params, smem, ctx->stream);
-        if (e != cudaSuccess) return cuda_status(e);
-        ctx->launches += 1;
-    }
+    e = cudaMemsetAsync(ctx->ws, 0, zero_bytes, ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    void* params[] = {&a, &tmaps[0], &tmaps[1]};
+    e = cudaLaunchCooperativeKernel(kernel, dim3((unsigned)G), dim3(kColThreads), params, smem, ctx->stream);
+    if (e != cudaSuccess) return cuda_status(e);
+    ctx->launches += 1;
     ctx->last_engine = ZIPML_ENGINE_COLUMN;
     return ZIPML_OK;
 }

@@ -95,6 +95,9 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 __device__ __forceinline__ void st_relaxed_u32(unsigned* p, unsigned v) {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_add_s64(long long* p, long long v) {
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "l"(v) : "memory");
+}
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
     uint64_t pol;
@@ -323,8 +326,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) sgd_stream_kernel(const Str
                     const long long v2 = q2 + 16384ll * __shfl_down_sync(0xffffffffu, q2, 1);
                     const int k = rblk * 16 + gl + 8 * e;
                     if (active && tl == 0 && k < bt) {
-                        atomicAdd(reinterpret_cast<unsigned long long*>(dots + k), (unsigned long long)v1);
-                        atomicAdd(reinterpret_cast<unsigned long long*>(dots + a.bpad + k), (unsigned long long)v2);
+                        // (a reduction that returns nothing: the warp does not wait for an old value it never reads)
+                        red_add_s64(dots + k, v1);
+                        red_add_s64(dots + a.bpad + k, v2);
                     }
                 }
                 __syncthreads();           // the next unit overwrites the staged digits

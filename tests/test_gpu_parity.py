@@ -304,6 +304,16 @@ def test_column_engine(ctx, case):
     T = (m + batch - 1) // batch
     order = np.random.default_rng(5).permutation(T).astype(np.int32)
     kw = dict(engine=binding.ENGINE_COLUMN, column_chunk_rows=chunk, batch_order=order)
+    # the same planes cut into 128-byte column blocks: the layout is what a plain reshape of the oracle's planes gives
+    bds = ctx.zipml_convert_layout(gds, binding.LAYOUT_COLUMN_BLOCKS)
+    nblk = (ods.row_bytes + 127) // 128
+    for got, plane in ((bds.plane1, ods.plane1), (bds.plane2, ods.plane2)):
+        padded = np.zeros((m, nblk * 128), np.uint8)
+        padded[:, : ods.row_bytes] = plane
+        assert (got.cpu().numpy().reshape(nblk, m, 128) == padded.reshape(m, nblk, 128).transpose(1, 0, 2)).all()
+    back = ctx.zipml_convert_layout(bds, binding.LAYOUT_ROWS)
+    ctx.zipml_sync()
+    assert (back.plane1.cpu().numpy() == ods.plane1).all() and (back.plane2.cpu().numpy() == ods.plane2).all()
     for x0 in (np.zeros(n, np.float32), (np.random.default_rng(4).standard_normal(n) * 0.05).astype(np.float32)):
         x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order)
         x_before, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order, num_steps=T - 1)
@@ -317,6 +327,10 @@ def test_column_engine(ctx, case):
             runs.append(x.cpu().numpy())
             assert rel(runs[-1], x_ref) <= MODEL_TOL
         assert (runs[0] == runs[1]).all()                 # integer sums and fixed orders: the same bits run to run
+        x = to_dev(x0, ctx)
+        ctx.zipml_sgd_epoch(bds, db, x, batch, lr, **{**kw, "engine": binding.ENGINE_AUTO})      # from the column blocks
+        ctx.zipml_sync()
+        assert ctx.zipml_last_engine() == binding.ENGINE_COLUMN and (x.cpu().numpy() == runs[0]).all()
         xb = to_dev(x_before, ctx)
         g = torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
         ctx.zipml_sgd_epoch(gds, db, xb, batch, lr, first_step=T - 1, num_steps=1, grad_out=g, **kw)
@@ -334,6 +348,13 @@ def test_column_engine(ctx, case):
         with pytest.raises(binding.ZipmlError) as e:
             ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=binding.ENGINE_COLUMN, **bad)
         assert e.value.code == binding.ERR_WORKSPACE
+    for engine in (binding.ENGINE_STREAM, binding.ENGINE_RING, binding.ENGINE_CLUSTER):     # the other engines read rows only
+        with pytest.raises(binding.ZipmlError) as e:
+            ctx.zipml_sgd_epoch(bds, db, to_dev(x0, ctx), batch, lr, engine=engine)
+        assert e.value.code == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_loss(binding.LOSS_CODES, db, to_dev(x0, ctx), data=bds)
+    assert e.value.code == binding.ERR_UNSUPPORTED
 
 
 def test_column_engine_limits(ctx):
