@@ -3,12 +3,15 @@
 
 A "step" is one pass of the whole path over one synthetic workload: quantize the dense fp32
 samples into two packed planes (after placing variance-optimal levels, if the workload asks for
-them), run the workload's SGD epochs over the planes, evaluate the dense training loss.
+them), run the workload's SGD epochs over the planes, evaluate the dense training loss.  The
+default workload is the largest configuration (c5).
 
-  value         samples/s = (m * epochs) / step time, inputs already resident in device memory
-  e2e           the same through zipml_train_host with pinned HOST buffers (copies in the timed region)
+  value         samples/s per SGD epoch = m / mean duration of a zipml_sgd_epoch launch (CUDA events),
+                planes resident in device memory; `whole_path_samples_per_s` beside it counts the
+                whole pass (quantize + epochs + loss)
+  e2e           the whole pass through zipml_train_host with pinned HOST buffers (copies in the timed region)
   roofline      packed-code bytes per SGD-epoch launch / its CUDA-event duration, against the
-                measured HBM copy rate
+                measured HBM copy rate; `latency_model` next to it: what the minibatch chain allows
   cpu_baseline  the CPU oracle as it stands, timed on this host (rank 0, N = 1 only)
 
 `--impl reference` times the oracle alone (the reference arm of this tier).
@@ -29,10 +32,13 @@ if ROOT not in sys.path:
 
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one epoch launch from the ncu capture summarised under profiles/
-# (workload, engine) -> bytes; an entry is removed when its kernel changes after the capture
-# (c5: captured on 16,384 of the 65,536 rows, 591.80 + 6.29 MB, and scaled by the rows: traffic grows with them)
-NCU_TRAFFIC_BYTES = {("c2", 5): 203.04e6 + 3.76e6, ("c5", 6): 4 * (591.80e6 + 6.29e6)}
+# dram__bytes_read.sum + dram__bytes_write.sum of one epoch launch, quoted from the ncu captures summarised under
+# profiles/ (a run cannot measure them itself): (workload, engine) -> (bytes, where they come from)
+NCU_TRAFFIC = {
+    ("c2", 5): (203.04e6 + 3.76e6, "profiles/sgd_cluster_kernel_c2_full.md"),
+    ("c5", 6): (4 * (591.80e6 + 6.29e6), "profiles/sgd_stream_kernel_c5_full.md, 16,384-row capture scaled x4 by the rows"),
+    ("c5", 7): (4 * (537.81e6 + 6.83e6), "profiles/sgd_column_kernel_c5_full.md, 16,384-row capture scaled x4 by the rows"),
+}
 ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
                   5: "sgd_cluster_kernel", 6: "sgd_stream_kernel", 7: "sgd_column_kernel"}
 
@@ -85,8 +91,27 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(mhz)}
 
 
+def latency_model(ctx, engine_ran, n, step_bytes, peak_gbs):
+    """What the minibatch chain allows: a step moves step_bytes and cannot start before the previous step's model
+    exists, so it costs at least step_bytes / BW plus its exchanges between SMs (measured here with the library's
+    communication skeleton: publish through L2, bounded-spin barrier, read the others' data).  ceiling_frac =
+    S / (S / BW + k t_exchange) / BW with t_compute taken as zero: an upper bound on roofline.frac."""
+    k = 1 if engine_ran in (6, 7) else 2           # stream, column: the dots; the others: gradient parts out, model back
+    ctas = {5: 16}.get(engine_ran, 128)            # the cluster engine is one cluster of at most 16 CTAs
+    floats = max(4, (n // ctas + 3) // 4 * 4)
+    try:
+        t_ns = ctx.zipml_barrier_latency(ctas, floats, 2000)
+    except Exception:
+        return None
+    t_stream_us = step_bytes / (peak_gbs * 1e3)
+    floor_us = k * t_ns * 1e-3
+    return {"exchanges_per_step": k, "ctas": ctas, "t_exchange_us": t_ns * 1e-3, "chain_floor_us": floor_us,
+            "us_per_step_at_copy_rate": t_stream_us, "ceiling_frac": t_stream_us / (t_stream_us + floor_us),
+            "note": "t_compute = 0; exchange measured with zipml_barrier_latency in this run"}
+
+
 def run_oracle_pass(w, A, b, max_seconds=None):
-    """One pass of the whole path on the CPU oracle; returns (seconds, samples processed, x, loss)."""
+    """One pass of the whole path on the CPU oracle; returns (seconds, samples processed, x, loss, seconds in SGD epochs)."""
     import numpy as np
     import oracle
     t0 = time.perf_counter()
@@ -96,11 +121,13 @@ def run_oracle_pass(w, A, b, max_seconds=None):
     ds = oracle.quantize(A, w.bits, seed=w.seed, mode=oracle.TABLE if levels is not None else oracle.UNIFORM,
                          levels=levels)
     x = np.zeros(w.n, np.float32)
+    te = time.perf_counter()
     for ep in range(w.epochs):
         x, _ = oracle.sgd_epoch(ds, b, x, w.batch, w.lr, model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed,
                                 epoch=ep)
+    te = time.perf_counter() - te
     loss = oracle.loss_dense(A, b, x)
-    return time.perf_counter() - t0, w.m * w.epochs, x, loss
+    return time.perf_counter() - t0, w.m * w.epochs, x, loss, te
 
 
 def oracle_sample_rows(w):
@@ -118,7 +145,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
+    ap.add_argument("--workload", default="c5", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
     ap.add_argument("--m", type=int, default=None, help="override the number of samples (smaller profiling cases)")
     ap.add_argument("--engine", default="auto", choices=["auto", "stepwise", "persistent", "ring", "lean", "cluster", "stream", "column"])
     ap.add_argument("--chunk-rows", type=int, default=0, help="column engine: rows per chunk (0 = automatic)")
@@ -136,7 +163,7 @@ def main():
 
     from paper_1611_05402_b200 import synth
     base = synth.WORKLOADS[args.workload]
-    metric, unit = "samples/sec over the whole path (quantize + SGD epochs + loss)", "samples/s"
+    metric, unit = "samples/sec and packed-code HBM GB/s per SGD epoch (fraction of B200 peak)", "samples/s"
 
     # ------------------------------------------------------------------ reference arm: the oracle
     if args.impl == "reference":
@@ -156,12 +183,14 @@ def main():
         A, b = A.numpy(), b.numpy()
         for _ in range(args.warmup):
             run_oracle_pass(w, A, b)
-        t = 0.0
+        t, t_ep = 0.0, 0.0
         for _ in range(args.steps):
-            dt, samples, _, _ = run_oracle_pass(w, A, b)
+            dt, samples, _, _, te = run_oracle_pass(w, A, b)
             t += dt
-        value = samples * args.steps / t
-        sample = f"first {rows} of {w0.m} rows of {args.workload}, all {w.epochs} epochs, single thread"
+            t_ep += te
+        value = samples * args.steps / t_ep            # samples/s per SGD epoch, like the other arm's value
+        sample = (f"first {rows} of {w0.m} rows of {args.workload}, all {w.epochs} epochs, single thread; "
+                  f"whole path (quantize + epochs + loss): {samples * args.steps / t:.0f} samples/s")
         print(json.dumps({
             "impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -240,7 +269,7 @@ def main():
     clocks = sampler.stop()
     ctx.zipml_sync()
     launches = ctx.zipml_kernel_launches() - launches0
-    value, ms_total = replicas.whole_job_value(w.m * w.epochs * args.steps, t0.elapsed_time(t1), dev)
+    whole_value, ms_total = replicas.whole_job_value(w.m * w.epochs * args.steps, t0.elapsed_time(t1), dev)
     final_loss = float(loss_dev.item())
 
     # dominant kernel: the SGD epoch launch
@@ -249,11 +278,13 @@ def main():
     packed_bytes = ds.packed_bytes
     peak, peak_kind = measured_peaks()
     achieved = packed_bytes / (epoch_avg_ms * 1e-3) / 1e9
+    value, _ = replicas.whole_job_value(w.m, epoch_avg_ms, dev)          # samples/s per SGD epoch, all ranks
     steps_per_epoch = (w.m + w.batch - 1) // w.batch
     step_us = 1e3 * epoch_avg_ms / steps_per_epoch
     step_bytes = packed_bytes / steps_per_epoch
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, ctx.zipml_last_engine())) if args.m is None else None,
+                "traffic": NCU_TRAFFIC.get((args.workload, ctx.zipml_last_engine()), (None, None))[0] if args.m is None else None,
+                "traffic_source": NCU_TRAFFIC.get((args.workload, ctx.zipml_last_engine()), (None, None))[1] if args.m is None else None,
                 "peak_kind": f"of {peak_kind} copy rate", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "kernel": ENGINE_KERNELS.get(ctx.zipml_last_engine(), "?") + " (one launch per epoch)",
                 "algorithmic_bytes_per_launch": packed_bytes,
@@ -262,7 +293,8 @@ def main():
                 # the minibatch chain is sequential: a step moves step_bytes and cannot start before the previous
                 # step's model exists, so the epoch is bound by steps * (exchange latency), not by bytes / bandwidth
                 "steps_per_launch": steps_per_epoch, "us_per_step": step_us, "bytes_per_step": step_bytes,
-                "us_per_step_at_hbm_peak": step_bytes / (peak * 1e3)}
+                "us_per_step_at_hbm_peak": step_bytes / (peak * 1e3),
+                "latency_model": latency_model(ctx, ctx.zipml_last_engine(), w.n, step_bytes, peak)}
 
     def stage(events, nbytes):
         ms_ = sorted(a_.elapsed_time(b_) for a_, b_ in events)
@@ -297,7 +329,7 @@ def main():
         h1.record()
         torch.cuda.synchronize()
         e2e_value, _ = replicas.whole_job_value(w.m * w.epochs * k_e2e, h0.elapsed_time(h1), dev)
-        e2e = {"value": e2e_value, "unit": unit,
+        e2e = {"value": e2e_value, "unit": unit, "what": "whole pass from pinned host buffers: copies, quantize, epochs, dense loss",
                "h2d_bytes_per_step": int(Ah.numel() * 4 + bh.numel() * 4 + xh.numel() * 4),
                "d2h_bytes_per_step": int(xh.numel() * 4 + 8), "steps": k_e2e, "loss": e2e_loss}
         del Ah
@@ -308,7 +340,7 @@ def main():
         others = {}
         del A
         torch.cuda.empty_cache()
-        for key in [k for k in ("c1", "c3", "c4", "c5") if k != args.workload]:
+        for key in [k for k in ("c1", "c2", "c3", "c4", "c5") if k != args.workload]:
             wo, Ao, bo, _ = synth.make(key, device=dev)
             lev = ctx.zipml_optimal_levels(Ao, wo.bits, wo.hist_bins) if wo.levels == "optimal" else None
             q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -332,11 +364,13 @@ def main():
             ctx.zipml_loss(binding.LOSS_CODES, bo, xo, data=dso, out=lc)
             l1.record()
             ctx.zipml_sync()
-            t_ep = min(a_.elapsed_time(b_) for a_, b_ in evs)
+            t_ep = sum(a_.elapsed_time(b_) for a_, b_ in evs) / len(evs)         # a mean, like the headline
             To = (wo.m + wo.batch - 1) // wo.batch
+            lm = latency_model(ctx, ctx.zipml_last_engine(), wo.n, dso.packed_bytes / To, peak)
             others[key] = {"workload": wo.name, "kernel": ENGINE_KERNELS.get(ctx.zipml_last_engine(), "?"), "epoch_ms": t_ep, "us_per_step": 1e3 * t_ep / To,
                            "samples_per_s": wo.m / (t_ep * 1e-3), "packed_GB/s": dso.packed_bytes / (t_ep * 1e-3) / 1e9,
                            "frac_of_copy_rate": dso.packed_bytes / (t_ep * 1e-3) / 1e9 / peak,
+                           "ceiling_frac": lm["ceiling_frac"] if lm else None, "chain_floor_us": lm["chain_floor_us"] if lm else None,
                            "quantize_GB/s": (8 * wo.m * wo.n + 2 * dso.m * dso.row_bytes) / (q0.elapsed_time(q1) * 1e-3) / 1e9,
                            "loss_codes_GB/s": dso.packed_bytes / (l0.elapsed_time(l1) * 1e-3) / 1e9}
             del Ao, dso, bo, xo
@@ -347,10 +381,11 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         rows = oracle_sample_rows(w)
         ws, As, bs, _ = synth.make(args.workload, m=rows)
-        dt, samples, _, _ = run_oracle_pass(ws, As.numpy(), bs.numpy())
-        cpu_baseline = {"value": samples / dt, "unit": unit, "cores": 1, "kind": "oracle",
-                        "sample": f"first {rows} of {w.m} rows of {args.workload}, whole path, all {w.epochs} epochs, "
-                                  f"{dt:.1f} s on one thread of {os.cpu_count()} host cores"}
+        dt, samples, _, _, te = run_oracle_pass(ws, As.numpy(), bs.numpy())
+        cpu_baseline = {"value": samples / te, "unit": unit, "cores": 1, "kind": "oracle",
+                        "whole_path_samples_per_s": samples / dt,
+                        "sample": f"first {rows} of {w.m} rows of {args.workload}, all {w.epochs} epochs ({te:.1f} s in the SGD "
+                                  f"epochs, {dt:.1f} s for the whole path) on one thread of {os.cpu_count()} host cores"}
 
     if rank == 0:
         print(json.dumps({
@@ -363,7 +398,8 @@ def main():
                        "multi_gpu": "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline, "final_loss": final_loss,
-            "packed_gb_per_s_per_epoch": achieved, "stages": stages, "other_workloads": others,
+            "packed_gb_per_s_per_epoch": achieved, "whole_path_samples_per_s": whole_value,
+            "stages": stages, "other_workloads": others,
         }))
     if world > 1:
         dist.destroy_process_group()
