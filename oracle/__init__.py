@@ -46,6 +46,10 @@ def _declare(L):
     L.orc_pack_codes.restype = None
     L.orc_unpack_codes.argtypes = [vp, i64, i32, vp]
     L.orc_unpack_codes.restype = None
+    L.orc_up_row_bytes.argtypes = [i64]
+    L.orc_up_row_bytes.restype = i64
+    L.orc_shared_base_encode.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, i64]
+    L.orc_shared_base_decode.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp]
     L.orc_column_range.argtypes = [vp, i64, i64, i64, vp, vp]
     L.orc_quantize.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
     L.orc_dequantize_row.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
@@ -124,6 +128,30 @@ def unpack_codes(row, n, bits):
 def unpack_plane(plane, n, bits):
     """(m, row_bytes) uint8 -> (m, n) uint8 codes."""
     return np.stack([unpack_codes(plane[k], n, bits) for k in range(plane.shape[0])])
+
+
+def up_row_bytes(n):
+    return int(lib().orc_up_row_bytes(n))
+
+
+def shared_base_encode(ds):
+    """(base, up1, up2) of a two-plane dataset: the smaller code once, one bit per sample."""
+    urb = up_row_bytes(ds.n)
+    base = np.zeros_like(ds.plane1)
+    up1 = np.zeros((ds.m, urb), np.uint8)
+    up2 = np.zeros((ds.m, urb), np.uint8)
+    _check(lib().orc_shared_base_encode(_p(ds.plane1), _p(ds.plane2), ds.row_bytes, ds.m, ds.n, ds.bits, _p(base),
+                                        _p(up1), _p(up2), urb))
+    return base, up1, up2
+
+
+def shared_base_decode(base, up1, up2, n, bits):
+    base, up1, up2 = (np.ascontiguousarray(a, dtype=np.uint8) for a in (base, up1, up2))
+    m, rb = base.shape
+    p1 = np.zeros_like(base)
+    p2 = np.zeros_like(base)
+    _check(lib().orc_shared_base_decode(_p(base), _p(up1), _p(up2), rb, up1.shape[1], m, n, bits, _p(p1), _p(p2)))
+    return p1, p2
 
 
 def column_range(A):

@@ -17,7 +17,9 @@
 //     update in full precision);
 //   * variance-optimal levels: Section 3 (problem statement, Lemma on endpoints, the recursion
 //     T(k, m) = min_j T(k-1, j) + V(j, m), "Dynamic Programming with Candidate Points");
-//   * objective: Eq. (leastsquares) with l = a^T x - b, i.e. 1/(2K) sum (a_k^T x - b_k)^2.
+//   * objective: Eq. (leastsquares) with l = a^T x - b, i.e. 1/(2K) sum (a_k^T x - b_k)^2;
+//   * shared-base storage of the two samples (base code + one bit per sample): Section 2.2,
+//     "Overhead of Storing Samples".
 //
 // Readings taken where the paper is silent (all listed in the design notes):
 //   samples use L = 2^bits unsigned levels on the per-feature range [lo_j, hi_j] (s = L-1
@@ -31,7 +33,8 @@
 // variance over 10^6 draws; the l2-scaled variance bound; naive-estimator bias in closed form;
 // zero bias of the double-sampled forms; pack/unpack round trip; on-grid data reduces the
 // minibatch gradient to the textbook least-squares gradient; DP against brute force over all level
-// subsets; convergence to the normal-equation solution; frozen-code fixed point in closed form.
+// subsets; convergence to the normal-equation solution; frozen-code fixed point in closed form;
+// shared-base encoding: a hand-written example, exhaustive code pairs, round trip on quantized data.
 // Parity partly unpinned by nature: Q3/Q4 trajectories (a sub-ulp difference may flip a stochastic
 // rounding); see the design notes.
 
@@ -126,6 +129,60 @@ void orc_pack_codes(const uint8_t* codes, int64_t n, int bits, uint8_t* row_out,
 void orc_unpack_codes(const uint8_t* row, int64_t n, int bits, uint8_t* codes_out) {
     const int cb = orc_container_bits(bits);
     for (int64_t j = 0; j < n; ++j) codes_out[j] = (uint8_t)get_code(row, j, cb);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Shared-base storage of the two samples (Section 2.2, "Overhead of Storing Samples"): the two
+// quantizations of a value land on the same interval of levels, so they can only be its lower or
+// its upper end.  It is enough to store the smaller of the two codes once (the base, `bits` wide)
+// and one bit per sample saying whether that sample lies one level higher: bits + 2 instead of
+// 2 * bits per value.  Layout: the base plane is an ordinary plane (container width cb); an "up"
+// plane holds one bit per feature, feature j at bit j of its row, low bits first, row stride
+// orc_up_row_bytes(n) = ceil(n / 8) rounded up to 16.  Decoding gives back exactly the two codes.
+// Returns ORC_ERR_INVALID_ARG if the two codes of a value differ by more than one level (then they
+// are not two samples of one value).
+// ---------------------------------------------------------------------------------------------
+int64_t orc_up_row_bytes(int64_t n) {
+    if (n <= 0) return 0;
+    return ((n + 7) / 8 + 15) / 16 * 16;
+}
+
+int orc_shared_base_encode(const uint8_t* plane1, const uint8_t* plane2, int64_t row_bytes, int64_t m, int64_t n, int bits,
+                           uint8_t* base, uint8_t* up1, uint8_t* up2, int64_t up_row_bytes) {
+    const int cb = orc_container_bits(bits);
+    if (cb == 0) return ORC_ERR_UNSUPPORTED;
+    if (!plane1 || !plane2 || !base || !up1 || !up2 || m <= 0 || n <= 0) return ORC_ERR_INVALID_ARG;
+    if (row_bytes < orc_row_bytes(n, bits) || up_row_bytes < orc_up_row_bytes(n)) return ORC_ERR_INVALID_ARG;
+    std::memset(base, 0, (size_t)(m * row_bytes));
+    std::memset(up1, 0, (size_t)(m * up_row_bytes));
+    std::memset(up2, 0, (size_t)(m * up_row_bytes));
+    for (int64_t k = 0; k < m; ++k)
+        for (int64_t j = 0; j < n; ++j) {
+            const uint32_t c1 = get_code(plane1 + k * row_bytes, j, cb), c2 = get_code(plane2 + k * row_bytes, j, cb);
+            const uint32_t lower = c1 < c2 ? c1 : c2;
+            if (c1 - lower > 1u || c2 - lower > 1u) return ORC_ERR_INVALID_ARG;
+            put_code(base + k * row_bytes, j, cb, lower);
+            put_code(up1 + k * up_row_bytes, j, 1, c1 - lower);
+            put_code(up2 + k * up_row_bytes, j, 1, c2 - lower);
+        }
+    return ORC_OK;
+}
+
+int orc_shared_base_decode(const uint8_t* base, const uint8_t* up1, const uint8_t* up2, int64_t row_bytes,
+                           int64_t up_row_bytes, int64_t m, int64_t n, int bits, uint8_t* plane1, uint8_t* plane2) {
+    const int cb = orc_container_bits(bits);
+    if (cb == 0) return ORC_ERR_UNSUPPORTED;
+    if (!plane1 || !plane2 || !base || !up1 || !up2 || m <= 0 || n <= 0) return ORC_ERR_INVALID_ARG;
+    if (row_bytes < orc_row_bytes(n, bits) || up_row_bytes < orc_up_row_bytes(n)) return ORC_ERR_INVALID_ARG;
+    std::memset(plane1, 0, (size_t)(m * row_bytes));
+    std::memset(plane2, 0, (size_t)(m * row_bytes));
+    for (int64_t k = 0; k < m; ++k)
+        for (int64_t j = 0; j < n; ++j) {
+            const uint32_t lower = get_code(base + k * row_bytes, j, cb);
+            put_code(plane1 + k * row_bytes, j, cb, lower + get_code(up1 + k * up_row_bytes, j, 1));
+            put_code(plane2 + k * row_bytes, j, cb, lower + get_code(up2 + k * up_row_bytes, j, 1));
+        }
+    return ORC_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
