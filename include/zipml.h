@@ -115,6 +115,27 @@ typedef struct zipml_dataset {
     const float* levels;    /* n * 2^bits ascending; TABLE                                           */
 } zipml_dataset;
 
+/* The same double-sampled data in the shared-base storage of the paper's Section 2.2 ("Overhead of Storing
+ * Samples"): the two quantizations of a value are the lower or the upper end of one interval of levels, so the
+ * smaller code is stored once and each sample keeps one bit saying whether it lies one level higher --
+ * bits + 2 instead of 2 * bits per value (container widths: 4 / 6 / 6 / 10 instead of 4 / 8 / 8 / 16).
+ *   base      an ordinary plane (layout ZIPML_LAYOUT_ROWS, stride row_bytes) of the smaller codes
+ *   up1, up2  one bit per feature: feature j at bit j of its row, low bits first, stride up_row_bytes
+ *             (a multiple of 16, >= zipml_up_row_bytes(n)); code of sample c = base + up_c
+ * Uniform grids only (value = lo_j + code * step_j). */
+typedef struct zipml_shared_base {
+    uint32_t struct_size;   /* sizeof(zipml_shared_base)                                             */
+    int32_t bits;           /* 2, 3, 4 or 8                                                          */
+    int64_t m, n;
+    int64_t row_bytes;      /* stride of the base plane                                              */
+    int64_t up_row_bytes;   /* stride of the two up planes                                           */
+    const uint8_t* base;    /* m * row_bytes bytes, 16-byte aligned                                  */
+    const uint8_t* up1;     /* m * up_row_bytes bytes, 16-byte aligned                               */
+    const uint8_t* up2;
+    const float* feat_lo;   /* n (not needed by the conversions)                                     */
+    const float* feat_step; /* n                                                                     */
+} zipml_shared_base;
+
 /* Parameters of one zipml_sgd_epoch call. */
 typedef struct zipml_sgd_params {
     uint32_t struct_size;       /* sizeof(zipml_sgd_params)                                          */
@@ -252,6 +273,25 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
  * Out: loss_out, one double in device memory.  Deterministic for a given device and shape. */
 int zipml_loss(zipml_ctx* ctx, int32_t mode, const float* A, int64_t m, int64_t n, int64_t lda,
                const zipml_dataset* data, const float* b, const float* x, double* loss_out);
+
+/* Shared-base storage (paper Section 2.2, "Overhead of Storing Samples"; see zipml_shared_base).
+ * zipml_up_row_bytes: smallest legal stride of an up plane, ceil(n / 8) rounded up to 16.
+ * zipml_shared_base_encode: the two planes of `data` (ZIPML_LAYOUT_ROWS) -> out->base, out->up1, out->up2 (the
+ *   caller's buffers behind the const pointers of `out`, fully written; bits, m, n, row_bytes as in `data`).
+ *   A value whose two codes lie more than one level apart makes the next zipml_sync() return
+ *   ZIPML_ERR_INVALID_ARG (such planes are not two samples of the same values).
+ * zipml_shared_base_decode: back to two planes of stride data->row_bytes, bit for bit.
+ * zipml_loss_shared_base: the estimate of zipml_loss(ZIPML_LOSS_CODES) computed from the three planes as they lie,
+ *   Q_c(a)^T x = lo^T x + base^T w + up_c^T w with w = step * x (fp32 products in short runs, combined in double).
+ * zipml_sgd_epoch_shared_base: zipml_sgd_epoch on such data.  The epoch engines read two planes: they are rebuilt in
+ *   the context's staging buffer first (shared with zipml_train_host, kept until the next such call), so the saving
+ *   is in what is stored, not in what an epoch reads. */
+int64_t zipml_up_row_bytes(int64_t n);
+int zipml_shared_base_encode(zipml_ctx* ctx, const zipml_dataset* data, const zipml_shared_base* out);
+int zipml_shared_base_decode(zipml_ctx* ctx, const zipml_shared_base* data, uint8_t* plane1, uint8_t* plane2);
+int zipml_loss_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const float* b, const float* x, double* loss_out);
+int zipml_sgd_epoch_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const float* b, float* x,
+                                const zipml_sgd_params* params, float* grad_out);
 
 /* Whole path from HOST buffers, for callers that hold their data in host memory: copies A and b to
  * the device, quantizes (UNIFORM, or TABLE with levels from zipml_optimal_levels when

@@ -18,7 +18,8 @@ REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM, ENGINE_COLUMN = 0, 1, 2, 3, 4, 5, 6, 7
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
-EXPORTS = ["zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+EXPORTS = ["zipml_up_row_bytes", "zipml_shared_base_encode", "zipml_shared_base_decode", "zipml_loss_shared_base",
+           "zipml_sgd_epoch_shared_base", "zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -38,6 +39,12 @@ class CDataset(C.Structure):
                 ("m", C.c_int64), ("n", C.c_int64), ("row_bytes", C.c_int64),
                 ("plane1", C.c_void_p), ("plane2", C.c_void_p),
                 ("feat_lo", C.c_void_p), ("feat_step", C.c_void_p), ("levels", C.c_void_p)]
+
+
+class CSharedBase(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("bits", C.c_int32), ("m", C.c_int64), ("n", C.c_int64),
+                ("row_bytes", C.c_int64), ("up_row_bytes", C.c_int64), ("base", C.c_void_p), ("up1", C.c_void_p),
+                ("up2", C.c_void_p), ("feat_lo", C.c_void_p), ("feat_step", C.c_void_p)]
 
 
 class CSgdParams(C.Structure):
@@ -77,6 +84,12 @@ def lib():
         L.zipml_column_blocks_bytes.argtypes = [i64, i64]
         L.zipml_column_blocks_bytes.restype = i64
         L.zipml_convert_layout.argtypes = [vp, C.POINTER(CDataset), i32, vp, vp]
+        L.zipml_up_row_bytes.argtypes = [i64]
+        L.zipml_up_row_bytes.restype = i64
+        L.zipml_shared_base_encode.argtypes = [vp, C.POINTER(CDataset), C.POINTER(CSharedBase)]
+        L.zipml_shared_base_decode.argtypes = [vp, C.POINTER(CSharedBase), vp, vp]
+        L.zipml_loss_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, vp]
+        L.zipml_sgd_epoch_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, C.POINTER(CSgdParams), vp]
         L.zipml_quantize.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
         L.zipml_optimal_levels.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp]
         L.zipml_sgd_epoch.argtypes = [vp, C.POINTER(CDataset), vp, vp, C.POINTER(CSgdParams), vp]
@@ -129,6 +142,29 @@ class Dataset:
     def packed_bytes(self):
         """Bytes one epoch has to read: both planes and the labels."""
         return 2 * self.m * self.row_bytes + 4 * self.m
+
+
+class SharedBase:
+    """Base plane plus two one-bit planes (see zipml_shared_base), all torch tensors on the context's device."""
+
+    def __init__(self, base, up1, up2, m, n, bits, feat_lo, feat_step):
+        self.base, self.up1, self.up2, self.m, self.n, self.bits = base, up1, up2, m, n, bits
+        self.row_bytes, self.up_row_bytes = base.shape[1], up1.shape[1]
+        self.feat_lo, self.feat_step = feat_lo, feat_step
+
+    def c_struct(self):
+        d = CSharedBase()
+        d.struct_size = C.sizeof(CSharedBase)
+        d.bits, d.m, d.n, d.row_bytes, d.up_row_bytes = self.bits, self.m, self.n, self.row_bytes, self.up_row_bytes
+        d.base, d.up1, d.up2 = self.base.data_ptr(), self.up1.data_ptr(), self.up2.data_ptr()
+        d.feat_lo = self.feat_lo.data_ptr() if self.feat_lo is not None else None
+        d.feat_step = self.feat_step.data_ptr() if self.feat_step is not None else None
+        return d
+
+    @property
+    def packed_bytes(self):
+        """Bytes of the three planes and the labels."""
+        return self.m * (self.row_bytes + 2 * self.up_row_bytes) + 4 * self.m
 
 
 class Context:
@@ -214,6 +250,38 @@ class Context:
         _check(lib().zipml_convert_layout(self._h, C.byref(d), to_layout, _ptr(p1), _ptr(p2)), "zipml_convert_layout")
         return Dataset(p1, p2, data.m, data.n, data.bits, data.level_mode, data.feat_lo, data.feat_step, data.levels,
                        layout=to_layout, row_bytes=data.row_bytes)
+
+    def zipml_shared_base_encode(self, data):
+        urb = int(lib().zipml_up_row_bytes(data.n))
+        base = torch.empty((data.m, data.row_bytes), dtype=torch.uint8, device=self.device)
+        up1 = torch.empty((data.m, urb), dtype=torch.uint8, device=self.device)
+        up2 = torch.empty((data.m, urb), dtype=torch.uint8, device=self.device)
+        sb = SharedBase(base, up1, up2, data.m, data.n, data.bits, data.feat_lo, data.feat_step)
+        d, o = data.c_struct(), sb.c_struct()
+        _check(lib().zipml_shared_base_encode(self._h, C.byref(d), C.byref(o)), "zipml_shared_base_encode")
+        return sb
+
+    def zipml_shared_base_decode(self, sb):
+        p1 = torch.empty((sb.m, sb.row_bytes), dtype=torch.uint8, device=self.device)
+        p2 = torch.empty((sb.m, sb.row_bytes), dtype=torch.uint8, device=self.device)
+        d = sb.c_struct()
+        _check(lib().zipml_shared_base_decode(self._h, C.byref(d), _ptr(p1), _ptr(p2)), "zipml_shared_base_decode")
+        return Dataset(p1, p2, sb.m, sb.n, sb.bits, LEVELS_UNIFORM, sb.feat_lo, sb.feat_step, None)
+
+    def zipml_loss_shared_base(self, sb, b, x, out=None):
+        out = torch.empty(1, dtype=torch.float64, device=self.device) if out is None else out
+        d = sb.c_struct()
+        _check(lib().zipml_loss_shared_base(self._h, C.byref(d), _ptr(b, torch.float32, self.device),
+                                            _ptr(x, torch.float32, self.device), _ptr(out)), "zipml_loss_shared_base")
+        return out
+
+    def zipml_sgd_epoch_shared_base(self, sb, b, x, batch, lr, grad_out=None, **kw):
+        p, keep = self.sgd_params(batch, lr, **kw)
+        d = sb.c_struct()
+        _check(lib().zipml_sgd_epoch_shared_base(self._h, C.byref(d), _ptr(b, torch.float32, self.device),
+                                                 _ptr(x, torch.float32, self.device), C.byref(p),
+                                                 _ptr(grad_out, torch.float32, self.device)), "zipml_sgd_epoch_shared_base")
+        del keep
 
     def zipml_optimal_levels(self, A, bits, hist_bins=1024, want_objective=False):
         m, n = A.shape

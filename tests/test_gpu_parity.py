@@ -696,6 +696,58 @@ def test_loss_codes_with_a_stride_far_above_the_minimum(ctx):
 
 
 # ---------------------------------------------------------------------------------------------
+# shared-base storage of the two samples (Section 2.2, "Overhead of Storing Samples")
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("key,m,n,bits", [("c1", 300, 64, 4), ("c2", 129, 1003, 8), ("c3", 77, 2050, 2), ("c4u", 100, 37, 3),
+                                          ("c5", 40, 4100, 4), ("c1", 1, 5, 8)])
+def test_shared_base_planes_bit_exact(ctx, key, m, n, bits):
+    _, A, b, xs = workload(key, m, n, seed=bits)
+    ods = oracle.quantize(A, bits, seed=21)
+    base, up1, up2 = oracle.shared_base_encode(ods)
+    gds = dev_dataset(ods, ctx)
+    sb = ctx.zipml_shared_base_encode(gds)
+    ctx.zipml_sync()
+    assert (sb.base.cpu().numpy() == base).all() and (sb.up1.cpu().numpy() == up1).all() and (sb.up2.cpu().numpy() == up2).all()
+    back = ctx.zipml_shared_base_decode(sb)
+    ctx.zipml_sync()
+    assert (back.plane1.cpu().numpy() == ods.plane1).all() and (back.plane2.cpu().numpy() == ods.plane2).all()
+    if bits > 2 and n > 256:                          # 6 instead of 8, 10 instead of 16 bits per value (2-bit codes gain nothing)
+        assert sb.packed_bytes < gds.packed_bytes
+    # the loss straight from the three planes is the oracle's estimate from the two
+    x = (xs * 0.9).astype(np.float32)
+    want = oracle.loss_codes(ods, b, x)
+    got = ctx.zipml_loss_shared_base(sb, to_dev(b, ctx), to_dev(x, ctx))
+    ctx.zipml_sync()
+    assert abs(got.item() - want) <= LOSS_TOL * max(abs(want), oracle.loss_dense(A, b, x))
+
+
+def test_shared_base_epoch_and_refusals(ctx):
+    """An epoch from shared-base data gives the model of the two-plane data, bit for bit (the same planes reach the
+    same engine); planes that are not two samples of one value are refused."""
+    _, A, b, _ = workload("c2", 2100, 1000, seed=1)
+    ods = oracle.quantize(A, 8, seed=7)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    sb = ctx.zipml_shared_base_encode(gds)
+    x0 = (np.random.default_rng(1).standard_normal(1000) * 0.1).astype(np.float32)
+    x_ref, g_ref = oracle.sgd_epoch(ods, b, x0, 256, 1e-3, want_grad=True)
+    x1, x2 = to_dev(x0, ctx), to_dev(x0, ctx)
+    g = torch.zeros((2, 1000), dtype=torch.float32, device=ctx.device)
+    ctx.zipml_sgd_epoch_shared_base(sb, db, x1, 256, 1e-3, grad_out=g)
+    ctx.zipml_sgd_epoch(gds, db, x2, 256, 1e-3)
+    ctx.zipml_sync()
+    assert rel(x1.cpu().numpy(), x_ref) <= MODEL_TOL and (x1 == x2).all()
+    assert rel(g[0].cpu().numpy(), g_ref[0]) <= 10 * GRAD_TOL           # (the epoch's last step, from the kernel's own model)
+    far = torch.zeros_like(gds.plane1)
+    far[:, 0] = 2                                                        # plane 1 says code 2 where plane 2 says 0
+    bad = binding.Dataset(far, torch.zeros_like(far), gds.m, gds.n, 8, binding.LEVELS_UNIFORM, gds.feat_lo, gds.feat_step, None)
+    ctx.zipml_shared_base_encode(bad)
+    with pytest.raises(binding.ZipmlError) as e:
+        ctx.zipml_sync()
+    assert e.value.code == binding.ERR_INVALID_ARG
+    ctx.zipml_sync()
+
+
+# ---------------------------------------------------------------------------------------------
 # the configurations at their own step shapes (a few minibatches of rows)
 # ---------------------------------------------------------------------------------------------
 def test_config5_step_shape(ctx):
