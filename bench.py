@@ -305,6 +305,12 @@ def main():
     stages = {"quantize" + ("+levels" if w.levels == "optimal" else ""):
               stage(quant_events, a_bytes * (2 if w.levels != "optimal" else 4) + 2 * ds.m * ds.row_bytes),
               "loss_dense": stage(loss_events, a_bytes + 4 * w.m)}
+    # the loss estimate straight from the two code planes (outside the timed region: the pass above ends in the dense loss)
+    lc_events, lc_dev = [], torch.zeros(1, dtype=torch.float64, device=dev)
+    for i in range(4):
+        timed(lc_events, i > 0, lambda: ctx.zipml_loss(binding.LOSS_CODES, b, x, data=ds, out=lc_dev))
+    ctx.zipml_sync()
+    stages["loss_codes"] = stage(lc_events, packed_bytes + 4 * w.m)
 
     # ------------------------------------------------------------------ end to end from host buffers
     e2e = None

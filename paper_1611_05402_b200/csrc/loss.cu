@@ -91,6 +91,110 @@ __global__ void __launch_bounds__(256) loss_codes_kernel(const uint32_t* __restr
 }
 
 // ---------------------------------------------------------------------------------------------
+// Level tables whose level * x table fits shared memory.  Every block stages a table of GROUP sums: GB bits of a
+// code word (GB / CB neighbouring codes) index one entry that already holds the sum of their level * x products, so a
+// word costs 32 / GB look-ups instead of 32 / CB.  Entry (group value v, group p of a word, word q of the row) sits at
+// (v * NP + p) * wpad + q with wpad a multiple of 32: the lanes of a warp -- consecutive words q, whatever their codes --
+// read 32 different banks.  EB is the number of index bits kept of a group (7 for byte groups of 3-bit codes in 4-bit
+// fields, whose bit 7 is always clear; else GB).  A warp takes four rows at a time (their loads are in flight
+// together) and folds the eight row sums with a halving butterfly.  From global memory every look-up of a warp
+// touched up to 32 cache lines (426 GB/s of packed codes on 500,000 x 512 3-bit rows).
+// ---------------------------------------------------------------------------------------------
+constexpr int kTableRows = 4;                             // rows per warp and pass
+
+template <int CB, int GB, int EB>
+__global__ void __launch_bounds__(1024) loss_codes_table_kernel(const uint32_t* __restrict__ p1, const uint32_t* __restrict__ p2,
+                                                                int64_t row_words, int64_t m, int64_t n, int L, int wpad,
+                                                                const float* __restrict__ levels, const float* __restrict__ x,
+                                                                const float* __restrict__ b, double* __restrict__ partials) {
+    constexpr int FPW = 32 / CB, NP = 32 / GB, CPG = GB / CB, E = 1 << EB;
+    extern __shared__ float tab[];                        // [E][NP][wpad], then the single products [L][n + n / 32 + 1]
+    __shared__ double red[40];
+    const int words = (int)((n + FPW - 1) / FPW);
+    // the products level * x of single codes first (levels read in their own order), feature j of code c at
+    // c * npad + j + j / 32: the group sums below read features NP * CPG apart, which that skew spreads over the banks
+    float* single = tab + (size_t)E * NP * wpad;
+    const int npad = (int)(n + n / 32 + 1);
+    for (int64_t idx = threadIdx.x; idx < n * L; idx += blockDim.x) {
+        const int j = (int)(idx / L), c = (int)(idx % L);
+        single[c * npad + j + (j >> 5)] = __ldg(levels + idx) * __ldg(x + j);
+    }
+    __syncthreads();
+    for (int vp = threadIdx.x / wpad; vp < E * NP; vp += blockDim.x / wpad) {   // (wpad divides the block size or exceeds it: see the host)
+        const int p = vp % NP, v = vp / NP;
+        for (int q = threadIdx.x % wpad; q < wpad; q += blockDim.x) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int s = 0; s < CPG; ++s) {
+                const int c = (v >> (CB * s)) & ((1 << CB) - 1);
+                const int64_t j = ((int64_t)q * NP + p) * CPG + s;
+                if (c < L && q < words && j < n) sum += single[c * npad + (int)j + (int)(j >> 5)];
+            }
+            tab[(size_t)vp * wpad + q] = sum;
+        }
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int stride = NP * wpad;
+    double total = 0.0;
+    for (int64_t k0 = warp_global * kTableRows; k0 < m; k0 += nwarps * kTableRows) {
+        const uint32_t* row1 = p1 + k0 * row_words;
+        const uint32_t* row2 = p2 + k0 * row_words;
+        const int nr = m - k0 < kTableRows ? (int)(m - k0) : kTableRows;   // rows past the end read as zero words
+        double d[2 * kTableRows];
+#pragma unroll
+        for (int i = 0; i < 2 * kTableRows; ++i) d[i] = 0.0;
+        for (int qb = 0; qb < words; qb += 256) {         // fp32 sums of at most 8 words' look-ups, then double
+            float acc[2 * kTableRows];
+#pragma unroll
+            for (int i = 0; i < 2 * kTableRows; ++i) acc[i] = 0.0f;
+            const int qe = words < qb + 256 ? words : qb + 256;
+            for (int q = qb + lane; q < qe; q += 32) {
+                uint32_t u[2 * kTableRows];
+#pragma unroll
+                for (int i = 0; i < 2 * kTableRows; ++i)
+                    u[i] = (i >> 1) < nr ? __ldcs(((i & 1) ? row2 : row1) + (i >> 1) * row_words + q) : 0u;
+                const float* tq = tab + q;
+#pragma unroll
+                for (int i = 0; i < 2 * kTableRows; ++i)
+#pragma unroll
+                    for (int p = 0; p < NP; ++p) acc[i] += tq[(int)((u[i] >> (GB * p)) & (uint32_t)(E - 1)) * stride + p * wpad];
+            }
+#pragma unroll
+            for (int i = 0; i < 2 * kTableRows; ++i) d[i] += (double)acc[i];
+        }
+        // d[2 r + plane]: lanes 16.. keep rows 2, 3, then lanes with bit 3 keep the odd row; both planes of that row go on
+        static_assert(kTableRows == 4, "the butterfly below folds four rows");
+        const bool hi16 = lane & 16, hi8 = lane & 8;
+        double w[4], z[2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const double keep = hi16 ? d[j + 4] : d[j], send = hi16 ? d[j] : d[j + 4];
+            w[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const double keep = hi8 ? w[j + 2] : w[j], send = hi8 ? w[j] : w[j + 2];
+            z[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+            z[0] += __shfl_xor_sync(0xffffffffu, z[0], o);
+            z[1] += __shfl_xor_sync(0xffffffffu, z[1], o);
+        }
+        const int64_t k = k0 + (hi16 ? 2 : 0) + (hi8 ? 1 : 0);
+        if ((lane & 7) == 0 && k < m) {
+            const double bk = (double)__ldg(b + k);
+            total += (z[0] - bk) * (z[1] - bk);
+        }
+    }
+    total = block_sum(total, red);
+    if (threadIdx.x == 0) partials[blockIdx.x] = total;
+}
+
+// ---------------------------------------------------------------------------------------------
 // The same estimate for uniform grids on the int8 tensor cores: a pure streaming pass (no step-to-step
 // dependency), so it shows what the unpack-and-dot arithmetic of the SGD step reaches against HBM.
 // w = step * x becomes four balanced base-128 int8 digits per entry (one rounding, 2^-27 of the
@@ -243,7 +347,46 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
         ctx->launches += 3;
         return cuda_status(cudaGetLastError());
     }
+    if (table) {
+        // group sums of the level * x table in shared memory: the widest group whose table fits (padding features of
+        // the last word read as zero there); none fits: the look-ups below go to global memory
+        const int fpw = 32 / cb;
+        const int64_t words = (d->n + fpw - 1) / fpw;
+        const int64_t wpad = (words + 31) / 32 * 32;
+        const int64_t room = (int64_t)ctx->smem_optin - 1024;
+        const uint32_t* q1 = reinterpret_cast<const uint32_t*>(d->plane1);
+        const uint32_t* q2 = reinterpret_cast<const uint32_t*>(d->plane2);
+        for (int gb = 8; gb >= cb; gb >>= 1) {
+            const int eb = (gb == 8 && cb == 4 && L <= 8) ? 7 : gb;
+            const int64_t smem = (int64_t)sizeof(float) * (((int64_t)1 << eb) * (32 / gb) * wpad + (int64_t)L * (d->n + d->n / 32 + 1));
+            if (smem > room) continue;
+            // one block of 1024 threads per SM, or several of 512 where the table is small
+            int per_sm = (int)((int64_t)ctx->smem_optin / (smem + 2048));
+            per_sm = per_sm < 1 ? 1 : per_sm > 4 ? 4 : per_sm;
+            int threads = per_sm == 1 ? 1024 : 512;
+            while (wpad < threads && threads % wpad != 0) threads -= 32;   // the staging loop wants wpad | threads (or wpad >= threads)
+            int blocks = ctx->sm_count * per_sm;
+            if (blocks > max_partials) blocks = max_partials;
+            const int64_t need = (d->m + 4 * (threads / 32) - 1) / (4 * (threads / 32));
+            if (blocks > need) blocks = (int)need;
+#define ZIPML_LAUNCH_LT(CB_, GB_, EB_)                                                                                     \
+    do {                                                                                                                   \
+        cudaError_t e_ = cudaFuncSetAttribute(loss_codes_table_kernel<CB_, GB_, EB_>,                                      \
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                     \
+        if (e_ != cudaSuccess) return cuda_status(e_);                                                                     \
+        loss_codes_table_kernel<CB_, GB_, EB_><<<blocks, threads, (size_t)smem, ctx->stream>>>(                            \
+            q1, q2, d->row_bytes / 4, d->m, d->n, L, (int)wpad, d->levels, x, b, partials);                                       \
+    } while (0)
+            if (cb == 2) { if (gb == 8) ZIPML_LAUNCH_LT(2, 8, 8); else if (gb == 4) ZIPML_LAUNCH_LT(2, 4, 4); else ZIPML_LAUNCH_LT(2, 2, 2); }
+            else { if (gb == 8 && eb == 7) ZIPML_LAUNCH_LT(4, 8, 7); else if (gb == 8) ZIPML_LAUNCH_LT(4, 8, 8); else ZIPML_LAUNCH_LT(4, 4, 4); }
+#undef ZIPML_LAUNCH_LT
+            loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)d->m), loss_out);
+            ctx->launches += 2;
+            return cuda_status(cudaGetLastError());
+        }
+    }
     loss_prepare_kernel<<<1, 1024, 0, ctx->stream>>>(d->feat_lo, d->feat_step, d->levels, x, d->n, L, table, wtab, base);
+    ++ctx->launches;
     int blocks = ctx->sm_count * 8;
     if (blocks > max_partials) blocks = max_partials;
     const int64_t need = (d->m + 7) / 8;
@@ -258,7 +401,7 @@ int launch_loss_codes(zipml_ctx* ctx, const zipml_dataset* d, const float* b, co
     else { ZIPML_LAUNCH_L(8, false); }
 #undef ZIPML_LAUNCH_L
     loss_finish_kernel<<<1, 256, 0, ctx->stream>>>(partials, blocks, 1.0 / (2.0 * (double)d->m), loss_out);
-    ctx->launches += 3;
+    ctx->launches += 2;
     return cuda_status(cudaGetLastError());
 }
 
