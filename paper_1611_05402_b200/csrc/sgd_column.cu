@@ -66,7 +66,8 @@ namespace zipml {
 
 constexpr int kColAWarps = 8, kColBWarps = 8, kColRWarps = 4, kColRShift = 2;     // (kColRWarps = 2^kColRShift)
 constexpr int kColWarpA0 = 1, kColWarpB0 = kColWarpA0 + kColAWarps, kColWarpR0 = kColWarpB0 + kColBWarps;
-constexpr int kColThreads = 32 * (kColWarpR0 + kColRWarps);
+constexpr int kColWarpS2 = kColWarpR0 + kColRWarps;             // the second service warp (second visits)
+constexpr int kColThreads = 32 * (kColWarpS2 + 1);
 constexpr int kColRThreads = 32 * kColRWarps;
 constexpr int kColBThreads = 32 * kColBWarps;
 constexpr int kColBlockBytes = 128;         // bytes of a packed row that a CTA owns
@@ -123,6 +124,7 @@ struct ColShared {
     float red_f[2][32];
     long long red_l[2][kColRWarps];
     int abort_flag;
+    int qa_issued;                             // chunks whose first copy has been issued
 };
 
 __device__ __forceinline__ bool col_aborted(const ColShared* sh) { return *reinterpret_cast<const volatile int*>(&sh->abort_flag) != 0; }
@@ -301,6 +303,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
         }
         sh->w_version = 0;
         sh->abort_flag = 0;
+        sh->qa_issued = 0;
         mbar_fence_init();
     }
     // ---- every CTA scans the model once, with the same arithmetic: the bound of the dots and its growth rate
@@ -324,66 +327,64 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     if (tid == 0) col_unit_of(dbound, sh->sp[0].U, sh->sp[0].invU);
     __syncthreads();                                      // barriers initialised, sums read, U(0) in place
 
-    // =================================================================================== service warp
-    if (warp == 0) {
+    // =================================================================================== service warps
+    // One lane each.  Warp 0, first visits: the next chunk as soon as a slot of the A ring is free.  The last warp, second
+    // visits: the next chunk that has had its first copy issued (it is in L2 or on its way there), as soon as a slot of
+    // the B ring is free.  Each sleeps on its ring's barrier and is woken by the release itself: a shared loop that
+    // looked at both rings in turn, with pauses, let a freed slot wait several hundred cycles for its next copy.
+    if (warp == 0 || warp == kColWarpS2) {
         if (lane == 0) {
-            // first visits: the next chunk as soon as a slot of the A ring is free; second visits: the next chunk that
-            // has had its first copy issued (it is in L2 or on its way there), as soon as a slot of the B ring is free
-            int qA = 0, tA = 0, cA = 0, qB = 0, tB = 0, cB = 0;
-            ColRing ra{0, 0u}, rb{0, 0u};
-            ColStep sA = col_step(a, a.first_step), sB = sA;
+            const bool first_visit = warp == 0;
+            unsigned long long* full = first_visit ? sh->full_a : sh->full_b;
+            unsigned long long* empty = first_visit ? sh->empty_a : sh->empty_b;
+            unsigned char* base = first_visit ? tiles : tiles_b;
+            const int nslots = first_visit ? a.slots_a : a.slots_b;
+            int q = 0, t = 0, c = 0;
+            ColRing ring{0, 0u};
+            ColStep st = col_step(a, a.first_step);
             uint64_t evict_first;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
-            long long idle0 = clock64();
-            int idle = 0;
             bool ok = true;
 #pragma unroll 1
-            while (ok && tB < steps) {
-                bool progress = false;
-                if (tA < steps && (qA < a.slots_a || mbar_test_wait(sh->empty_a + ra.slot, ra.phase ^ 1u))) {
-                    unsigned char* dst = tiles + (size_t)ra.slot * slot_bytes;
-                    mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(sh->full_a + ra.slot), slot_bytes);
-                    const int y = (int)(y_own + sA.row0 + (int64_t)cA * R);
-                    tensor_load_2d(dst, &tm1, x_own, y, sh->full_a + ra.slot);
-                    tensor_load_2d(dst + plane_bytes, &tm2, x_own, y, sh->full_a + ra.slot);
-                    ++qA;
-                    ra.next(a.slots_a);
-                    if (++cA == sA.nch) { cA = 0; if (++tA < steps) sA = col_step(a, a.first_step + tA); }
-                    progress = true;
-                }
-                if (qB < qA && (qB < a.slots_b || mbar_test_wait(sh->empty_b + rb.slot, rb.phase ^ 1u))) {
-                    unsigned char* dst = tiles_b + (size_t)rb.slot * slot_bytes;
-                    mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(sh->full_b + rb.slot), slot_bytes);
-                    const int y = (int)(y_own + sB.row0 + (int64_t)cB * R);
-                    // (nobody reads these lines again this epoch: they may leave L2 ahead of the rest)
-                    tensor_load_2d_hint(dst, &tm1, x_own, y, sh->full_b + rb.slot, evict_first);
-                    tensor_load_2d_hint(dst + plane_bytes, &tm2, x_own, y, sh->full_b + rb.slot, evict_first);
-                    ++qB;
-                    rb.next(a.slots_b);
-                    if (++cB == sB.nch) { cB = 0; if (++tB < steps) sB = col_step(a, a.first_step + tB); }
-                    progress = true;
-                }
-                if (progress) { idle0 = clock64(); idle = 0; }
-                else {
-                    __nanosleep(idle < 8 ? 100 : 300);
-                    if ((++idle & 15) == 15) {
-                        if (col_aborted(sh)) ok = false;
-                        else if (clock64() - idle0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 70); ok = false; }
+            while (ok && t < steps) {
+                if (q >= nslots) ok = col_wait(empty + ring.slot, ring.phase ^ 1u, sh, a.status, 70);
+                if (ok && !first_visit) {
+                    const long long t0 = clock64();
+#pragma unroll 1
+                    for (int spin = 0; *reinterpret_cast<volatile int*>(&sh->qa_issued) <= q; ++spin) {
+                        __nanosleep(50);
+                        if ((spin & 63) == 63 && (col_aborted(sh) || clock64() - t0 > kColWaitCycles)) {
+                            if (!col_aborted(sh)) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 78); }
+                            ok = false;
+                            break;
+                        }
                     }
                 }
+                if (!ok) break;
+                unsigned char* dst = base + (size_t)ring.slot * slot_bytes;
+                mbar_arrive_expect_tx(reinterpret_cast<uint64_t*>(full + ring.slot), slot_bytes);
+                const int y = (int)(y_own + st.row0 + (int64_t)c * R);
+                if (first_visit) {
+                    tensor_load_2d(dst, &tm1, x_own, y, full + ring.slot);
+                    tensor_load_2d(dst + plane_bytes, &tm2, x_own, y, full + ring.slot);
+                    *reinterpret_cast<volatile int*>(&sh->qa_issued) = q + 1;
+                } else {
+                    // (nobody reads these lines again this epoch: they may leave L2 ahead of the rest)
+                    tensor_load_2d_hint(dst, &tm1, x_own, y, full + ring.slot, evict_first);
+                    tensor_load_2d_hint(dst + plane_bytes, &tm2, x_own, y, full + ring.slot, evict_first);
+                }
+                ++q;
+                ring.next(nslots);
+                if (++c == st.nch) { c = 0; if (++t < steps) st = col_step(a, a.first_step + t); }
             }
             if (!ok) {
                 // leaving early: the copies in flight must land before the CTA's shared memory goes away
                 const long long t0 = clock64();
 #pragma unroll 1
                 for (int s = 0; s < kColMaxSlots; ++s) {
-                    if (s < a.slots_a && s < qA) {
-                        const uint32_t par = (uint32_t)((((qA - 1 - ((qA - 1 - s + a.slots_a) % a.slots_a)) / a.slots_a)) & 1);
-                        while (!mbar_test_wait(sh->full_a + s, par) && clock64() - t0 < kColWaitCycles) {}
-                    }
-                    if (s < a.slots_b && s < qB) {
-                        const uint32_t par = (uint32_t)((((qB - 1 - ((qB - 1 - s + a.slots_b) % a.slots_b)) / a.slots_b)) & 1);
-                        while (!mbar_test_wait(sh->full_b + s, par) && clock64() - t0 < kColWaitCycles) {}
+                    if (s < nslots && s < q) {
+                        const uint32_t par = (uint32_t)((((q - 1 - ((q - 1 - s + nslots) % nslots)) / nslots)) & 1);
+                        while (!mbar_test_wait(full + s, par) && clock64() - t0 < kColWaitCycles) {}
                     }
                 }
             }
@@ -434,8 +435,10 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 if (lane == 0 && c == 0 && j == 0) col_mark(a, t_rel, 0);
             }
             const long long w0c = (a.trace && aw == 0) ? clock64() : 0;
-            ok = __all_sync(0xffffffffu, col_wait(sh->full_a + ring.slot, ring.phase, sh, a.status, 72));
-            if (!ok) break;
+            if (!__all_sync(0xffffffffu, mbar_test_wait(sh->full_a + ring.slot, ring.phase))) {      // (usually there already)
+                ok = __all_sync(0xffffffffu, col_wait(sh->full_a + ring.slot, ring.phase, sh, a.status, 72));
+                if (!ok) break;
+            }
             if (a.trace && aw == 0 && lane == 0) col_tally(a, t_rel, 1, clock64() - w0c);
             const uint32_t tile = smem_u32(tiles) + (uint32_t)ring.slot * slot_bytes;
             const int k0 = c * R + j * 32;                                // first row of the task within the step
@@ -579,40 +582,55 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             for (int c = 0; c < st.nch; ++c, ++q) {
                 const int rbuf = q & (kColRWarps - 1);
                 const long long w0c = (a.trace && p == 0) ? clock64() : 0;
-                ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1), sh, a.status, 73);
-                const long long w1c = (a.trace && p == 0) ? clock64() : 0;
-                ok = ok && col_wait(sh->full_b + ring.slot, ring.phase, sh, a.status, 74);
+                long long w1c = w0c;
+                // both are usually there already: one look at each, side by side, before the waiting routine is called
+                const bool have_r = mbar_test_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1));
+                const bool have_c = mbar_test_wait(sh->full_b + ring.slot, ring.phase);
+                if (!__all_sync(0xffffffffu, ok && have_r && have_c)) {
+                    ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1), sh, a.status, 73);
+                    w1c = (a.trace && p == 0) ? clock64() : 0;
+                    ok = ok && col_wait(sh->full_b + ring.slot, ring.phase, sh, a.status, 74);
+                    ok = __all_sync(0xffffffffu, ok);                  // the warp acts as one
+                }
                 if (a.trace && p == 0 && lane == 0) { col_tally(a, t_rel, 4, w1c - w0c); col_tally(a, t_rel, 5, clock64() - w1c); }
-                ok = __all_sync(0xffffffffu, ok);                      // the warp acts as one
                 const uint32_t tile = smem_u32(tiles_b) + (uint32_t)ring.slot * slot_bytes + b_off;
                 const int nrb = ok ? (min(R, st.bt - c * R) + 31) >> 5 : 0;
 #pragma unroll
                 for (int rb2 = 0; rb2 < kColMaxChunkRows / 32; rb2 += 2) {
+                    // the four operand pairs of two 32-row blocks are fetched together, then used: one wait for shared
+                    // memory per pair of blocks instead of one per block and plane
+                    uint32_t r4[2][2][4], b0[2][2], b1[2][2];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int rb = rb2 + h;
-                        if (rb < nrb) {
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
-                            for (int pl = 0; pl < 2; ++pl) {
-                                uint32_t r4[4], b0, b1;
-                                ldsm_x4_trans(r4, tile + (uint32_t)pl * plane_bytes + (uint32_t)rb * 32u * kColBlockBytes);
-                                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1)
+                        for (int pl = 0; pl < 2; ++pl) {
+                            const int rb = rb2 + h;
+                            if (rb < nrb) {
+                                ldsm_x4_trans(r4[h][pl], tile + (uint32_t)pl * plane_bytes + (uint32_t)rb * 32u * kColBlockBytes);
+                                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0[h][pl]), "=r"(b1[h][pl])
                                              : "r"(rdig_lane + (uint32_t)(((rbuf * 2 + pl) * NRD) * rstride + rb * 32)));
+                            }
+                        }
+#pragma unroll
+                    for (int pl = 0; pl < 2; ++pl)                   // (neighbouring MMAs go to different accumulators)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (rb2 + h < nrb) {
                                 // bytes {2g, 2g+1} of rows {2t, 2t+1} of the four 8-row groups -> byte 2g (and 2g+1) of rows
                                 // {2t, 2t+1, 8+2t, 9+2t} (+16): features x rows, in the row order of the residual digits
-                                const uint32_t e0 = __byte_perm(r4[0], r4[1], 0x6420), o0 = __byte_perm(r4[0], r4[1], 0x7531);
-                                const uint32_t e1 = __byte_perm(r4[2], r4[3], 0x6420), o1 = __byte_perm(r4[2], r4[3], 0x7531);
+                                const uint32_t* r = r4[h][pl];
+                                const uint32_t e0 = __byte_perm(r[0], r[1], 0x6420), o0 = __byte_perm(r[0], r[1], 0x7531);
+                                const uint32_t e1 = __byte_perm(r[2], r[3], 0x6420), o1 = __byte_perm(r[2], r[3], 0x7531);
 #pragma unroll
                                 for (int g = 0; g < NG; ++g) {
                                     // All groups of a byte meet the same residual digits, so the sums may nest: accumulator g
                                     // takes the byte with the groups below g cleared (g = 0: the byte as it is), i.e.
                                     // sum_{h >= g} 2^(h CB) code_h; group g is the difference of two neighbours.
                                     const uint32_t mk = 0x01010101u * (uint32_t)((0xFFu << (g * CB)) & 0xFFu);
-                                    mma_u8s8(acc2[h][g], e0 & mk, o0 & mk, e1 & mk, o1 & mk, b0, b1);
+                                    mma_u8s8(acc2[h][g], e0 & mk, o0 & mk, e1 & mk, o1 & mk, b0[h][pl], b1[h][pl]);
                                 }
                             }
                         }
-                    }
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -659,7 +677,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
         }
     }
     // =================================================================================== R warps: residual digits
-    else {
+    else if (warp < kColWarpS2) {
         // Each R warp works alone on the chunks q = rw (mod kColRWarps) of the launch's sequence, with a digit buffer
         // of its own: that many exchanges are in flight at a time.  The warps meet twice per step: for the largest
         // |label| and for the step's sums.
@@ -765,16 +783,6 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         if (__any_sync(0xffffffffu, give_up)) { sh->abort_flag = 1; ok = false; }
                     }
                 }
-                // every CTA has left step t - 1 behind: its buffer of dot words is cleared for step t + 2 (this CTA's share)
-                if (c == 0 && ok) {
-                    __threadfence();        // (see "Memory order" above: the others' reads of that buffer before these stores)
-                    long long* z = a.dots + (size_t)((t_rel + 2) % 3) * ngrp * 2 * a.bpad;
-                    const int z0 = cta * zper, z1 = min(a.bpad, z0 + zper);
-#pragma unroll 1
-                    for (int g = 0; g < 2 * ngrp; ++g)
-#pragma unroll 1
-                        for (int i = z0 + lane; i < z1; i += 32) z[(size_t)g * a.bpad + i] = 0;
-                }
                 const long long e0c = (a.trace && rw == 0) ? clock64() : 0;
                 if (ok && q >= kColRWarps) ok = col_wait(sh->rempty + rw, (uint32_t)(((q >> kColRShift) - 1) & 1), sh, a.status, 76);
                 ok = __all_sync(0xffffffffu, ok);
@@ -797,24 +805,41 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         u1[i] = (unsigned long long)(R1 + kColBiasR);
                         u2[i] = (unsigned long long)(R2 + kColBiasR);
                     }
+                    // a 28-bit half becomes four 7-bit digits, a byte each, minus 64 as signed bytes; the four rows' words are
+                    // then transposed into one word per digit
                     signed char* dst = rd + blk * 32 + tl * 8 + hf * 4;
 #pragma unroll
-                    for (int s = 0; s < NRD; ++s) {
-                        uint32_t wa = 0u, wb = 0u;                       // digit s of r2 (meets plane 1) and of r1 (meets plane 2)
+                    for (int h = 0; h < 4; ++h) {                        // digits 0..3, 4..7 of r2 (meets plane 1), then of r1
+                        uint32_t e[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            wa |= (uint32_t)((u2[i] >> (7 * s)) & 127ull) << (8 * i);
-                            wb |= (uint32_t)((u1[i] >> (7 * s)) & 127ull) << (8 * i);
+                            const unsigned long long u = h < 2 ? u2[i] : u1[i];
+                            const uint32_t x = (h & 1) ? (uint32_t)(u >> 28) : ((uint32_t)u & 0xFFFFFFFu);
+                            uint32_t v = (x & 0x7Fu) | ((x & 0x3F80u) << 1) | ((x & 0x1FC000u) << 2) | ((x & 0xFE00000u) << 3);
+                            v ^= 0x40404040u; v |= (v & 0x40404040u) << 1;
+                            e[i] = v;
                         }
-                        wa ^= 0x40404040u; wa |= (wa & 0x40404040u) << 1;      // every byte minus 64, as a signed byte
-                        wb ^= 0x40404040u; wb |= (wb & 0x40404040u) << 1;
-                        *reinterpret_cast<uint32_t*>(dst + (size_t)s * rstride) = wa;
-                        *reinterpret_cast<uint32_t*>(dst + (size_t)(NRD + s) * rstride) = wb;
+                        const uint32_t t0 = __byte_perm(e[0], e[1], 0x5140), t1 = __byte_perm(e[2], e[3], 0x5140);
+                        const uint32_t t2 = __byte_perm(e[0], e[1], 0x7362), t3 = __byte_perm(e[2], e[3], 0x7362);
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)(4 * h + 0) * rstride) = __byte_perm(t0, t1, 0x5410);
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)(4 * h + 1) * rstride) = __byte_perm(t0, t1, 0x7632);
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)(4 * h + 2) * rstride) = __byte_perm(t2, t3, 0x5410);
+                        *reinterpret_cast<uint32_t*>(dst + (size_t)(4 * h + 3) * rstride) = __byte_perm(t2, t3, 0x7632);
                     }
                 }
                 if (c != c_last) {                       // (the step's last chunk is released below, after the step's sums)
                     __syncwarp();
                     if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rw));
+                }
+                // (off the chunk's path) every CTA has left step t - 1 behind, as chunk 0's complete dots showed: its buffer of dot words is cleared for step t + 2 (this CTA's share)
+                if (c == 0 && ok) {
+                    __threadfence();        // (see "Memory order" above: the others' reads of that buffer before these stores)
+                    long long* z = a.dots + (size_t)((t_rel + 2) % 3) * ngrp * 2 * a.bpad;
+                    const int z0 = cta * zper, z1 = min(a.bpad, z0 + zper);
+#pragma unroll 1
+                    for (int g = 0; g < 2 * ngrp; ++g)
+#pragma unroll 1
+                        for (int i = z0 + lane; i < z1; i += 32) z[(size_t)g * a.bpad + i] = 0;
                 }
             }
             // ---- the step's residuals are all known: their sum for the B warps, the next step's bound and unit
