@@ -14,9 +14,10 @@
 // exchange of its dots (several L2 round trips under load) may take as long as it likes without holding
 // the stream up:
 //
-//   service   (1 warp)   lane 0: tensor copies into two rings of slots, "A" (first visit, ahead of the A
-//                        warps, across step boundaries: codes do not depend on the model) and "B" (second
-//                        visit, in the same order, as far ahead of the B warps as that ring allows)
+//   service   (2 warps)  lane 0 of each: tensor copies into a ring of slots, "A" (first visit, ahead of the A
+//                        warps, across step boundaries: codes do not depend on the model) for warp 0, "B"
+//                        (second visit, in the same order, as far ahead of the B warps as that ring allows) for
+//                        the last warp; each sleeps on its ring's barrier
 //   A warps   (8)        partial dots of the chunk on the int8 tensor cores (mma.sync m16n8k32, u8 codes x
 //                        s8 digits of w), converted to a fixed-point unit common to all CTAs and added to
 //                        the row's word with one 64-bit integer atomic, whose low byte counts the CTAs
@@ -47,13 +48,17 @@
 //
 // The machine code is kept small on purpose (four roles share the instruction cache): 32-bit counters kept up
 // step by step instead of 64-bit divisions, waits as functions with one copy, loops unrolled only where
-// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 26.2 us per step (stream engine:
-// 29.8), DRAM reads 1.00 x the packed bytes; the R warps (an L2 round trip or two and the digits per chunk)
-// and the instruction issue rate of the SM, not HBM, bound it.
+// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 25.2 us per step (stream engine:
+// 29.8), DRAM reads 1.00 x the packed bytes.  Not HBM bounds it but the chain of a step: the first chunk's dots
+// have to cross L2 and become digits before pass B can start (about 9 k cycles), pass B then follows the R
+// warps (about 2 k cycles per chunk for the four of them together) rather than the copies, and the next
+// step's first dots come 6 k cycles after the last chunk's gradient.  With pass B's arithmetic taken out the
+// step is 13 % shorter, with pass A's arithmetic taken out not at all; more warps for any one role slow the
+// others by as much (the SM issues about two instructions per cycle in every variant tried).
 //
 // Memory order.  A buffer of dot words serves every third step and is cleared in between by the R warp that
-// has just seen the first chunk of step t complete (then every CTA has left step t-1, the buffer's last
-// use, behind: hence its fence before the stores); the A warps fence once per step before their first
+// has seen the first chunk of step t complete (then every CTA has left step t-1, the buffer's last use,
+// behind: hence its fence before the stores), once that chunk's digits are out; the A warps fence once per step before their first
 // addition, so that whoever sees a CTA's additions of step t+1 -- which every adder of step t+2 has -- also
 // sees its cleared share.
 #include <cuda.h>
