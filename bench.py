@@ -151,6 +151,9 @@ def main():
     ap.add_argument("--chunk-rows", type=int, default=0, help="column engine: rows per chunk (0 = automatic)")
     ap.add_argument("--feature-parts", type=int, default=0)
     ap.add_argument("--row-parts", type=int, default=0)
+    ap.add_argument("--sharded", action="store_true",
+                    help="N > 1: one epoch over all ranks' rows (every minibatch split by rows, one all-reduce of n floats "
+                         "per step) instead of N independent replicas")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", dest="others", action="store_false",
@@ -218,7 +221,14 @@ def main():
               "ring": binding.ENGINE_RING, "lean": binding.ENGINE_LEAN, "cluster": binding.ENGINE_CLUSTER,
               "stream": binding.ENGINE_STREAM, "column": binding.ENGINE_COLUMN}[args.engine]
 
-    w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + rank)
+    sharded = args.sharded and world > 1
+    w, A, b, _ = synth.make(args.workload, m=args.m, device=dev, seed=base.seed + (0 if sharded else rank))
+    plan = None
+    if sharded:
+        # every rank draws the same samples and keeps its rows of every minibatch (quantized with its own draws)
+        from paper_1611_05402_b200 import sharded as sh
+        plan = sh.ShardPlan(w.m, w.batch, rank, world)
+        A, b = sh.take_rows(plan, A), sh.take_rows(plan, b)
     ctx = binding.Context(dev)
     loss_dev = torch.zeros(1, dtype=torch.float64, device=dev)
     kw = dict(model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed, engine=engine,
@@ -243,7 +253,12 @@ def main():
         ds = timed(quant_events, record, quant)
         x = torch.zeros(w.n, dtype=torch.float32, device=dev)
         for ep in range(w.epochs):
-            timed(epoch_events, record, lambda: ctx.zipml_sgd_epoch(ds, b, x, w.batch, w.lr, epoch=ep, **kw))
+            if sharded:
+                run = sh.ShardedEpoch(ctx, plan, ds, b, x, w.lr, model_bits=w.model_bits, grad_bits=w.grad_bits, seed=w.seed,
+                                      epoch=ep, engine=engine)
+                timed(epoch_events, record, run.run)
+            else:
+                timed(epoch_events, record, lambda: ctx.zipml_sgd_epoch(ds, b, x, w.batch, w.lr, epoch=ep, **kw))
         timed(loss_events, record, lambda: ctx.zipml_loss(binding.LOSS_DENSE, b, x, A=A, out=loss_dev))
         return ds, x
 
@@ -269,7 +284,8 @@ def main():
     clocks = sampler.stop()
     ctx.zipml_sync()
     launches = ctx.zipml_kernel_launches() - launches0
-    whole_value, ms_total = replicas.whole_job_value(w.m * w.epochs * args.steps, t0.elapsed_time(t1), dev)
+    units = w.m / world if sharded else w.m           # (whole_job_value multiplies by the ranks)
+    whole_value, ms_total = replicas.whole_job_value(units * w.epochs * args.steps, t0.elapsed_time(t1), dev)
     final_loss = float(loss_dev.item())
 
     # dominant kernel: the SGD epoch launch
@@ -278,7 +294,7 @@ def main():
     packed_bytes = ds.packed_bytes
     peak, peak_kind = measured_peaks()
     achieved = packed_bytes / (epoch_avg_ms * 1e-3) / 1e9
-    value, _ = replicas.whole_job_value(w.m, epoch_avg_ms, dev)          # samples/s per SGD epoch, all ranks
+    value, _ = replicas.whole_job_value(units, epoch_avg_ms, dev)        # samples/s per SGD epoch, all ranks
     steps_per_epoch = (w.m + w.batch - 1) // w.batch
     step_us = 1e3 * epoch_avg_ms / steps_per_epoch
     step_bytes = packed_bytes / steps_per_epoch
@@ -314,7 +330,7 @@ def main():
 
     # ------------------------------------------------------------------ end to end from host buffers
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sharded:           # (the host entry point runs one device's rows: a replica's figure)
         Ah = torch.empty(A.shape, dtype=torch.float32, pin_memory=True)
         Ah.copy_(A)
         bh = torch.empty(b.shape, dtype=torch.float32, pin_memory=True)
@@ -396,12 +412,12 @@ def main():
     if rank == 0:
         print(json.dumps({
             "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "m": w.m, "n": w.n, "bits": w.bits, "batch": w.batch, "epochs": w.epochs,
                        "levels": w.levels, "model_bits": w.model_bits, "grad_bits": w.grad_bits, "engine": args.engine,
                        "l2": "inputs larger than L2 (dense A and both planes are streamed every step)",
-                       "multi_gpu": "replicas only"},
+                       "multi_gpu": "row-sharded epoch, one all-reduce of n floats per step" if sharded else "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline, "final_loss": final_loss,
             "packed_gb_per_s_per_epoch": achieved, "whole_path_samples_per_s": whole_value,

@@ -293,6 +293,18 @@ int zipml_loss_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const 
 int zipml_sgd_epoch_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const float* b, float* x,
                                 const zipml_sgd_params* params, float* grad_out);
 
+/* The end of a step on its own: x <- R(x - lr * Q4(g)) for a gradient g (n floats, device memory) that the caller has
+ * formed, e.g. the sum of several devices' shares of a minibatch (paper "End-to-end Quantization" for Q4, the
+ * l2-scaled sign-magnitude quantizer of the Supplement; Eq. (proxupdate) and the LS-SVM term for R).  Read from
+ * `params`: lr, grad_bits (0: g as it is), seed and epoch (with `step`, the step's position in the batch order, they
+ * key Q4's draws exactly as zipml_sgd_epoch does, so a gradient equal to the one that call forms gives the same
+ * update), reg, reg_param.  x (n floats, device memory) is updated in place; applied_out (DEVICE pointer or NULL)
+ * receives the n floats of Q4(g).  The pre-Q4 gradient of one step comes from zipml_sgd_epoch with num_steps = 1,
+ * lr = 0, grad_bits = 0, reg = ZIPML_REG_NONE and grad_out set (its first n floats; x is left as it was).
+ * Errors: ZIPML_ERR_INVALID_ARG / ZIPML_ERR_UNSUPPORTED as for zipml_sgd_epoch; nothing is launched then. */
+int zipml_sgd_apply_gradient(zipml_ctx* ctx, float* x, const float* g, int64_t n, const zipml_sgd_params* params,
+                             int64_t step, float* applied_out);
+
 /* Whole path from HOST buffers, for callers that hold their data in host memory: copies A and b to
  * the device, quantizes (UNIFORM, or TABLE with levels from zipml_optimal_levels when
  * optimal_levels != 0), runs `epochs` epochs of zipml_sgd_epoch (epoch index e = 0..epochs-1, step

@@ -19,7 +19,7 @@ ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGIN
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
 EXPORTS = ["zipml_up_row_bytes", "zipml_shared_base_encode", "zipml_shared_base_decode", "zipml_loss_shared_base",
-           "zipml_sgd_epoch_shared_base", "zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+           "zipml_sgd_epoch_shared_base", "zipml_sgd_apply_gradient", "zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -90,6 +90,7 @@ def lib():
         L.zipml_shared_base_decode.argtypes = [vp, C.POINTER(CSharedBase), vp, vp]
         L.zipml_loss_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, vp]
         L.zipml_sgd_epoch_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, C.POINTER(CSgdParams), vp]
+        L.zipml_sgd_apply_gradient.argtypes = [vp, vp, vp, C.c_int64, C.POINTER(CSgdParams), C.c_int64, vp]
         L.zipml_quantize.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
         L.zipml_optimal_levels.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp]
         L.zipml_sgd_epoch.argtypes = [vp, C.POINTER(CDataset), vp, vp, C.POINTER(CSgdParams), vp]
@@ -281,6 +282,14 @@ class Context:
         _check(lib().zipml_sgd_epoch_shared_base(self._h, C.byref(d), _ptr(b, torch.float32, self.device),
                                                  _ptr(x, torch.float32, self.device), C.byref(p),
                                                  _ptr(grad_out, torch.float32, self.device)), "zipml_sgd_epoch_shared_base")
+        del keep
+
+    def zipml_sgd_apply_gradient(self, x, g, step, lr, applied_out=None, **kw):
+        """x <- R(x - lr * Q4(g)) in place (see zipml_sgd_apply_gradient); kw as for sgd_params."""
+        p, keep = self.sgd_params(1, lr, **kw)
+        _check(lib().zipml_sgd_apply_gradient(self._h, _ptr(x, torch.float32, self.device), _ptr(g, torch.float32, self.device),
+                                              x.numel(), C.byref(p), step, _ptr(applied_out, torch.float32, self.device)),
+               "zipml_sgd_apply_gradient")
         del keep
 
     def zipml_optimal_levels(self, A, bits, hist_bins=1024, want_objective=False):

@@ -285,6 +285,19 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     return launch_sgd_epoch(ctx, data, b, x, params, first, count, grad_out);
 }
 
+int zipml_sgd_apply_gradient(zipml_ctx* ctx, float* x, const float* g, int64_t n, const zipml_sgd_params* params,
+                             int64_t step, float* applied_out) {
+    if (!ctx || !params || params->struct_size != sizeof(zipml_sgd_params)) return ZIPML_ERR_INVALID_ARG;
+    if (!x || !g || n <= 0 || n > 0x7fffffffLL || step < 0 || step > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
+    if (params->grad_bits != 0 && (params->grad_bits < 2 || params->grad_bits > 8)) return ZIPML_ERR_UNSUPPORTED;
+    if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
+    if (params->reg < ZIPML_REG_NONE || params->reg > ZIPML_REG_LSSVM) return ZIPML_ERR_INVALID_ARG;
+    if (params->reg != ZIPML_REG_NONE && params->reg != ZIPML_REG_NONNEG && !(params->reg_param >= 0.0f)) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    return launch_sgd_apply(ctx, x, g, n, params, step, applied_out);
+}
+
 int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, int32_t iterations, uint64_t* ns_out) {
     if (!ctx || !ns_out || ctas < 1 || floats_per_cta < 0 || floats_per_cta % 4 != 0 || iterations < 1 || iterations > (1 << 20))
         return ZIPML_ERR_INVALID_ARG;

@@ -94,6 +94,8 @@ int launch_sgd_cluster(zipml_ctx* ctx, const zipml_dataset* d, const float* b, f
 int launch_sgd_stream(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                       int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
 // Column engine (uniform grids, fp32 model and gradient, rows of at most 128 bytes per SM).
+int launch_sgd_apply(zipml_ctx* ctx, float* x, const float* g, int64_t n, const zipml_sgd_params* p, int64_t step,
+                     float* applied_out);
 int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, float* x, const zipml_sgd_params* p,
                       int64_t first_step, int64_t num_steps, float* grad_out, bool only_if_profitable);
 // Both planes of d into the other layout (see ZIPML_LAYOUT_* in zipml.h).

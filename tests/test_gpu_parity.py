@@ -871,3 +871,89 @@ def test_train_host_matches_oracle_pipeline(ctx):
         xr, _ = oracle.sgd_epoch(ods, b, xr, 512, np.float32(0.05) / np.float32(ep + 1), epoch=ep)
     assert rel(x.numpy(), xr) <= MODEL_TOL
     assert abs(loss - oracle.loss_dense(A, b, xr)) <= 1e-3 * oracle.loss_dense(A, b, xr)
+
+
+@pytest.mark.parametrize("grad_bits,reg,reg_param", [(0, 0, 0.0), (6, 0, 0.0), (8, 1, 0.5), (4, 2, 0.01), (0, 3, 0.0), (5, 4, 0.3)])
+def test_apply_gradient_is_the_end_of_a_step(ctx, grad_bits, reg, reg_param):
+    """zipml_sgd_apply_gradient: Q4 (Supplement "Quantizing the Gradients") and the update (Eq. (proxupdate), LS-SVM
+    term) on a gradient from outside, with the draws of zipml_sgd_epoch: fed the oracle's own pre-Q4 gradient of a
+    step it must land on the oracle's model after that step."""
+    m, n, batch, lr, seed, epoch, step = 1500, 700, 256, 0.02, 9, 3, 4
+    _, A, b, _ = workload("c1", m, n, seed=8)
+    ods = oracle.quantize(A, 4, seed=1)
+    x0 = (np.random.default_rng(2).standard_normal(n) * 0.1).astype(np.float32)
+    x1, g_ref = oracle.sgd_epoch(ods, b, x0, batch, lr, grad_bits=grad_bits, seed=seed, epoch=epoch, first_step=step,
+                                 num_steps=1, want_grad=True, reg=reg, reg_param=reg_param)
+    x, g = to_dev(x0, ctx), to_dev(g_ref[0], ctx)
+    applied = torch.zeros(n, dtype=torch.float32, device=ctx.device)
+    ctx.zipml_sgd_apply_gradient(x, g, step, lr, applied_out=applied, grad_bits=grad_bits, seed=seed, epoch=epoch, reg=reg,
+                                 reg_param=reg_param)
+    ctx.zipml_sync()
+    got, app = x.cpu().numpy(), applied.cpu().numpy()
+    if grad_bits:
+        unit = np.linalg.norm(g_ref[0]) / ((1 << (grad_bits - 1)) - 1)
+        flips = np.abs(app - g_ref[1]) > 0.5 * unit                # (a last-bit difference in the norm may flip a rounding)
+        assert flips.sum() <= 2
+        assert np.abs(app - g_ref[1])[~flips].max() <= 1e-5 * unit + 1e-12
+        assert np.abs(got - x1)[~flips].max() <= 1e-6 * max(1.0, np.abs(x1).max())
+    else:
+        assert (app == g_ref[0]).all()
+        assert np.abs(got - x1).max() <= 1e-6 * max(1.0, np.abs(x1).max())
+    # refusals: nothing runs
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_apply_gradient(x, g, -1, lr)
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_apply_gradient(x, g, 0, lr, grad_bits=1)
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_apply_gradient(x, g, 0, lr, reg=1, reg_param=-1.0)
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+@pytest.mark.parametrize("case", ["plain_ragged", "q3_q4_shuffled", "wide_l2"])
+def test_row_sharded_epoch_matches_the_whole_epoch(ctx, world, case):
+    """The row-sharded epoch (one all-reduce of n floats per step) with its ranks run in turn on this GPU, every
+    rank on its own rows and its own replica of x: all replicas end as the same bits, at the model of the
+    unsharded zipml_sgd_epoch and of the oracle's epoch."""
+    from paper_1611_05402_b200.sharded import ShardPlan, ShardedEpoch, take_rows
+    m, n, bits, batch, mb, gb, shuffled, reg, rp = {
+        "plain_ragged": (1100, 300, 4, 128, 0, 0, False, 0, 0.0),      # last batch: 76 rows: some ranks hold none of it
+        "q3_q4_shuffled": (1024, 520, 2, 256, 8, 8, True, 0, 0.0),
+        "wide_l2": (900, 4096, 4, 512, 0, 0, False, 1, 0.2),           # big steps: other engines serve the shares
+    }[case]
+    lr, seed, epoch = 0.01, 11, 2
+    _, A, b, _ = workload("c1", m, n, seed=4)
+    ods = oracle.quantize(A, bits, seed=3)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    T = (m + batch - 1) // batch
+    order = [int(o) for o in np.random.default_rng(1).permutation(T)] if shuffled else None
+    x0 = np.zeros(n, np.float32)
+    kw = dict(model_bits=mb, grad_bits=gb, seed=seed, epoch=epoch, reg=reg, reg_param=rp)
+    ranks = []
+    for r in range(world):
+        plan = ShardPlan(m, batch, r, world)
+        p1, p2 = take_rows(plan, gds.plane1), take_rows(plan, gds.plane2)
+        dl = binding.Dataset(p1, p2, p1.shape[0], n, bits, gds.level_mode, gds.feat_lo, gds.feat_step, gds.levels)
+        ranks.append(ShardedEpoch(ctx, plan, dl, take_rows(plan, db), to_dev(x0, ctx), lr, batch_order=order, **kw))
+    pos = [0]
+
+    def all_reduce(v):                     # rank 0's share arrives; the others' are formed and added, and applied
+        t = order[pos[0]] if order else pos[0]
+        for other in ranks[1:]:
+            v += other.share(pos[0], t, other.plan.weight(t))
+        for other in ranks[1:]:
+            other.apply(v.clone(), pos[0])
+        pos[0] += 1
+
+    ranks[0].run(all_reduce=all_reduce)
+    ctx.zipml_sync()
+    xs = [rk.x.cpu().numpy() for rk in ranks]
+    for other in xs[1:]:
+        assert np.array_equal(xs[0], other)
+    whole = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, whole, batch, lr, batch_order=order, **kw)
+    ctx.zipml_sync()
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, batch_order=order, **kw)
+    assert np.abs(x_ref).max() > 1e-3
+    tol = (20 if (mb or gb) else 1) * MODEL_TOL
+    assert rel(xs[0], x_ref) <= tol
+    assert rel(xs[0], whole.cpu().numpy()) <= 2 * tol
