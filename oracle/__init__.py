@@ -52,6 +52,9 @@ def _declare(L):
     L.orc_shared_base_decode.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp]
     L.orc_column_range.argtypes = [vp, i64, i64, i64, vp, vp]
     L.orc_quantize.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
+    L.orc_quantize_pair.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, C.c_uint32, vp, vp, i64, vp, vp]
+    L.orc_poly_rows.argtypes = [vp, i32, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.orc_weighted_plane_mean.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp]
     L.orc_dequantize_row.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
     L.orc_dequantize_row.restype = None
     L.orc_quantize_vector.argtypes = [vp, i64, i32, u64, u32, u32, u32, vp, vp]
@@ -194,6 +197,47 @@ def quantize(A, bits, seed, mode=UNIFORM, levels=None):
         levels = np.ascontiguousarray(levels, dtype=np.float32)
     _check(lib().orc_quantize(_p(A), m, n, n, bits, mode, _p(levels), seed, _p(p1), _p(p2), rb, _p(lo), _p(step)))
     return Dataset(p1, p2, m, n, bits, mode, lo, step, levels)
+
+
+def quantize_pair(A, bits, seed, pair, mode=UNIFORM, levels=None):
+    """Pair `pair` of independent quantizations of A on the grid of quantize(): planes 2 pair + 1, 2 pair + 2 of
+    Q_1, Q_2, ... (Section 4.1); pair 0 is quantize()."""
+    A = np.ascontiguousarray(A, dtype=np.float32)
+    m, n = A.shape
+    rb = row_bytes(n, bits)
+    p1, p2 = np.zeros((m, rb), np.uint8), np.zeros((m, rb), np.uint8)
+    lo = np.zeros(n, np.float32)
+    step = np.zeros(n, np.float32) if mode == UNIFORM else None
+    if levels is not None:
+        levels = np.ascontiguousarray(levels, dtype=np.float32)
+    _check(lib().orc_quantize_pair(_p(A), m, n, n, bits, mode, _p(levels), seed, pair, _p(p1), _p(p2), rb, _p(lo), _p(step)))
+    return Dataset(p1, p2, m, n, bits, mode, lo, step, levels)
+
+
+def poly_rows(planes, ds, x, coef, scale=None):
+    """Q(P) per sample (Section 4.1) from the planes Q_1 .. Q_d (arrays like ds.plane1), coef = (m_0 .. m_d); times
+    scale[k] where given."""
+    d = len(coef) - 1
+    assert len(planes) >= d
+    planes = [np.ascontiguousarray(p) for p in planes[:d]]
+    ptrs = (C.c_void_p * max(d, 1))(*[p.ctypes.data for p in planes])
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    coef = np.ascontiguousarray(coef, dtype=np.float64)
+    scale = None if scale is None else np.ascontiguousarray(scale, dtype=np.float32)
+    out = np.zeros(ds.m, np.float64)
+    _check(lib().orc_poly_rows(ptrs, d, ds.row_bytes, ds.m, ds.n, ds.bits, ds.mode, _p(ds.feat_lo), _p(ds.feat_step),
+                               _p(ds.levels), _p(x), _p(coef), _p(scale), _p(out)))
+    return out
+
+
+def weighted_plane_mean(plane, ds, c):
+    """(1/m) sum_k c_k Q(a_k) for the plane Q (Section 4.2: the gradient for factors c_k = b_k Q(P)_k)."""
+    plane = np.ascontiguousarray(plane)
+    c = np.ascontiguousarray(c, dtype=np.float64)
+    g = np.zeros(ds.n, np.float64)
+    _check(lib().orc_weighted_plane_mean(_p(plane), ds.row_bytes, ds.m, ds.n, ds.bits, ds.mode, _p(ds.feat_lo),
+                                         _p(ds.feat_step), _p(ds.levels), _p(c), _p(g)))
+    return g
 
 
 def quantize_vector(v, bits, seed, epoch, step, stream):

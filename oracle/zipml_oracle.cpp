@@ -76,8 +76,15 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 // 24-bit uniform integer for sample element (row, feature), copy in {1, 2}.  One Philox block
 // serves the feature pair (2f, 2f+1): counter (row_lo, row_hi, feature >> 1, 0), key = seed,
 // output word 2*(feature & 1) + (copy - 1); the top 24 bits of the word are used.
+uint32_t orc_u24_sample_pair(uint64_t seed, uint64_t row, uint32_t feature, uint32_t copy, uint32_t pair);
 uint32_t orc_u24_sample(uint64_t seed, uint64_t row, uint32_t feature, uint32_t copy) {
-    const uint32_t ctr[4] = {(uint32_t)row, (uint32_t)(row >> 32), feature >> 1, 0u};
+    return orc_u24_sample_pair(seed, row, feature, copy, 0u);
+}
+
+// The same for further, independent pairs of quantizations of the same sample (Section 4.1 "Quantizing
+// Polynomials" uses d of them): pair q differs in the counter's last word, (row_lo, row_hi, feature >> 1, q).
+uint32_t orc_u24_sample_pair(uint64_t seed, uint64_t row, uint32_t feature, uint32_t copy, uint32_t pair) {
+    const uint32_t ctr[4] = {(uint32_t)row, (uint32_t)(row >> 32), feature >> 1, pair};
     const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
@@ -237,9 +244,20 @@ static inline void table_cell(float v, const float* lev, int s, uint32_t* cell, 
 // Two independent unbiased quantizations of every sample, bit-packed (double sampling, Eq. (double)).
 // Out: plane1, plane2 (m * row_bytes each), feat_lo (n), feat_step (n; uniform grid only: (hi-lo)/s).
 // For ORC_LEVELS_TABLE `levels` is n x L ascending fp32 with levels[j][0] <= every value <= levels[j][s].
+int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
+                      const float* levels, uint64_t seed, uint32_t pair, uint8_t* plane1, uint8_t* plane2,
+                      int64_t row_bytes, float* feat_lo, float* feat_step);
 int orc_quantize(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
                  const float* levels, uint64_t seed, uint8_t* plane1, uint8_t* plane2,
                  int64_t row_bytes, float* feat_lo, float* feat_step) {
+    return orc_quantize_pair(A, m, n, lda, bits, level_mode, levels, seed, 0u, plane1, plane2, row_bytes, feat_lo, feat_step);
+}
+
+// Pair `pair` of quantizations of the same samples on the same grid: planes 2 pair + 1 and 2 pair + 2 of the
+// sequence Q_1, Q_2, ... (pair 0 is orc_quantize).
+int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
+                      const float* levels, uint64_t seed, uint32_t pair, uint8_t* plane1, uint8_t* plane2,
+                      int64_t row_bytes, float* feat_lo, float* feat_step) {
     const int cb = orc_container_bits(bits);
     if (cb == 0) return ORC_ERR_UNSUPPORTED;
     if (level_mode == ORC_LEVELS_TABLE && bits == 8) return ORC_ERR_UNSUPPORTED;
@@ -268,8 +286,8 @@ int orc_quantize(const float* A, int64_t m, int64_t n, int64_t lda, int bits, in
             uint32_t cell; float p;
             if (level_mode == ORC_LEVELS_UNIFORM) uniform_cell(v, lo[j], inv[j], s, &cell, &p);
             else table_cell(v, levels + j * L, s, &cell, &p);
-            put_code(r1, j, cb, round_up_if(cell, p, orc_u24_sample(seed, (uint64_t)k, (uint32_t)j, 1)));
-            put_code(r2, j, cb, round_up_if(cell, p, orc_u24_sample(seed, (uint64_t)k, (uint32_t)j, 2)));
+            put_code(r1, j, cb, round_up_if(cell, p, orc_u24_sample_pair(seed, (uint64_t)k, (uint32_t)j, 1, pair)));
+            put_code(r2, j, cb, round_up_if(cell, p, orc_u24_sample_pair(seed, (uint64_t)k, (uint32_t)j, 2, pair)));
         }
     }
     return ORC_OK;
@@ -458,6 +476,47 @@ int orc_loss_codes(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byt
         acc += (d1 - (double)b[k]) * (d2 - (double)b[k]);
     }
     *loss_out = acc / (2.0 * (double)m);
+    return ORC_OK;
+}
+
+// Section 4.1 "Quantizing Polynomials": with d independent quantizations Q_1 .. Q_d of a sample a, the estimate
+// of P(a^T x) for P(z) = sum_{i=0}^{d} coef_i z^i is  Q(P) = sum_i coef_i prod_{j <= i} Q_j(a)^T x  (unbiased: the
+// factors of a product are independent).  planes[j] is Q_{j+1} (m x row_bytes, all on one grid).  rows_out[k] is
+// Q(P) of sample k, times scale_or_null[k] where that is given (the label b_k of Section 4.2's protocol).
+int orc_poly_rows(const uint8_t* const* planes, int d, int64_t row_bytes, int64_t m, int64_t n, int bits, int level_mode,
+                  const float* feat_lo, const float* feat_step, const float* levels, const float* x,
+                  const double* coef, const float* scale_or_null, double* rows_out) {
+    if (orc_container_bits(bits) == 0) return ORC_ERR_UNSUPPORTED;
+    if (!planes || d < 0 || !x || !coef || !rows_out || m <= 0 || n <= 0) return ORC_ERR_INVALID_ARG;
+    std::vector<double> q((size_t)n);
+    for (int64_t k = 0; k < m; ++k) {
+        double value = coef[0], prod = 1.0;
+        for (int i = 1; i <= d; ++i) {
+            orc_dequantize_row(planes[i - 1] + k * row_bytes, n, bits, level_mode, feat_lo, feat_step, levels, q.data());
+            double z = 0.0;
+            for (int64_t j = 0; j < n; ++j) z += q[j] * (double)x[j];
+            prod *= z;
+            value += coef[i] * prod;
+        }
+        rows_out[k] = scale_or_null ? (double)scale_or_null[k] * value : value;
+    }
+    return ORC_OK;
+}
+
+// The gradient of Section 4.2's protocol for given per-sample factors c_k (there: b_k Q(P)_k): the mean of
+// c_k Q_{d+1}(a_k) over the samples, with `plane` holding Q_{d+1}.
+int orc_weighted_plane_mean(const uint8_t* plane, int64_t row_bytes, int64_t m, int64_t n, int bits, int level_mode,
+                            const float* feat_lo, const float* feat_step, const float* levels, const double* c,
+                            double* g_out) {
+    if (orc_container_bits(bits) == 0) return ORC_ERR_UNSUPPORTED;
+    if (!plane || !c || !g_out || m <= 0 || n <= 0) return ORC_ERR_INVALID_ARG;
+    std::vector<double> q((size_t)n);
+    for (int64_t j = 0; j < n; ++j) g_out[j] = 0.0;
+    for (int64_t k = 0; k < m; ++k) {
+        orc_dequantize_row(plane + k * row_bytes, n, bits, level_mode, feat_lo, feat_step, levels, q.data());
+        for (int64_t j = 0; j < n; ++j) g_out[j] += c[k] * q[j];
+    }
+    for (int64_t j = 0; j < n; ++j) g_out[j] /= (double)m;
     return ORC_OK;
 }
 
