@@ -100,7 +100,7 @@ def test_weighted_plane_mean_against_exact_samples():
     ds = oracle.quantize_pair(A, 4, 9, 1)
     c = np.random.default_rng(4).standard_normal(30)
     assert np.allclose(oracle.weighted_plane_mean(ds.plane2, ds, c), (c[:, None] * A).mean(axis=0), rtol=1e-12, atol=1e-12)
-    assert np.allclose(oracle.weighted_plane_mean(ds.plane1, ds, np.ones(30)), A.mean(axis=0), rtol=1e-12)
+    assert np.allclose(oracle.weighted_plane_mean(ds.plane1, ds, np.ones(30)), A.astype(np.float64).mean(axis=0), rtol=1e-12)
     e = np.zeros(30)
     e[17] = 1.0
-    assert np.allclose(oracle.weighted_plane_mean(ds.plane1, ds, e), A[17] / 30.0, rtol=1e-12)
+    assert np.allclose(oracle.weighted_plane_mean(ds.plane1, ds, e), A[17].astype(np.float64) / 30.0, rtol=1e-12)
