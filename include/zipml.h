@@ -293,6 +293,30 @@ int zipml_loss_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const 
 int zipml_sgd_epoch_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, const float* b, float* x,
                                 const zipml_sgd_params* params, float* grad_out);
 
+/* Polynomials of a^T x over several independent quantizations (paper Section 4.1 "Quantizing Polynomials"; Section 4.2
+ * uses them for smooth classification losses).  ZIPML_POLY_MAX_DEGREE bounds the degree d.
+ * zipml_quantize_draw: zipml_quantize with a draw index: draw q gives the quantizations Q_{2q+1}, Q_{2q+2} of the same
+ *   samples on the same grid, independent of every other draw (the Philox counter's last word is q; draw 0 is
+ *   zipml_quantize itself).  d quantizations take ceil(d / 2) calls with the same seed.
+ * zipml_poly_rows: rows_out[k] (m doubles, device memory) = Q(P)_k = sum_{i=0..d} coef[i] * prod_{j<=i} Q_j(a_k)^T x,
+ *   times scale[k] where scale (m floats, device memory, e.g. the labels) is not NULL.  `grid` gives bits, level mode,
+ *   m, n, row_bytes and feat_lo / feat_step / levels (its plane pointers are checked like any data set's but not
+ *   read); planes is a HOST array of d
+ *   device pointers (16-byte aligned, stride grid->row_bytes, ZIPML_LAYOUT_ROWS), coef a HOST array of d + 1 doubles.
+ *   Dots as in zipml_loss's code path (fp32 products in short runs, combined in double); product and sum in double.
+ * zipml_weighted_plane_mean: g_out (n floats, device memory) = (1/m) sum_k c[k] * Q(a_k) for the plane Q and the m
+ *   doubles c (device memory): with c = b_k Q(P)_k and Q = Q_{d+1} the gradient of Section 4.2's protocol.  Sums
+ *   in double in a fixed order.
+ * Errors: ZIPML_ERR_INVALID_ARG (null or misaligned pointers, degree out of range, a bad `grid`), ZIPML_ERR_UNSUPPORTED
+ * (layout other than ZIPML_LAYOUT_ROWS); nothing is launched then. */
+#define ZIPML_POLY_MAX_DEGREE 8
+int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
+                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
+                        uint8_t* plane2, int64_t row_bytes, float* feat_lo, float* feat_step);
+int zipml_poly_rows(zipml_ctx* ctx, const zipml_dataset* grid, const uint8_t* const* planes, int32_t degree,
+                    const double* coef, const float* x, const float* scale, double* rows_out);
+int zipml_weighted_plane_mean(zipml_ctx* ctx, const zipml_dataset* grid, const uint8_t* plane, const double* c, float* g_out);
+
 /* The end of a step on its own: x <- R(x - lr * Q4(g)) for a gradient g (n floats, device memory) that the caller has
  * formed, e.g. the sum of several devices' shares of a minibatch (paper "End-to-end Quantization" for Q4, the
  * l2-scaled sign-magnitude quantizer of the Supplement; Eq. (proxupdate) and the LS-SVM term for R).  Read from

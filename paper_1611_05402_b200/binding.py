@@ -19,7 +19,7 @@ ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGIN
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "csrc", "libzipml.so")
 EXPORTS = ["zipml_up_row_bytes", "zipml_shared_base_encode", "zipml_shared_base_decode", "zipml_loss_shared_base",
-           "zipml_sgd_epoch_shared_base", "zipml_sgd_apply_gradient", "zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
+           "zipml_sgd_epoch_shared_base", "zipml_sgd_apply_gradient", "zipml_quantize_draw", "zipml_poly_rows", "zipml_weighted_plane_mean", "zipml_column_blocks_bytes", "zipml_convert_layout", "zipml_create", "zipml_destroy", "zipml_sync", "zipml_kernel_launches", "zipml_last_engine", "zipml_barrier_latency", "zipml_wait_probe", "zipml_strerror", "zipml_row_bytes", "zipml_quantize",
            "zipml_optimal_levels", "zipml_sgd_epoch", "zipml_loss", "zipml_train_host",
            "zipml_loss_codes_static"]
 
@@ -91,6 +91,9 @@ def lib():
         L.zipml_loss_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, vp]
         L.zipml_sgd_epoch_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, C.POINTER(CSgdParams), vp]
         L.zipml_sgd_apply_gradient.argtypes = [vp, vp, vp, C.c_int64, C.POINTER(CSgdParams), C.c_int64, vp]
+        L.zipml_quantize_draw.argtypes = [vp, vp, i64, i64, i64, C.c_int32, C.c_int32, vp, C.c_uint64, C.c_uint32, vp, vp, i64, vp, vp]
+        L.zipml_poly_rows.argtypes = [vp, C.POINTER(CDataset), vp, C.c_int32, vp, vp, vp, vp]
+        L.zipml_weighted_plane_mean.argtypes = [vp, C.POINTER(CDataset), vp, vp, vp]
         L.zipml_quantize.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
         L.zipml_optimal_levels.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp]
         L.zipml_sgd_epoch.argtypes = [vp, C.POINTER(CDataset), vp, vp, C.POINTER(CSgdParams), vp]
@@ -223,7 +226,8 @@ class Context:
         """Enqueues a bounded wait that must give up; the next zipml_sync raises ZipmlError(ERR_TIMEOUT)."""
         _check(lib().zipml_wait_probe(self._h, spin_limit), "zipml_wait_probe")
 
-    def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None):
+    def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None, draw=0):
+        """Two packed quantizations of A; draw > 0: further independent pairs on the same grid (zipml_quantize_draw)."""
         m, n = A.shape
         assert A.stride(1) == 1 and A.dtype == torch.float32 and A.device == self.device
         rb = int(lib().zipml_row_bytes(n, bits)) if row_bytes is None else row_bytes
@@ -233,9 +237,14 @@ class Context:
         p2 = torch.empty((m, rb), dtype=torch.uint8, device=self.device)
         lo = torch.empty(n, dtype=torch.float32, device=self.device)
         step = torch.empty(n, dtype=torch.float32, device=self.device) if level_mode == LEVELS_UNIFORM else None
-        _check(lib().zipml_quantize(self._h, C.c_void_p(A.data_ptr()), m, n, A.stride(0), bits, level_mode,
-                                    _ptr(levels, torch.float32, self.device), seed, _ptr(p1), _ptr(p2), rb, _ptr(lo),
-                                    _ptr(step)), "zipml_quantize")
+        if draw:
+            _check(lib().zipml_quantize_draw(self._h, C.c_void_p(A.data_ptr()), m, n, A.stride(0), bits, level_mode,
+                                             _ptr(levels, torch.float32, self.device), seed, draw, _ptr(p1), _ptr(p2), rb,
+                                             _ptr(lo), _ptr(step)), "zipml_quantize_draw")
+        else:
+            _check(lib().zipml_quantize(self._h, C.c_void_p(A.data_ptr()), m, n, A.stride(0), bits, level_mode,
+                                        _ptr(levels, torch.float32, self.device), seed, _ptr(p1), _ptr(p2), rb, _ptr(lo),
+                                        _ptr(step)), "zipml_quantize")
         return Dataset(p1, p2, m, n, bits, level_mode, lo, step, levels)
 
     def zipml_convert_layout(self, data, to_layout):
@@ -291,6 +300,29 @@ class Context:
                                               x.numel(), C.byref(p), step, _ptr(applied_out, torch.float32, self.device)),
                "zipml_sgd_apply_gradient")
         del keep
+
+    def zipml_poly_rows(self, grid, planes, coef, x, scale=None, out=None):
+        """Q(P) per sample from the planes Q_1 .. Q_d (device uint8 tensors of grid's shape), coef = (m_0 .. m_d)."""
+        d = len(coef) - 1
+        assert len(planes) >= d
+        for p in planes[:d]:
+            assert p.is_contiguous() and p.dtype == torch.uint8 and p.device == self.device
+        ptrs = (C.c_void_p * max(d, 1))(*[p.data_ptr() for p in planes[:d]])
+        cf = (C.c_double * (d + 1))(*[float(c) for c in coef])
+        out = torch.empty(grid.m, dtype=torch.float64, device=self.device) if out is None else out
+        g = grid.c_struct()
+        _check(lib().zipml_poly_rows(self._h, C.byref(g), ptrs, d, cf, _ptr(x, torch.float32, self.device),
+                                     _ptr(scale, torch.float32, self.device), _ptr(out, torch.float64, self.device)), "zipml_poly_rows")
+        return out
+
+    def zipml_weighted_plane_mean(self, grid, plane, c, out=None):
+        """(1/m) sum_k c[k] Q(a_k) for the plane Q (n floats)."""
+        out = torch.empty(grid.n, dtype=torch.float32, device=self.device) if out is None else out
+        g = grid.c_struct()
+        _check(lib().zipml_weighted_plane_mean(self._h, C.byref(g), _ptr(plane, torch.uint8, self.device),
+                                               _ptr(c, torch.float64, self.device), _ptr(out, torch.float32, self.device)),
+               "zipml_weighted_plane_mean")
+        return out
 
     def zipml_optimal_levels(self, A, bits, hist_bins=1024, want_objective=False):
         m, n = A.shape

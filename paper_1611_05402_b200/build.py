@@ -12,7 +12,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "_build")
 LIB = os.path.join(CSRC, "libzipml.so")
 SOURCES = ["api.cu", "quantize.cu", "levels.cu", "sgd.cu", "sgd_ring.cu", "sgd_lean.cu", "sgd_cluster.cu", "sgd_stream.cu",
-           "sgd_column.cu", "sgd_apply.cu", "shared_base.cu", "loss.cu"]
+           "sgd_column.cu", "sgd_apply.cu", "shared_base.cu", "poly.cu", "loss.cu"]
 HEADERS = ["common.cuh", "internal.h", "sgd_common.cuh", "int_digits.cuh", os.path.join("..", "..", "include", "zipml.h")]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--fmad=true",
          "-Xcompiler", "-fPIC"]

@@ -176,6 +176,12 @@ int zipml_sync(zipml_ctx* ctx) {
 int zipml_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
                    int32_t level_mode, const float* levels, uint64_t seed, uint8_t* plane1, uint8_t* plane2,
                    int64_t row_bytes, float* feat_lo, float* feat_step) {
+    return zipml_quantize_draw(ctx, A, m, n, lda, bits, level_mode, levels, seed, 0u, plane1, plane2, row_bytes, feat_lo, feat_step);
+}
+
+int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
+                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
+                        uint8_t* plane2, int64_t row_bytes, float* feat_lo, float* feat_step) {
     if (!ctx) return ZIPML_ERR_INVALID_ARG;
     const int cb = container_bits(bits);
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
@@ -197,7 +203,7 @@ int zipml_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t
     float* step_tmp = cv.take<float>((size_t)n);
     rc = launch_column_range(ctx, A, m, n, lda, s, keys, feat_lo, nullptr, inv, feat_step ? feat_step : step_tmp);
     if (rc != ZIPML_OK) return rc;
-    return launch_quantize(ctx, A, m, n, lda, bits, level_mode, feat_lo, inv, levels, seed, plane1, plane2, row_bytes);
+    return launch_quantize(ctx, A, m, n, lda, bits, level_mode, feat_lo, inv, levels, seed, draw, plane1, plane2, row_bytes);
 }
 
 int zipml_optimal_levels(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
@@ -304,6 +310,42 @@ int zipml_barrier_latency(zipml_ctx* ctx, int32_t ctas, int32_t floats_per_cta, 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
     return launch_barrier_latency(ctx, ctas, floats_per_cta, iterations, reinterpret_cast<unsigned long long*>(ns_out));
+}
+
+int zipml_poly_rows(zipml_ctx* ctx, const zipml_dataset* grid, const uint8_t* const* planes, int32_t degree,
+                    const double* coef, const float* x, const float* scale, double* rows_out) {
+    if (!ctx || !coef || !x || !rows_out || degree < 0 || degree > ZIPML_POLY_MAX_DEGREE) return ZIPML_ERR_INVALID_ARG;
+    int rc = check_dataset(grid);
+    if (rc != ZIPML_OK) return rc;
+    if (grid->layout != ZIPML_LAYOUT_ROWS) return ZIPML_ERR_UNSUPPORTED;
+    if (degree > 0 && !planes) return ZIPML_ERR_INVALID_ARG;
+    for (int i = 0; i < degree; ++i)
+        if (!planes[i] || !aligned16(planes[i])) return ZIPML_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    const bool table = grid->level_mode == ZIPML_LEVELS_TABLE;
+    const size_t wcount = (size_t)grid->n * (table ? ((size_t)1 << grid->bits) : 1);
+    rc = ws_reserve(ctx, carve_size(sizeof(float) * wcount) + carve_size(sizeof(double)));
+    if (rc != ZIPML_OK) return rc;
+    Carver cv(ctx->ws);
+    float* wtab = cv.take<float>(wcount);
+    double* base = cv.take<double>(1);
+    rc = launch_code_weights(ctx, grid, x, wtab, base);
+    if (rc != ZIPML_OK) return rc;
+    return launch_poly_rows(ctx, grid, planes, degree, coef, wtab, base, scale, rows_out);
+}
+
+int zipml_weighted_plane_mean(zipml_ctx* ctx, const zipml_dataset* grid, const uint8_t* plane, const double* c, float* g_out) {
+    if (!ctx || !plane || !c || !g_out || !aligned16(plane)) return ZIPML_ERR_INVALID_ARG;
+    int rc = check_dataset(grid);
+    if (rc != ZIPML_OK) return rc;
+    if (grid->layout != ZIPML_LAYOUT_ROWS) return ZIPML_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return ZIPML_ERR_CUDA;
+    const size_t count = (size_t)plane_mean_chunks(ctx, grid->m) * ((size_t)grid->n + 1);
+    rc = ws_reserve(ctx, carve_size(sizeof(double) * count));
+    if (rc != ZIPML_OK) return rc;
+    return launch_plane_mean(ctx, grid, plane, c, reinterpret_cast<double*>(ctx->ws), g_out);
 }
 
 int zipml_wait_probe(zipml_ctx* ctx, int64_t spin_limit) {

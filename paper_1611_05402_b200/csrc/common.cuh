@@ -52,8 +52,9 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
 
 // Random block of the sample feature pair (2p, 2p+1) of row `row`: words {2p copy 1, 2p copy 2,
 // 2p+1 copy 1, 2p+1 copy 2}; the top 24 bits of a word are the uniform integer.
-__device__ __forceinline__ Philox4 sample_block(uint64_t seed, uint64_t row, uint32_t pair) {
-    return philox4x32_10((uint32_t)row, (uint32_t)(row >> 32), pair, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+// `draw` numbers further independent pairs of quantizations of the same samples (0: the two samples of the SGD path).
+__device__ __forceinline__ Philox4 sample_block(uint64_t seed, uint64_t row, uint32_t pair, uint32_t draw) {
+    return philox4x32_10((uint32_t)row, (uint32_t)(row >> 32), pair, draw, (uint32_t)seed, (uint32_t)(seed >> 32));
 }
 
 // Uniform 24-bit integer for coordinate `coord` of the model (stream 3) / gradient (stream 4)

@@ -68,8 +68,14 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
                         float* step_out);
 
 int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
-                    const float* lo, const float* inv, const float* levels, uint64_t seed, uint8_t* plane1,
+                    const float* lo, const float* inv, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
                     uint8_t* plane2, int64_t row_bytes);
+int launch_code_weights(zipml_ctx* ctx, const zipml_dataset* d, const float* x, float* wtab, double* base);
+int launch_poly_rows(zipml_ctx* ctx, const zipml_dataset* d, const uint8_t* const* planes, int degree, const double* coef,
+                     const float* wtab, const double* base, const float* scale, double* rows_out);
+int plane_mean_chunks(const zipml_ctx* ctx, int64_t m);
+int launch_plane_mean(zipml_ctx* ctx, const zipml_dataset* d, const uint8_t* plane, const double* c, double* partial,
+                      float* g_out);
 
 int launch_histogram(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bins,
                      const float* lo, const float* inv, uint32_t* counts /* n x bins, zeroed here */);

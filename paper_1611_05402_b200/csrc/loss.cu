@@ -31,6 +31,14 @@ __global__ void loss_prepare_kernel(const float* __restrict__ lo, const float* _
     if (threadIdx.x == 0) *base_out = base;
 }
 
+// w = step * x (or level * x per code) and lo^T x for a data set's grid: shared by the loss and the polynomial estimator.
+int launch_code_weights(zipml_ctx* ctx, const zipml_dataset* d, const float* x, float* wtab, double* base) {
+    loss_prepare_kernel<<<1, 1024, 0, ctx->stream>>>(d->feat_lo, d->feat_step, d->levels, x, d->n, 1 << d->bits,
+                                                     d->level_mode == ZIPML_LEVELS_TABLE, wtab, base);
+    ++ctx->launches;
+    return cuda_status(cudaGetLastError());
+}
+
 template <int CB, bool TABLE>
 __global__ void __launch_bounds__(256) loss_codes_kernel(const uint32_t* __restrict__ p1, const uint32_t* __restrict__ p2,
                                                          int64_t row_words, int64_t m, int64_t n,

@@ -195,7 +195,7 @@ template <int CB, bool TABLE>
 __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__ A, int64_t m, int64_t n, int64_t lda,
                                                        int bits, const float* __restrict__ lo,
                                                        const float* __restrict__ inv, const float* __restrict__ levels,
-                                                       uint64_t seed, uint32_t* __restrict__ plane1,
+                                                       uint64_t seed, uint32_t draw, uint32_t* __restrict__ plane1,
                                                        uint32_t* __restrict__ plane2, int64_t row_words, bool vec_ok,
                                                        int passes) {
     constexpr int FPW = 32 / CB;
@@ -292,12 +292,12 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                 constexpr uint32_t kAllPairs = (1u << (FPW / 2)) - 1u;
                 if (__all_sync(__activemask(), need == kAllPairs)) {
     #pragma unroll
-                    for (int pr = 0; pr < FPW / 2; ++pr) apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr)));
+                    for (int pr = 0; pr < FPW / 2; ++pr) apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr), draw));
                 } else {
                     while (need) {
                         const int pr = __ffs(need) - 1;
                         need &= need - 1u;
-                        apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr)));
+                        apply(pr, sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr), draw));
                     }
                 }
         
@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
                     }
                     const bool random = (t[0] > 0u && t[0] < 16777216u) || (t[1] > 0u && t[1] < 16777216u);
                     Philox4 rnd;
-                    if (random) rnd = sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr));
+                    if (random) rnd = sample_block(seed, (uint64_t)row, (uint32_t)((j0 >> 1) + pr), draw);
                     else rnd.v[0] = rnd.v[1] = rnd.v[2] = rnd.v[3] = 0u;    // decided without them: 0 never up, 2^24 always up
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(const float* __restrict__
 }
 
 int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
-                    const float* lo, const float* inv, const float* levels, uint64_t seed, uint8_t* plane1,
+                    const float* lo, const float* inv, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
                     uint8_t* plane2, int64_t row_bytes) {
     const int cb = container_bits(bits);
     const int64_t row_words = row_bytes / 4;
@@ -367,7 +367,7 @@ int launch_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_
     uint32_t* p1 = reinterpret_cast<uint32_t*>(plane1);
     uint32_t* p2 = reinterpret_cast<uint32_t*>(plane2);
 #define ZIPML_LAUNCH_Q(CB_, T_) \
-    quantize_kernel<CB_, T_><<<grid, block, smem, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, p1, p2, row_words, vec_ok, passes)
+    quantize_kernel<CB_, T_><<<grid, block, smem, ctx->stream>>>(A, m, n, lda, bits, lo, inv, levels, seed, draw, p1, p2, row_words, vec_ok, passes)
     if (cb == 2) { if (table) ZIPML_LAUNCH_Q(2, true); else ZIPML_LAUNCH_Q(2, false); }
     else if (cb == 4) { if (table) ZIPML_LAUNCH_Q(4, true); else ZIPML_LAUNCH_Q(4, false); }
     else { ZIPML_LAUNCH_Q(8, false); }

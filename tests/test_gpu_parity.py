@@ -957,3 +957,45 @@ def test_row_sharded_epoch_matches_the_whole_epoch(ctx, world, case):
     tol = (20 if (mb or gb) else 1) * MODEL_TOL
     assert rel(xs[0], x_ref) <= tol
     assert rel(xs[0], whole.cpu().numpy()) <= 2 * tol
+
+
+@pytest.mark.parametrize("bits,mode", [(2, "uniform"), (4, "uniform"), (8, "uniform"), (3, "table")])
+def test_polynomial_estimator_over_independent_quantizations(ctx, bits, mode):
+    """Section 4.1 "Quantizing Polynomials" and Section 4.2's gradient: further draws of zipml_quantize_draw are
+    bit-exact against the oracle's (and differ from draw 0), Q(P) per sample and the weighted plane mean match the
+    oracle from the same planes."""
+    m, n, d = 1300, 333, 5
+    _, A, b, _ = workload("c4" if mode == "table" else "c1", m, n, seed=9)
+    dA = to_dev(A, ctx)
+    kw, okw = {}, {}
+    if mode == "table":
+        lev, _ = oracle.optimal_levels(A, bits, 256)
+        kw = dict(level_mode=binding.LEVELS_TABLE, levels=to_dev(lev, ctx))
+        okw = dict(mode=oracle.TABLE, levels=lev)
+    planes, oplanes, grid, ogrid = [], [], None, None
+    for q in range((d + 2) // 2):                                  # d planes for Q(P), one more for the gradient
+        ds = ctx.zipml_quantize(dA, bits, seed=5, draw=q, **kw)
+        ods = oracle.quantize_pair(A, bits, 5, q, **okw)
+        ctx.zipml_sync()
+        assert np.array_equal(ds.plane1.cpu().numpy(), ods.plane1) and np.array_equal(ds.plane2.cpu().numpy(), ods.plane2)
+        grid, ogrid = grid or ds, ogrid or ods
+        planes += [ds.plane1, ds.plane2]
+        oplanes += [ods.plane1, ods.plane2]
+    assert not np.array_equal(oplanes[0], oplanes[2])
+    x = (np.random.default_rng(2).standard_normal(n) * (0.3 / np.sqrt(n))).astype(np.float32)
+    coef = [0.5, 0.25, -0.125, 0.3, -0.2, 0.1]
+    labels = np.where(b > np.median(b), 1.0, -1.0).astype(np.float32)
+    for deg in (0, 1, 3, 5):
+        want = oracle.poly_rows(oplanes, ogrid, x, coef[:deg + 1], scale=labels)
+        got = ctx.zipml_poly_rows(grid, planes, coef[:deg + 1], to_dev(x, ctx), scale=to_dev(labels, ctx))
+        ctx.zipml_sync()
+        assert np.abs(got.cpu().numpy() - want).max() <= 1e-5 * max(1.0, np.abs(want).max()), deg
+    c = oracle.poly_rows(oplanes, ogrid, x, coef, scale=labels)
+    g_want = oracle.weighted_plane_mean(oplanes[d], ogrid, c)
+    g = ctx.zipml_weighted_plane_mean(grid, planes[d], torch.from_numpy(c).to(ctx.device))
+    ctx.zipml_sync()
+    assert rel(g.cpu().numpy(), g_want) <= GRAD_TOL
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_poly_rows(grid, planes * 2, [1.0] * 10, to_dev(x, ctx))          # degree 9 > ZIPML_POLY_MAX_DEGREE
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_poly_rows(grid, [planes[0].view(-1)[1:]], [0.0, 1.0], to_dev(x, ctx))     # a misaligned plane
