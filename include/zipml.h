@@ -17,7 +17,7 @@
  *
  * Packed sample layout ("plane"): row-major, `row_bytes` bytes per row, row_bytes a multiple of 16
  * and >= zipml_row_bytes(n, bits).  Feature j occupies cb bits at bit position j*cb of its row,
- * low bits first, where the container width cb is 2, 4, 4, 8 for bits = 2, 3, 4, 8.  Padding bits
+ * low bits first, where the container width cb is 2 for bits = 1, 2; 4 for bits = 3, 4; 8 for bits = 5 .. 8.  Padding bits
  * are zero.  A double-sampled dataset is two such planes (two independent quantizations of every
  * sample, Eq. (double) of the paper) plus what turns a code back into a value: per-feature
  * (lo_j, step_j) for a uniform grid, value = lo_j + code * step_j, or an n x 2^bits table of
@@ -35,7 +35,7 @@ extern "C" {
 enum {
     ZIPML_OK = 0,
     ZIPML_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, bad stride or alignment        */
-    ZIPML_ERR_UNSUPPORTED = -2, /* bits not in {2,3,4,8}, a level table with 8 bits, ...            */
+    ZIPML_ERR_UNSUPPORTED = -2, /* bits not in 1..8, a level table with more than 4 bits, ...   */
     ZIPML_ERR_NONFINITE = -3,   /* the sample matrix holds a NaN or an infinity (seen on device)   */
     ZIPML_ERR_CUDA = -4,        /* a CUDA runtime call failed (no device, out of memory, ...)       */
     ZIPML_ERR_TIMEOUT = -5,     /* a device-side wait gave up; the context stays usable            */
@@ -103,7 +103,7 @@ typedef struct zipml_ctx zipml_ctx;
 /* A double-sampled, bit-packed dataset in device memory. */
 typedef struct zipml_dataset {
     uint32_t struct_size;   /* sizeof(zipml_dataset), for ABI evolution                              */
-    int32_t bits;           /* 2, 3, 4 or 8                                                          */
+    int32_t bits;           /* 1 .. 8 (level tables: 1 .. 4)                                         */
     int32_t level_mode;     /* ZIPML_LEVELS_UNIFORM or ZIPML_LEVELS_TABLE                            */
     int32_t layout;         /* ZIPML_LAYOUT_ROWS, or ZIPML_LAYOUT_COLUMN_BLOCKS (zipml_sgd_epoch only)         */
     int64_t m, n;           /* samples, features                                                     */
@@ -125,7 +125,7 @@ typedef struct zipml_dataset {
  * Uniform grids only (value = lo_j + code * step_j). */
 typedef struct zipml_shared_base {
     uint32_t struct_size;   /* sizeof(zipml_shared_base)                                             */
-    int32_t bits;           /* 2, 3, 4 or 8                                                          */
+    int32_t bits;           /* 1 .. 8                                                                */
     int64_t m, n;
     int64_t row_bytes;      /* stride of the base plane                                              */
     int64_t up_row_bytes;   /* stride of the two up planes                                           */
@@ -229,10 +229,11 @@ int zipml_convert_layout(zipml_ctx* ctx, const zipml_dataset* data, int32_t to_l
 /* Stochastic quantization with double sampling (paper Section 2.1, Eq. (double); Supplement
  * "Randomized Quantization", "Column Scaling").
  *   A          m x n fp32, leading dimension lda >= n.
- *   bits       2, 3, 4 or 8: L = 2^bits levels, s = L-1 intervals.
+ *   bits       1 .. 8: L = 2^bits levels, s = L-1 intervals (the paper's operating points are 5-6 bits and below;
+ *              codes of 1, 3, 5, 6, 7 bits live in the next wider container).
  *   level_mode UNIFORM: levels lo_j + i*(hi_j-lo_j)/s on the feature's own range [lo_j, hi_j]
  *              (found by this call).  TABLE: `levels` (n x L ascending, levels[j][0] <= every value
- *              of feature j <= levels[j][L-1], e.g. from zipml_optimal_levels); bits = 8 unsupported.
+ *              of feature j <= levels[j][L-1], e.g. from zipml_optimal_levels); more than 4 bits unsupported.
  *   seed       each element (row k, feature j) is rounded twice, to the lower or upper neighbouring
  *              level with the probabilities that make the expectation equal to the value, using
  *              two 24-bit uniforms from Philox4x32-10 keyed by (seed, k, j, copy).

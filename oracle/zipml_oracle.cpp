@@ -107,7 +107,7 @@ uint32_t orc_u24_vector(uint64_t seed, uint32_t epoch, uint32_t step, uint32_t c
 // for bits = 2, 3, 4, 8 (3-bit codes sit in 4-bit containers).
 // ---------------------------------------------------------------------------------------------
 int orc_container_bits(int bits) {
-    switch (bits) { case 2: return 2; case 3: return 4; case 4: return 4; case 8: return 8; default: return 0; }
+    switch (bits) { case 1: case 2: return 2; case 3: case 4: return 4; case 5: case 6: case 7: case 8: return 8; default: return 0; }
 }
 
 int64_t orc_row_bytes(int64_t n, int bits) {
@@ -260,7 +260,7 @@ int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bit
                       int64_t row_bytes, float* feat_lo, float* feat_step) {
     const int cb = orc_container_bits(bits);
     if (cb == 0) return ORC_ERR_UNSUPPORTED;
-    if (level_mode == ORC_LEVELS_TABLE && bits == 8) return ORC_ERR_UNSUPPORTED;
+    if (level_mode == ORC_LEVELS_TABLE && bits > 4) return ORC_ERR_UNSUPPORTED;
     if (!A || !plane1 || !plane2 || !feat_lo || m <= 0 || n <= 0 || lda < n) return ORC_ERR_INVALID_ARG;
     if (row_bytes < orc_row_bytes(n, bits) || row_bytes % 16 != 0) return ORC_ERR_INVALID_ARG;
     if (level_mode == ORC_LEVELS_TABLE && !levels) return ORC_ERR_INVALID_ARG;
@@ -375,7 +375,7 @@ int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byte
     float reg_cst = 0.0f;
     if (reg == 1) reg_cst = (float)(1.0 / (1.0 + (double)lr * (double)reg_param));
     if (reg == 2 || reg == 4) reg_cst = (float)((double)lr * (double)reg_param);
-    if (level_mode == ORC_LEVELS_TABLE && bits == 8) return ORC_ERR_UNSUPPORTED;
+    if (level_mode == ORC_LEVELS_TABLE && bits > 4) return ORC_ERR_UNSUPPORTED;
     if (model_bits != 0 && (model_bits < 2 || model_bits > 8)) return ORC_ERR_UNSUPPORTED;
     if (grad_bits != 0 && (grad_bits < 2 || grad_bits > 8)) return ORC_ERR_UNSUPPORTED;
     if (!plane1 || !plane2 || !b || !x || m <= 0 || n <= 0 || batch <= 0) return ORC_ERR_INVALID_ARG;

@@ -47,7 +47,7 @@ int check_dataset(const zipml_dataset* d) {
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
     if (d->level_mode != ZIPML_LEVELS_UNIFORM && d->level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
     if (d->layout != ZIPML_LAYOUT_ROWS && d->layout != ZIPML_LAYOUT_COLUMN_BLOCKS) return ZIPML_ERR_INVALID_ARG;
-    if (d->level_mode == ZIPML_LEVELS_TABLE && d->bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (d->level_mode == ZIPML_LEVELS_TABLE && d->bits > 4) return ZIPML_ERR_UNSUPPORTED;
     if (d->m <= 0 || d->n <= 0) return ZIPML_ERR_INVALID_ARG;
     if (d->n > 0x7fffffffLL / 8) return ZIPML_ERR_WORKSPACE;
     if (!d->plane1 || !d->plane2 || !aligned16(d->plane1) || !aligned16(d->plane2)) return ZIPML_ERR_INVALID_ARG;
@@ -186,7 +186,7 @@ int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
     const int cb = container_bits(bits);
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
     if (level_mode != ZIPML_LEVELS_UNIFORM && level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
-    if (level_mode == ZIPML_LEVELS_TABLE && bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (level_mode == ZIPML_LEVELS_TABLE && bits > 4) return ZIPML_ERR_UNSUPPORTED;
     if (!A || !plane1 || !plane2 || !feat_lo || m <= 0 || n <= 0 || lda < n) return ZIPML_ERR_INVALID_ARG;
     if (level_mode == ZIPML_LEVELS_TABLE && !levels) return ZIPML_ERR_INVALID_ARG;
     if (level_mode == ZIPML_LEVELS_UNIFORM && !feat_step) return ZIPML_ERR_INVALID_ARG;
@@ -394,7 +394,7 @@ int zipml_train_host(zipml_ctx* ctx, const float* A_host, int64_t m, int64_t n, 
         return ZIPML_ERR_INVALID_ARG;
     const int64_t rb = zipml_row_bytes(n, bits);
     if (rb == 0) return ZIPML_ERR_UNSUPPORTED;
-    if (optimal_levels && bits == 8) return ZIPML_ERR_UNSUPPORTED;
+    if (optimal_levels && (bits < 2 || bits > 4)) return ZIPML_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
     const size_t L = (size_t)1 << bits;

@@ -20,7 +20,7 @@ __device__ __forceinline__ void set_status(DeviceStatus* st, int code, int detai
 }
 
 __host__ __device__ __forceinline__ int container_bits(int bits) {
-    return bits == 2 ? 2 : (bits == 3 || bits == 4) ? 4 : bits == 8 ? 8 : 0;
+    return (bits == 1 || bits == 2) ? 2 : (bits == 3 || bits == 4) ? 4 : (bits >= 5 && bits <= 8) ? 8 : 0;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -28,10 +28,10 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_host_only_helpers(lib):
-    for bits in (2, 3, 4, 8):
+    for bits in (1, 2, 3, 4, 5, 6, 7, 8):
         for n in (1, 7, 64, 1000, 2048, 32768):
             assert lib.zipml_row_bytes(n, bits) == oracle.row_bytes(n, bits)
-    assert lib.zipml_row_bytes(10, 5) == 0 and lib.zipml_row_bytes(0, 4) == 0
+    assert lib.zipml_row_bytes(10, 9) == 0 and lib.zipml_row_bytes(10, 0) == 0 and lib.zipml_row_bytes(0, 4) == 0
     assert lib.zipml_strerror(0) == b"ok"
     assert b"non-finite" in lib.zipml_strerror(binding.ERR_NONFINITE)
     assert C.sizeof(binding.CDataset) == 80 and C.sizeof(binding.CSgdParams) == 120

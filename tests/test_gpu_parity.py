@@ -121,7 +121,7 @@ def test_quantize_reports_bad_input(ctx):
         ctx.zipml_sync()
     assert e.value.code == binding.ERR_NONFINITE
     good = torch.rand((64, 16), device=ctx.device)
-    for bits in (1, 5, 16):
+    for bits in (0, 9, 16):
         with pytest.raises(binding.ZipmlError) as e:
             ctx.zipml_quantize(good, bits, seed=0)
         assert e.value.code == binding.ERR_UNSUPPORTED
@@ -999,3 +999,43 @@ def test_polynomial_estimator_over_independent_quantizations(ctx, bits, mode):
         ctx.zipml_poly_rows(grid, planes * 2, [1.0] * 10, to_dev(x, ctx))          # degree 9 > ZIPML_POLY_MAX_DEGREE
     with pytest.raises(binding.ZipmlError):
         ctx.zipml_poly_rows(grid, [planes[0].view(-1)[1:]], [0.0, 1.0], to_dev(x, ctx))     # a misaligned plane
+
+
+@pytest.mark.parametrize("bits", [1, 5, 6, 7])
+def test_bit_widths_in_wider_containers(ctx, bits):
+    """1-bit codes in 2-bit fields and 5- to 7-bit codes in bytes (the paper's operating points are 5-6 bits): planes
+    bit-exact, the code-plane loss, an epoch through AUTO on a small step and through the column and stream engines
+    on a large one."""
+    _, A, b, _ = workload("c2", 700, 200, seed=bits)
+    ods = oracle.quantize(A, bits, seed=4)
+    gds = ctx.zipml_quantize(to_dev(A, ctx), bits, seed=4)
+    ctx.zipml_sync()
+    assert np.array_equal(gds.plane1.cpu().numpy(), ods.plane1) and np.array_equal(gds.plane2.cpu().numpy(), ods.plane2)
+    assert np.array_equal(gds.feat_step.cpu().numpy(), ods.feat_step)
+    x0 = (np.random.default_rng(1).standard_normal(200) * 0.05).astype(np.float32)
+    loss = ctx.zipml_loss(binding.LOSS_CODES, to_dev(b, ctx), to_dev(x0, ctx), data=gds)
+    ctx.zipml_sync()
+    want = oracle.loss_codes(ods, b, x0)
+    assert abs(loss.item() - want) <= LOSS_TOL * abs(want)
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, to_dev(b, ctx), x, 64, 1e-3, model_bits=bits if bits > 1 else 0, grad_bits=0, seed=3)
+    ctx.zipml_sync()
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, 64, 1e-3, model_bits=bits if bits > 1 else 0, grad_bits=0, seed=3)
+    assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
+    # a large step: 300 rows of 16 KB (1-bit: 8 KB), B = 300 -> the column engine, and the stream engine beside it
+    n2 = 16384 if bits > 1 else 32768
+    _, A2, b2, _ = workload("c5", 300, n2, seed=bits)
+    ods2 = oracle.quantize(A2, bits, seed=6)
+    gds2 = dev_dataset(ods2, ctx)
+    x_ref2, _ = oracle.sgd_epoch(ods2, b2, np.zeros(n2, np.float32), 300, 1e-3)
+    for engine in (binding.ENGINE_COLUMN, binding.ENGINE_STREAM):
+        x2 = torch.zeros(n2, device=ctx.device)
+        ctx.zipml_sgd_epoch(gds2, to_dev(b2, ctx), x2, 300, 1e-3, engine=engine)
+        ctx.zipml_sync()
+        assert rel(x2.cpu().numpy(), x_ref2) <= MODEL_TOL, engine
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_quantize(to_dev(A, ctx), 9, seed=0)
+    if bits > 4:
+        with pytest.raises(binding.ZipmlError):
+            ctx.zipml_quantize(to_dev(A, ctx), bits, seed=0, level_mode=binding.LEVELS_TABLE,
+                               levels=torch.zeros((200, 1 << bits), device=ctx.device))

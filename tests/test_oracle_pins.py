@@ -178,7 +178,7 @@ def test_quantize_edge_cases():
     with pytest.raises(oracle.OracleError) as e:
         oracle.quantize(bad, 4, seed=0)
     assert e.value.code == oracle.ERR_NONFINITE
-    for bits in (1, 5, 16):
+    for bits in (0, 9, 16):
         with pytest.raises(oracle.OracleError):
             oracle.quantize(A, bits, seed=0)
     with pytest.raises(oracle.OracleError):
@@ -493,3 +493,28 @@ def test_regulariser_arguments():
         oracle.sgd_epoch(ds, b, np.zeros(n, np.float32), batch=m, lr=0.1, reg=7)
     with pytest.raises(Exception):
         oracle.sgd_epoch(ds, b, np.zeros(n, np.float32), batch=m, lr=0.1, reg=oracle.REG_L1, reg_param=-1.0)
+
+
+@pytest.mark.parametrize("bits", [1, 5, 6, 7])
+def test_the_other_bit_widths_live_in_the_next_wider_container(bits):
+    """1-bit codes in 2-bit fields, 5- to 7-bit codes in bytes: same quantizer (Supplement "Randomized Quantization")
+    with s = 2^bits - 1 intervals; pinned by exact samples, the code range, and the unbiased mean."""
+    s = (1 << bits) - 1
+    cb = {1: 2, 5: 8, 6: 8, 7: 8}[bits]
+    assert oracle.container_bits(bits) == cb and oracle.row_bytes(33, bits) == (33 * cb + 7) // 8 + (-((33 * cb + 7) // 8)) % 16
+    rng = np.random.default_rng(bits)
+    A = rng.integers(0, s + 1, size=(20, 9)).astype(np.float32)
+    A[0], A[1] = 0.0, float(s)
+    ds = oracle.quantize(A, bits, seed=1)
+    for plane in (ds.plane1, ds.plane2):                             # samples on the grid: the codes are the samples
+        assert np.array_equal(oracle.unpack_plane(plane, 9, bits), A.astype(np.int64))
+    B = rng.uniform(-1.0, 1.0, (4, 6)).astype(np.float32)
+    B[0], B[1] = -1.0, 1.0
+    acc, N = np.zeros((4, 6)), 3000
+    for seed in range(N):
+        d = oracle.quantize(B, bits, seed=seed)
+        c = oracle.unpack_plane(d.plane1, 6, bits)
+        assert c.max() <= s and c.min() >= 0
+        acc += d.feat_lo + d.feat_step * c
+    step = 2.0 / s
+    assert np.abs(acc / N - B).max() < 5 * (step / 2) / np.sqrt(N) + 1e-6
