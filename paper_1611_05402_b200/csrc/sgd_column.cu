@@ -124,7 +124,6 @@ struct ColShared {
     unsigned long long full_b[kColMaxSlots], empty_b[kColMaxSlots];     // B ring: copies landed / the B warps are done
     unsigned long long rfull[kColRWarps], rempty[kColRWarps];   // residual digits of a chunk (one buffer per R warp): written / consumed
     int w_version;                             // steps (+1) whose digits of w are in place
-    unsigned long long wbar;                   // one arrival per publication of w: lets the A warps sleep until the next one
     ColStepParams sp[2];
     double red_d[2][32];
     float red_f[2][32];
@@ -198,13 +197,11 @@ __device__ __forceinline__ int ld_acquire_cta(const int* p) {
 }
 
 // Bounded wait until a version count in shared memory has reached `want`.
-// (The count decides; the barrier only parks the warp until the publication it is waiting for, or for a microsecond:
-// a warp without a task in some step may be phases behind, where a parity alone would be ambiguous.)
 __device__ __noinline__ bool col_wait_version(const int* version, int want, ColShared* sh, DeviceStatus* status, int where) {
     const long long t0 = clock64();
 #pragma unroll 1
     for (int spin = 0; ld_acquire_cta(version) < want; ++spin) {
-        mbar_try_wait_parked(&sh->wbar, (uint32_t)((want - 1) & 1));
+        __nanosleep(100);
         if ((spin & 15) == 15) {
             if (col_aborted(sh)) return false;
             if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(status, ZIPML_ERR_TIMEOUT, where); return false; }
@@ -310,7 +307,6 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             mbar_init(reinterpret_cast<uint64_t*>(sh->rempty + s), kColBWarps);
         }
         sh->w_version = 0;
-        mbar_init(reinterpret_cast<uint64_t*>(&sh->wbar), 1);
         sh->abort_flag = 0;
         sh->qa_issued = 0;
         mbar_fence_init();
@@ -577,10 +573,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     }
                 }
                 named_barrier(kColNamedB, kColBThreads);     // every digit is written (also: red_* may be reused)
-                if (btid == 0) {
-                    st_release_cta(&sh->w_version, t_rel + 1);
-                    mbar_arrive(reinterpret_cast<uint64_t*>(&sh->wbar));
-                }
+                if (btid == 0) st_release_cta(&sh->w_version, t_rel + 1);
                 if (t_rel > 0 && p == 0 && lane == 0) col_mark(a, t_rel - 1, 7);
             }
             int acc2[2][NG][4];                                  // two sets, for alternate 32-row blocks: shorter dependency chains
