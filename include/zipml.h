@@ -296,9 +296,12 @@ int zipml_sgd_epoch_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, c
 
 /* Polynomials of a^T x over several independent quantizations (paper Section 4.1 "Quantizing Polynomials"; Section 4.2
  * uses them for smooth classification losses).  ZIPML_POLY_MAX_DEGREE bounds the degree d.
- * zipml_quantize_draw: zipml_quantize with a draw index: draw q gives the quantizations Q_{2q+1}, Q_{2q+2} of the same
- *   samples on the same grid, independent of every other draw (the Philox counter's last word is q; draw 0 is
- *   zipml_quantize itself).  d quantizations take ceil(d / 2) calls with the same seed.
+ * zipml_quantize_draw: zipml_quantize with a draw index and a choice of grid.  Draw q gives the quantizations Q_{2q+1},
+ *   Q_{2q+2} of the same samples on the same grid, independent of every other draw (the Philox counter's last word is
+ *   q; draw 0 with ZIPML_GRID_RANGE is zipml_quantize itself); d quantizations take ceil(d / 2) calls with the same
+ *   seed.  grid: ZIPML_GRID_RANGE, the feature's own range [min_j, max_j]; ZIPML_GRID_SYMMETRIC (uniform levels
+ *   only), the paper's [-M_j, M_j] with M_j = max |value| of the feature (Supplement "Column Scaling"): feat_lo is
+ *   then -M_j and feat_step 2 M_j / s.
  * zipml_poly_rows: rows_out[k] (m doubles, device memory) = Q(P)_k = sum_{i=0..d} coef[i] * prod_{j<=i} Q_j(a_k)^T x,
  *   times scale[k] where scale (m floats, device memory, e.g. the labels) is not NULL.  `grid` gives bits, level mode,
  *   m, n, row_bytes and feat_lo / feat_step / levels (its plane pointers are checked like any data set's but not
@@ -311,8 +314,9 @@ int zipml_sgd_epoch_shared_base(zipml_ctx* ctx, const zipml_shared_base* data, c
  * Errors: ZIPML_ERR_INVALID_ARG (null or misaligned pointers, degree out of range, a bad `grid`), ZIPML_ERR_UNSUPPORTED
  * (layout other than ZIPML_LAYOUT_ROWS); nothing is launched then. */
 #define ZIPML_POLY_MAX_DEGREE 8
+enum { ZIPML_GRID_RANGE = 0, ZIPML_GRID_SYMMETRIC = 1 };
 int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
-                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
+                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, int32_t grid, uint8_t* plane1,
                         uint8_t* plane2, int64_t row_bytes, float* feat_lo, float* feat_step);
 int zipml_poly_rows(zipml_ctx* ctx, const zipml_dataset* grid, const uint8_t* const* planes, int32_t degree,
                     const double* coef, const float* x, const float* scale, double* rows_out);

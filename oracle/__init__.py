@@ -52,7 +52,7 @@ def _declare(L):
     L.orc_shared_base_decode.argtypes = [vp, vp, vp, i64, i64, i64, i64, i32, vp, vp]
     L.orc_column_range.argtypes = [vp, i64, i64, i64, vp, vp]
     L.orc_quantize.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
-    L.orc_quantize_pair.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, C.c_uint32, vp, vp, i64, vp, vp]
+    L.orc_quantize_pair.argtypes = [vp, i64, i64, i64, i32, i32, vp, u64, C.c_uint32, i32, vp, vp, i64, vp, vp]
     L.orc_poly_rows.argtypes = [vp, i32, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     L.orc_weighted_plane_mean.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp]
     L.orc_dequantize_row.argtypes = [vp, i64, i32, i32, vp, vp, vp, vp]
@@ -199,7 +199,7 @@ def quantize(A, bits, seed, mode=UNIFORM, levels=None):
     return Dataset(p1, p2, m, n, bits, mode, lo, step, levels)
 
 
-def quantize_pair(A, bits, seed, pair, mode=UNIFORM, levels=None):
+def quantize_pair(A, bits, seed, pair, mode=UNIFORM, levels=None, symmetric=False):
     """Pair `pair` of independent quantizations of A on the grid of quantize(): planes 2 pair + 1, 2 pair + 2 of
     Q_1, Q_2, ... (Section 4.1); pair 0 is quantize()."""
     A = np.ascontiguousarray(A, dtype=np.float32)
@@ -210,7 +210,8 @@ def quantize_pair(A, bits, seed, pair, mode=UNIFORM, levels=None):
     step = np.zeros(n, np.float32) if mode == UNIFORM else None
     if levels is not None:
         levels = np.ascontiguousarray(levels, dtype=np.float32)
-    _check(lib().orc_quantize_pair(_p(A), m, n, n, bits, mode, _p(levels), seed, pair, _p(p1), _p(p2), rb, _p(lo), _p(step)))
+    _check(lib().orc_quantize_pair(_p(A), m, n, n, bits, mode, _p(levels), seed, pair, int(symmetric), _p(p1), _p(p2), rb, _p(lo),
+                                   _p(step)))
     return Dataset(p1, p2, m, n, bits, mode, lo, step, levels)
 
 

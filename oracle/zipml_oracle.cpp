@@ -245,19 +245,21 @@ static inline void table_cell(float v, const float* lev, int s, uint32_t* cell, 
 // Out: plane1, plane2 (m * row_bytes each), feat_lo (n), feat_step (n; uniform grid only: (hi-lo)/s).
 // For ORC_LEVELS_TABLE `levels` is n x L ascending fp32 with levels[j][0] <= every value <= levels[j][s].
 int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
-                      const float* levels, uint64_t seed, uint32_t pair, uint8_t* plane1, uint8_t* plane2,
+                      const float* levels, uint64_t seed, uint32_t pair, int symmetric, uint8_t* plane1, uint8_t* plane2,
                       int64_t row_bytes, float* feat_lo, float* feat_step);
 int orc_quantize(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
                  const float* levels, uint64_t seed, uint8_t* plane1, uint8_t* plane2,
                  int64_t row_bytes, float* feat_lo, float* feat_step) {
-    return orc_quantize_pair(A, m, n, lda, bits, level_mode, levels, seed, 0u, plane1, plane2, row_bytes, feat_lo, feat_step);
+    return orc_quantize_pair(A, m, n, lda, bits, level_mode, levels, seed, 0u, 0, plane1, plane2, row_bytes, feat_lo, feat_step);
 }
 
 // Pair `pair` of quantizations of the same samples on the same grid: planes 2 pair + 1 and 2 pair + 2 of the
-// sequence Q_1, Q_2, ... (pair 0 is orc_quantize).
+// sequence Q_1, Q_2, ... (pair 0 is orc_quantize).  symmetric != 0 (uniform levels only): the grid of the Supplement's
+// "Column Scaling", [-M_j, M_j] with M_j the feature's largest |value|, instead of the feature's own range.
 int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bits, int level_mode,
-                      const float* levels, uint64_t seed, uint32_t pair, uint8_t* plane1, uint8_t* plane2,
+                      const float* levels, uint64_t seed, uint32_t pair, int symmetric, uint8_t* plane1, uint8_t* plane2,
                       int64_t row_bytes, float* feat_lo, float* feat_step) {
+    if (symmetric && level_mode != ORC_LEVELS_UNIFORM) return ORC_ERR_INVALID_ARG;
     const int cb = orc_container_bits(bits);
     if (cb == 0) return ORC_ERR_UNSUPPORTED;
     if (level_mode == ORC_LEVELS_TABLE && bits > 4) return ORC_ERR_UNSUPPORTED;
@@ -271,6 +273,10 @@ int orc_quantize_pair(const float* A, int64_t m, int64_t n, int64_t lda, int bit
     const int rc = orc_column_range(A, m, n, lda, lo.data(), hi.data());
     if (rc != ORC_OK) return rc;
     for (int64_t j = 0; j < n; ++j) {
+        if (symmetric) {
+            hi[j] = std::fmax(std::fabs(lo[j]), std::fabs(hi[j]));
+            lo[j] = -hi[j];
+        }
         feat_lo[j] = lo[j];
         const float range = hi[j] - lo[j];
         inv[j] = (range > 0.0f) ? (float)s / range : 0.0f;

@@ -14,6 +14,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NONFINITE, ERR_CUDA, ERR_TIMEOUT, ERR_WORK
 LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
 LAYOUT_ROWS, LAYOUT_COLUMN_BLOCKS = 0, 1
+GRID_RANGE, GRID_SYMMETRIC = 0, 1
 REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM, ENGINE_COLUMN = 0, 1, 2, 3, 4, 5, 6, 7
 
@@ -91,7 +92,8 @@ def lib():
         L.zipml_loss_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, vp]
         L.zipml_sgd_epoch_shared_base.argtypes = [vp, C.POINTER(CSharedBase), vp, vp, C.POINTER(CSgdParams), vp]
         L.zipml_sgd_apply_gradient.argtypes = [vp, vp, vp, C.c_int64, C.POINTER(CSgdParams), C.c_int64, vp]
-        L.zipml_quantize_draw.argtypes = [vp, vp, i64, i64, i64, C.c_int32, C.c_int32, vp, C.c_uint64, C.c_uint32, vp, vp, i64, vp, vp]
+        L.zipml_quantize_draw.argtypes = [vp, vp, i64, i64, i64, C.c_int32, C.c_int32, vp, C.c_uint64, C.c_uint32, C.c_int32, vp, vp, i64,
+                                          vp, vp]
         L.zipml_poly_rows.argtypes = [vp, C.POINTER(CDataset), vp, C.c_int32, vp, vp, vp, vp]
         L.zipml_weighted_plane_mean.argtypes = [vp, C.POINTER(CDataset), vp, vp, vp]
         L.zipml_quantize.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, u64, vp, vp, i64, vp, vp]
@@ -226,7 +228,7 @@ class Context:
         """Enqueues a bounded wait that must give up; the next zipml_sync raises ZipmlError(ERR_TIMEOUT)."""
         _check(lib().zipml_wait_probe(self._h, spin_limit), "zipml_wait_probe")
 
-    def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None, draw=0):
+    def zipml_quantize(self, A, bits, seed, level_mode=LEVELS_UNIFORM, levels=None, row_bytes=None, draw=0, grid=0):
         """Two packed quantizations of A; draw > 0: further independent pairs on the same grid (zipml_quantize_draw)."""
         m, n = A.shape
         assert A.stride(1) == 1 and A.dtype == torch.float32 and A.device == self.device
@@ -237,9 +239,9 @@ class Context:
         p2 = torch.empty((m, rb), dtype=torch.uint8, device=self.device)
         lo = torch.empty(n, dtype=torch.float32, device=self.device)
         step = torch.empty(n, dtype=torch.float32, device=self.device) if level_mode == LEVELS_UNIFORM else None
-        if draw:
+        if draw or grid:
             _check(lib().zipml_quantize_draw(self._h, C.c_void_p(A.data_ptr()), m, n, A.stride(0), bits, level_mode,
-                                             _ptr(levels, torch.float32, self.device), seed, draw, _ptr(p1), _ptr(p2), rb,
+                                             _ptr(levels, torch.float32, self.device), seed, draw, grid, _ptr(p1), _ptr(p2), rb,
                                              _ptr(lo), _ptr(step)), "zipml_quantize_draw")
         else:
             _check(lib().zipml_quantize(self._h, C.c_void_p(A.data_ptr()), m, n, A.stride(0), bits, level_mode,

@@ -176,13 +176,16 @@ int zipml_sync(zipml_ctx* ctx) {
 int zipml_quantize(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
                    int32_t level_mode, const float* levels, uint64_t seed, uint8_t* plane1, uint8_t* plane2,
                    int64_t row_bytes, float* feat_lo, float* feat_step) {
-    return zipml_quantize_draw(ctx, A, m, n, lda, bits, level_mode, levels, seed, 0u, plane1, plane2, row_bytes, feat_lo, feat_step);
+    return zipml_quantize_draw(ctx, A, m, n, lda, bits, level_mode, levels, seed, 0u, ZIPML_GRID_RANGE, plane1, plane2, row_bytes, feat_lo,
+                               feat_step);
 }
 
 int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int32_t bits,
-                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, uint8_t* plane1,
+                        int32_t level_mode, const float* levels, uint64_t seed, uint32_t draw, int32_t grid, uint8_t* plane1,
                         uint8_t* plane2, int64_t row_bytes, float* feat_lo, float* feat_step) {
     if (!ctx) return ZIPML_ERR_INVALID_ARG;
+    if (grid != ZIPML_GRID_RANGE && grid != ZIPML_GRID_SYMMETRIC) return ZIPML_ERR_INVALID_ARG;
+    if (grid == ZIPML_GRID_SYMMETRIC && level_mode != ZIPML_LEVELS_UNIFORM) return ZIPML_ERR_INVALID_ARG;
     const int cb = container_bits(bits);
     if (cb == 0) return ZIPML_ERR_UNSUPPORTED;
     if (level_mode != ZIPML_LEVELS_UNIFORM && level_mode != ZIPML_LEVELS_TABLE) return ZIPML_ERR_INVALID_ARG;
@@ -201,7 +204,8 @@ int zipml_quantize_draw(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
     uint32_t* keys = cv.take<uint32_t>(2 * (size_t)n);
     float* inv = cv.take<float>((size_t)n);
     float* step_tmp = cv.take<float>((size_t)n);
-    rc = launch_column_range(ctx, A, m, n, lda, s, keys, feat_lo, nullptr, inv, feat_step ? feat_step : step_tmp);
+    rc = launch_column_range(ctx, A, m, n, lda, s, grid == ZIPML_GRID_SYMMETRIC, keys, feat_lo, nullptr, inv,
+                             feat_step ? feat_step : step_tmp);
     if (rc != ZIPML_OK) return rc;
     return launch_quantize(ctx, A, m, n, lda, bits, level_mode, feat_lo, inv, levels, seed, draw, plane1, plane2, row_bytes);
 }
@@ -224,7 +228,7 @@ int zipml_optimal_levels(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, i
     float* hi = cv.take<float>((size_t)n);
     float* inv = cv.take<float>((size_t)n);
     uint32_t* counts = cv.take<uint32_t>((size_t)n * hist_bins);
-    rc = launch_column_range(ctx, A, m, n, lda, hist_bins, keys, lo, hi, inv, nullptr);
+    rc = launch_column_range(ctx, A, m, n, lda, hist_bins, false, keys, lo, hi, inv, nullptr);
     if (rc != ZIPML_OK) return rc;
     rc = launch_histogram(ctx, A, m, n, lda, hist_bins, lo, inv, counts);
     if (rc != ZIPML_OK) return rc;

@@ -63,7 +63,7 @@ inline size_t carve_size(size_t bytes) { return (bytes + 255) / 256 * 256; }
 // Launchers (each enqueues on ctx->stream and returns a status) -------------------------------
 // Column range: lo/hi per feature, inv = s/(hi-lo) and step = (hi-lo)/s for a grid of s intervals.
 // Any of hi_out, inv_out, step_out may be null.  Sets NONFINITE in the device status.
-int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int s,
+int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int s, bool symmetric,
                         uint32_t* key_scratch /* 2n */, float* lo_out, float* hi_out, float* inv_out,
                         float* step_out);
 

@@ -123,11 +123,15 @@ __global__ void __launch_bounds__(256) range_scan_wide_kernel(const float* __res
         }
 }
 
-__global__ void range_finalize_kernel(const uint32_t* lo_key, const uint32_t* hi_key, int64_t n, int s,
+__global__ void range_finalize_kernel(const uint32_t* lo_key, const uint32_t* hi_key, int64_t n, int s, bool symmetric,
                                       float* lo_out, float* hi_out, float* inv_out, float* step_out) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n) return;
-    const float lo = float_from_order_key(lo_key[j]), hi = float_from_order_key(hi_key[j]);
+    float lo = float_from_order_key(lo_key[j]), hi = float_from_order_key(hi_key[j]);
+    if (symmetric) {                     // the grid [-M_j, M_j], M_j = max |value| (Supplement "Column Scaling")
+        hi = fmaxf(fabsf(lo), fabsf(hi));
+        lo = -hi;
+    }
     const float range = __fsub_rn(hi, lo);
     lo_out[j] = lo;
     if (hi_out) hi_out[j] = hi;
@@ -135,7 +139,7 @@ __global__ void range_finalize_kernel(const uint32_t* lo_key, const uint32_t* hi
     if (step_out) step_out[j] = __fdiv_rn(range, (float)s);
 }
 
-int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int s,
+int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, int64_t lda, int s, bool symmetric,
                         uint32_t* key_scratch, float* lo_out, float* hi_out, float* inv_out, float* step_out) {
     uint32_t* lo_key = key_scratch;
     uint32_t* hi_key = key_scratch + n;
@@ -152,7 +156,7 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
         if (chunks > 65535) { rows_per_block = (m + 65534) / 65535; chunks = (m + rows_per_block - 1) / rows_per_block; }
         range_scan_wide_kernel<<<dim3((unsigned)col_tiles, (unsigned)chunks), 256, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key,
                                                                                                    hi_key, ctx->d_status);
-        range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, lo_out, hi_out, inv_out, step_out);
+        range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, symmetric, lo_out, hi_out, inv_out, step_out);
         ctx->launches += 3;
         return cuda_status(cudaGetLastError());
     }
@@ -168,7 +172,7 @@ int launch_column_range(zipml_ctx* ctx, const float* A, int64_t m, int64_t n, in
     const dim3 grid((unsigned)col_tiles, (unsigned)chunks), block(32, 8);
     if (vec) range_scan_kernel<4><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key, hi_key, ctx->d_status);
     else range_scan_kernel<1><<<grid, block, 0, ctx->stream>>>(A, m, n, lda, rows_per_block, lo_key, hi_key, ctx->d_status);
-    range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, lo_out, hi_out, inv_out, step_out);
+    range_finalize_kernel<<<nb, 256, 0, ctx->stream>>>(lo_key, hi_key, n, s, symmetric, lo_out, hi_out, inv_out, step_out);
     ctx->launches += 3;
     return cuda_status(cudaGetLastError());
 }

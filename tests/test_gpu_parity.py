@@ -1039,3 +1039,27 @@ def test_bit_widths_in_wider_containers(ctx, bits):
         with pytest.raises(binding.ZipmlError):
             ctx.zipml_quantize(to_dev(A, ctx), bits, seed=0, level_mode=binding.LEVELS_TABLE,
                                levels=torch.zeros((200, 1 << bits), device=ctx.device))
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_symmetric_grid(ctx, bits):
+    """ZIPML_GRID_SYMMETRIC (Supplement "Column Scaling": levels on [-M_j, M_j]): planes, lo and step bit-exact against
+    the oracle, and an epoch on such data."""
+    _, A, b, _ = workload("c2", 900, 260, seed=bits)
+    A = (A + 0.3).astype(np.float32)                          # ranges that are not symmetric by themselves
+    ods = oracle.quantize_pair(A, bits, 7, 0, symmetric=True)
+    gds = ctx.zipml_quantize(to_dev(A, ctx), bits, seed=7, grid=binding.GRID_SYMMETRIC)
+    ctx.zipml_sync()
+    assert np.array_equal(gds.plane1.cpu().numpy(), ods.plane1) and np.array_equal(gds.plane2.cpu().numpy(), ods.plane2)
+    assert np.array_equal(gds.feat_lo.cpu().numpy(), ods.feat_lo) and np.array_equal(gds.feat_step.cpu().numpy(), ods.feat_step)
+    assert np.array_equal(ods.feat_lo, -np.abs(A).max(axis=0))
+    x = torch.zeros(260, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, to_dev(b, ctx), x, 128, 1e-3)
+    ctx.zipml_sync()
+    x_ref, _ = oracle.sgd_epoch(ods, b, np.zeros(260, np.float32), 128, 1e-3)
+    assert rel(x.cpu().numpy(), x_ref) <= MODEL_TOL
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_quantize(to_dev(A, ctx), 3, seed=0, grid=binding.GRID_SYMMETRIC, level_mode=binding.LEVELS_TABLE,
+                           levels=torch.zeros((260, 8), device=ctx.device))
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_quantize(to_dev(A, ctx), bits, seed=0, grid=2)

@@ -518,3 +518,28 @@ def test_the_other_bit_widths_live_in_the_next_wider_container(bits):
         acc += d.feat_lo + d.feat_step * c
     step = 2.0 / s
     assert np.abs(acc / N - B).max() < 5 * (step / 2) / np.sqrt(N) + 1e-6
+
+
+def test_symmetric_grid_of_the_supplements_column_scaling():
+    """Grid [-M_j, M_j] with M_j = max |value| (Supplement "Column Scaling"): lo = -M, step = 2M/s, samples on the
+    grid come back exactly, the mean over seeds is the sample, and the codes differ from the range grid's."""
+    rng = np.random.default_rng(11)
+    bits, s = 3, 7
+    A = rng.uniform(-0.4, 1.0, (12, 5)).astype(np.float32)
+    M = np.abs(A).max(axis=0)
+    ds = oracle.quantize_pair(A, bits, 3, 0, symmetric=True)
+    assert np.array_equal(ds.feat_lo, -M) and np.allclose(ds.feat_step, 2 * M / s, rtol=1e-7)
+    assert not np.array_equal(ds.plane1, oracle.quantize(A, bits, 3).plane1)
+    # exact samples: integers -7, -5, ..., 7 are the eight levels of M = 7
+    G = (2 * rng.integers(0, s + 1, size=(16, 4)) - s).astype(np.float32)
+    G[0] = -7.0
+    dg = oracle.quantize_pair(G, bits, 5, 1, symmetric=True)
+    for plane in (dg.plane1, dg.plane2):
+        assert np.array_equal(-7.0 + 2.0 * oracle.unpack_plane(plane, 4, bits), G)
+    acc, N = np.zeros(A.shape), 4000
+    for seed in range(N):
+        d = oracle.quantize_pair(A, bits, seed, 0, symmetric=True)
+        acc += d.feat_lo + d.feat_step * oracle.unpack_plane(d.plane2, 5, bits)
+    assert np.abs(acc / N - A).max() < 5 * (2 * M.max() / s / 2) / np.sqrt(N) + 1e-6
+    with pytest.raises(oracle.OracleError):
+        oracle.quantize_pair(A, bits, 0, 0, mode=oracle.TABLE, levels=np.zeros((5, 8), np.float32), symmetric=True)
