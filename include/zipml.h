@@ -137,6 +137,8 @@ typedef struct zipml_shared_base {
 } zipml_shared_base;
 
 /* Parameters of one zipml_sgd_epoch call. */
+enum { ZIPML_NORM_L2 = 0, ZIPML_NORM_LINF = 1 };
+
 typedef struct zipml_sgd_params {
     uint32_t struct_size;       /* sizeof(zipml_sgd_params)                                          */
     int32_t model_bits;         /* 0: gradients see the fp32 model; 2..8: see Q3(x), redrawn per step */
@@ -186,7 +188,11 @@ typedef struct zipml_sgd_params {
     int32_t column_chunk_rows;  /* tuning, column engine: 0 = automatic, else rows of a minibatch that
                                    travel through shared memory together (a multiple of 32; values
                                    above 128 count as 128)                                            */
-    int32_t reserved0;          /* must be 0                                                         */
+    int32_t vector_norm;        /* scale M(v) of Q3 and Q4 (Supplement Eq. (quant2) leaves it general):
+                                   ZIPML_NORM_L2 = ||v||_2, the paper's choice and the default;
+                                   ZIPML_NORM_LINF = max |v_i| (lower variance; the largest entry is exact).
+                                   With LINF and model_bits or grad_bits set only the first-generation
+                                   engine runs (AUTO picks it; the others answer ZIPML_ERR_UNSUPPORTED) */
 } zipml_sgd_params;
 
 /* Context: binds a device, a stream (a cudaStream_t passed as void*, NULL = the legacy default

@@ -59,8 +59,10 @@ def _declare(L):
     L.orc_dequantize_row.restype = None
     L.orc_quantize_vector.argtypes = [vp, i64, i32, u64, u32, u32, u32, vp, vp]
     L.orc_quantize_vector.restype = None
+    L.orc_quantize_vector_norm.argtypes = [vp, i64, i32, u64, u32, u32, u32, i32, vp, vp]
+    L.orc_quantize_vector_norm.restype = None
     L.orc_sgd_epoch.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, i64, f32, i32, i32,
-                                u64, i64, i64, i64, vp, vp, i32, f32]
+                                u64, i64, i64, i64, vp, vp, i32, f32, i32]
     L.orc_estimator_mean.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, i32, vp]
     L.orc_loss_dense.argtypes = [vp, i64, i64, i64, vp, vp, vp]
     L.orc_loss_codes.argtypes = [vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -241,11 +243,14 @@ def weighted_plane_mean(plane, ds, c):
     return g
 
 
-def quantize_vector(v, bits, seed, epoch, step, stream):
+NORM_L2, NORM_LINF = 0, 1
+
+
+def quantize_vector(v, bits, seed, epoch, step, stream, norm=NORM_L2):
     v = np.ascontiguousarray(v, dtype=np.float32)
     out = np.zeros_like(v)
     codes = np.zeros(v.shape[0], np.int32)
-    lib().orc_quantize_vector(_p(v), v.shape[0], bits, seed, epoch, step, stream, _p(out), _p(codes))
+    lib().orc_quantize_vector_norm(_p(v), v.shape[0], bits, seed, epoch, step, stream, norm, _p(out), _p(codes))
     return out, codes
 
 
@@ -253,7 +258,7 @@ REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 
 
 def sgd_epoch(ds, b, x, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=None,
-              batch_order=None, want_grad=False, reg=REG_NONE, reg_param=0.0):
+              batch_order=None, want_grad=False, reg=REG_NONE, reg_param=0.0, vector_norm=NORM_L2):
     """Runs steps in place on a copy of x; returns (x_new, grad(2, n) or None)."""
     b = np.ascontiguousarray(b, dtype=np.float32)
     x = np.array(x, dtype=np.float32, copy=True)
@@ -266,7 +271,7 @@ def sgd_epoch(ds, b, x, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, f
     _check(lib().orc_sgd_epoch(_p(ds.plane1), _p(ds.plane2), ds.row_bytes, ds.m, ds.n, ds.bits, ds.mode,
                                _p(ds.feat_lo), _p(ds.feat_step), _p(ds.levels), _p(b), _p(x), batch, lr,
                                model_bits, grad_bits, seed, epoch, first_step, num_steps, _p(batch_order), _p(g),
-                               int(reg), C.c_float(reg_param)))
+                               int(reg), C.c_float(reg_param), int(vector_norm)))
     return x, g
 
 

@@ -319,12 +319,26 @@ void orc_dequantize_row(const uint8_t* row, int64_t n, int bits, int level_mode,
 // M = (float) sqrt(sum in double of v_i^2); a = |v_i| / M; t = a * s_m; l = min(floor(t), s_m-1);
 // p = t - l; Q_i = sgn(v_i) * M * ((l + up) / s_m), each op rounded to fp32.  Q(0) = 0.
 // ---------------------------------------------------------------------------------------------
+void orc_quantize_vector_norm(const float* v, int64_t n, int bits, uint64_t seed, uint32_t epoch, uint32_t step,
+                              uint32_t stream, int norm, float* out, int32_t* codes_out_or_null);
 void orc_quantize_vector(const float* v, int64_t n, int bits, uint64_t seed, uint32_t epoch,
                          uint32_t step, uint32_t stream, float* out, int32_t* codes_out_or_null) {
+    orc_quantize_vector_norm(v, n, bits, seed, epoch, step, stream, 0, out, codes_out_or_null);
+}
+
+// The scaling function M(v) of Eq. (quant2) is left general by the Supplement ("Randomized Quantization"): norm 0 is
+// the paper's choice ||v||_2, norm 1 is max |v_i| (every |v_i| / M still lies in [0, 1]; the largest entry is exact).
+void orc_quantize_vector_norm(const float* v, int64_t n, int bits, uint64_t seed, uint32_t epoch, uint32_t step,
+                              uint32_t stream, int norm, float* out, int32_t* codes_out_or_null) {
     const int sm = (1 << (bits - 1)) - 1;
-    double ss = 0.0;
-    for (int64_t i = 0; i < n; ++i) ss += (double)v[i] * (double)v[i];
-    const float M = (float)std::sqrt(ss);
+    float M = 0.0f;
+    if (norm == 1) {
+        for (int64_t i = 0; i < n; ++i) M = fmaxf(M, fabsf(v[i]));
+    } else {
+        double ss = 0.0;
+        for (int64_t i = 0; i < n; ++i) ss += (double)v[i] * (double)v[i];
+        M = (float)std::sqrt(ss);
+    }
     for (int64_t i = 0; i < n; ++i) {
         if (!(M > 0.0f)) { out[i] = 0.0f; if (codes_out_or_null) codes_out_or_null[i] = 0; continue; }
         const float a = fabsf(v[i]) / M;
@@ -374,7 +388,9 @@ int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byte
                   int bits, int level_mode, const float* feat_lo, const float* feat_step,
                   const float* levels, const float* b, float* x, int64_t batch, float lr,
                   int model_bits, int grad_bits, uint64_t seed, int64_t epoch, int64_t first_step,
-                  int64_t num_steps, const int32_t* batch_order, float* grad_out_or_null, int reg, float reg_param) {
+                  int64_t num_steps, const int32_t* batch_order, float* grad_out_or_null, int reg, float reg_param,
+                  int vector_norm) {
+    if (vector_norm != 0 && vector_norm != 1) return ORC_ERR_INVALID_ARG;
     const int cb = orc_container_bits(bits);
     if (cb == 0) return ORC_ERR_UNSUPPORTED;
     if (reg < 0 || reg > 4 || (reg != 0 && reg != 3 && !(reg_param >= 0.0f))) return ORC_ERR_INVALID_ARG;
@@ -394,7 +410,7 @@ int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byte
         const int64_t t = batch_order ? (int64_t)batch_order[it] : it;
         if (t < 0 || t >= T) return ORC_ERR_INVALID_ARG;
         const int64_t r0 = t * batch, r1 = (r0 + batch < m) ? r0 + batch : m;
-        if (model_bits > 0) orc_quantize_vector(x, n, model_bits, seed, (uint32_t)epoch, (uint32_t)it, 3, xt.data(), nullptr);
+        if (model_bits > 0) orc_quantize_vector_norm(x, n, model_bits, seed, (uint32_t)epoch, (uint32_t)it, 3, vector_norm, xt.data(), nullptr);
         else std::memcpy(xt.data(), x, sizeof(float) * (size_t)n);
         for (int64_t j = 0; j < n; ++j) gacc[j] = 0.0;
         for (int64_t k = r0; k < r1; ++k) {
@@ -409,7 +425,7 @@ int orc_sgd_epoch(const uint8_t* plane1, const uint8_t* plane2, int64_t row_byte
         for (int64_t j = 0; j < n; ++j) g[j] = (float)(gacc[j] * scale);
         const float* gu = g.data();
         if (grad_bits > 0) {
-            orc_quantize_vector(g.data(), n, grad_bits, seed, (uint32_t)epoch, (uint32_t)it, 4, gq.data(), nullptr);
+            orc_quantize_vector_norm(g.data(), n, grad_bits, seed, (uint32_t)epoch, (uint32_t)it, 4, vector_norm, gq.data(), nullptr);
             gu = gq.data();
         }
         for (int64_t j = 0; j < n; ++j) {

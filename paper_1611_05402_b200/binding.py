@@ -15,6 +15,7 @@ LEVELS_UNIFORM, LEVELS_TABLE = 0, 1
 LOSS_DENSE, LOSS_CODES = 0, 1
 LAYOUT_ROWS, LAYOUT_COLUMN_BLOCKS = 0, 1
 GRID_RANGE, GRID_SYMMETRIC = 0, 1
+NORM_L2, NORM_LINF = 0, 1
 REG_NONE, REG_L2, REG_L1, REG_NONNEG, REG_LSSVM = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_STEPWISE, ENGINE_PERSISTENT, ENGINE_RING, ENGINE_LEAN, ENGINE_CLUSTER, ENGINE_STREAM, ENGINE_COLUMN = 0, 1, 2, 3, 4, 5, 6, 7
 
@@ -55,7 +56,7 @@ class CSgdParams(C.Structure):
                 ("grid_feature_parts", C.c_int32), ("grid_row_parts", C.c_int32), ("trace_steps", C.c_int32),
                 ("trace", C.c_void_p), ("reg", C.c_int32), ("reg_param", C.c_float),
                 ("model_out", C.c_void_p), ("cluster_contraction", C.c_int32), ("stream_prefetch", C.c_int32),
-                ("column_chunk_rows", C.c_int32), ("reserved0", C.c_int32)]
+                ("column_chunk_rows", C.c_int32), ("vector_norm", C.c_int32)]
 
 
 _lib = None
@@ -338,7 +339,7 @@ class Context:
     def sgd_params(self, batch, lr, model_bits=0, grad_bits=0, seed=0, epoch=0, first_step=0, num_steps=-1,
                    batch_order=None, engine=ENGINE_AUTO, grid_feature_parts=0, grid_row_parts=0, trace=None,
                    reg=REG_NONE, reg_param=0.0, model_out=None, cluster_contraction=0, stream_prefetch=0,
-                   column_chunk_rows=0):
+                   column_chunk_rows=0, vector_norm=NORM_L2):
         p = CSgdParams()
         p.struct_size = C.sizeof(CSgdParams)
         p.model_bits, p.grad_bits, p.engine = model_bits, grad_bits, engine
@@ -347,6 +348,7 @@ class Context:
         p.reg, p.reg_param = reg, reg_param
         p.cluster_contraction, p.stream_prefetch = cluster_contraction, stream_prefetch
         p.column_chunk_rows = column_chunk_rows
+        p.vector_norm = vector_norm
         if model_out is not None:  # (n,) fp32 device tensor
             assert model_out.dtype == torch.float32 and model_out.is_contiguous() and model_out.device == self.device
             p.model_out = model_out.data_ptr()

@@ -250,7 +250,11 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->cluster_contraction < 0 || params->cluster_contraction > 2) return ZIPML_ERR_INVALID_ARG;
     if (params->stream_prefetch < 0 || params->stream_prefetch > 9) return ZIPML_ERR_INVALID_ARG;
     if (params->column_chunk_rows < 0 || params->column_chunk_rows > 256 || params->column_chunk_rows % 32 != 0) return ZIPML_ERR_INVALID_ARG;
-    if (params->reserved0 != 0) return ZIPML_ERR_INVALID_ARG;
+    if (params->vector_norm != ZIPML_NORM_L2 && params->vector_norm != ZIPML_NORM_LINF) return ZIPML_ERR_INVALID_ARG;
+    // the other scaling of Q3/Q4 lives in the first-generation engine only
+    const bool linf = params->vector_norm == ZIPML_NORM_LINF && (params->model_bits > 0 || params->grad_bits > 0);
+    if (linf && params->engine != ZIPML_ENGINE_AUTO && params->engine != ZIPML_ENGINE_STEPWISE && params->engine != ZIPML_ENGINE_PERSISTENT)
+        return ZIPML_ERR_UNSUPPORTED;
     const int64_t T = (data->m + params->batch - 1) / params->batch;
     const int64_t first = params->first_step;
     const int64_t count = params->num_steps < 0 ? T - first : params->num_steps;
@@ -261,6 +265,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (count == 0) return ZIPML_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
+    if (linf && data->layout == ZIPML_LAYOUT_COLUMN_BLOCKS) return ZIPML_ERR_UNSUPPORTED;
     if (data->layout == ZIPML_LAYOUT_COLUMN_BLOCKS) {                 // the column engine's own layout
         if (params->engine != ZIPML_ENGINE_AUTO && params->engine != ZIPML_ENGINE_COLUMN) return ZIPML_ERR_UNSUPPORTED;
         rc = launch_sgd_column(ctx, data, b, x, params, first, count, grad_out, false);
@@ -271,7 +276,7 @@ int zipml_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* data, const float* b, f
     if (params->engine == ZIPML_ENGINE_CLUSTER) return launch_sgd_cluster(ctx, data, b, x, params, first, count, grad_out);
     if (params->engine == ZIPML_ENGINE_STREAM) return launch_sgd_stream(ctx, data, b, x, params, first, count, grad_out, false);
     if (params->engine == ZIPML_ENGINE_COLUMN) return launch_sgd_column(ctx, data, b, x, params, first, count, grad_out, false);
-    if (params->engine == ZIPML_ENGINE_AUTO) {
+    if (params->engine == ZIPML_ENGINE_AUTO && !linf) {
         // Small minibatch tiles are bound by the step-to-step chain, not by HBM: one cluster whose CTAs
         // exchange through shared memory, else row parts exchanging through L2.  Larger tiles go to the
         // column engine (codes read once per step), the stream engine, then the ring engine.  Each engine
@@ -303,6 +308,7 @@ int zipml_sgd_apply_gradient(zipml_ctx* ctx, float* x, const float* g, int64_t n
     if (params->epoch < 0 || params->epoch > 0xffffffffLL) return ZIPML_ERR_INVALID_ARG;
     if (params->reg < ZIPML_REG_NONE || params->reg > ZIPML_REG_LSSVM) return ZIPML_ERR_INVALID_ARG;
     if (params->reg != ZIPML_REG_NONE && params->reg != ZIPML_REG_NONNEG && !(params->reg_param >= 0.0f)) return ZIPML_ERR_INVALID_ARG;
+    if (params->vector_norm != ZIPML_NORM_L2 && params->vector_norm != ZIPML_NORM_LINF) return ZIPML_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return ZIPML_ERR_CUDA;
     return launch_sgd_apply(ctx, x, g, n, params, step, applied_out);

@@ -130,6 +130,23 @@ __device__ __forceinline__ double block_sum(double v, double* scratch) {
     return scratch[32];
 }
 
+// The same for a maximum of non-negative values.
+__device__ __forceinline__ double block_max(double v, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < nwarps; ++w) t = fmax(t, scratch[w]);
+        scratch[32] = t;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
 // Order-preserving map float -> uint32 so that integer atomicMin/Max order floats (-0 < +0).
 __device__ __forceinline__ uint32_t float_order_key(float f) {
     const uint32_t b = __float_as_uint(f);

@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_kernel(const SgdArgs a) {
         // ------------------------------------------------------------------ phase A: dots
         if (a.phases & kPhaseA) {
             VecQuant q3{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 3u};
-            if (a.model_bits > 0) { q3.M = l2_norm_smem(xs, F, red); q3.sm = (1 << (a.model_bits - 1)) - 1; }
+            if (a.model_bits > 0) { q3.M = vector_scale_smem(xs, F, red, a.vector_norm); q3.sm = (1 << (a.model_bits - 1)) - 1; }
             double base = 0.0;
             if constexpr (!TABLE) {
                 for (int q = threadIdx.x; q < a.wc; q += kSgdThreads) {
@@ -461,7 +461,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_kernel(const SgdArgs a) {
             }
             __syncthreads();
             VecQuant q4{0.0f, 1, a.seed, a.epoch, (uint32_t)it, 4u};
-            if (a.grad_bits > 0) { q4.M = l2_norm_smem(gs, F, red); q4.sm = (1 << (a.grad_bits - 1)) - 1; }
+            if (a.grad_bits > 0) { q4.M = vector_scale_smem(gs, F, red, a.vector_norm); q4.sm = (1 << (a.grad_bits - 1)) - 1; }
             for (int f = threadIdx.x; f < fcnt; f += kSgdThreads) {
                 float g = gs[f];
                 if (a.grad_bits > 0) g = q4.apply(g, (uint32_t)(j0 + f));
@@ -629,7 +629,7 @@ int launch_sgd_epoch(zipml_ctx* ctx, const zipml_dataset* d, const float* b, flo
     a.b = b; a.x = x; a.grad_out = grad_out; a.model_out = p->model_out;
     a.batch = p->batch < d->m ? p->batch : d->m;
     a.first_step = first_step; a.num_steps = num_steps;
-    a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits;
+    a.lr = p->lr; a.reg = p->reg; a.reg_cst = reg_constant(p); a.model_bits = p->model_bits; a.grad_bits = p->grad_bits; a.vector_norm = p->vector_norm;
     a.seed = p->seed; a.epoch = (uint32_t)p->epoch;
     a.na = plan.na; a.nb = plan.nb; a.wc = plan.wc; a.rc = plan.rc; a.stages = plan.stages;
     a.pd = reinterpret_cast<double*>(ctx->ws + sc.pd_off);

@@ -33,7 +33,7 @@ struct SgdArgs {
     float lr;
     int reg;                // ZIPML_REG_* and its fp32 constant
     float reg_cst;
-    int model_bits, grad_bits;
+    int model_bits, grad_bits, vector_norm;
     uint64_t seed;
     uint32_t epoch;
     int na, nb;             // feature parts, row parts
@@ -135,6 +135,15 @@ struct VecQuant {
         return v < 0.0f ? -q : q;
     }
 };
+
+// The scale M(v) of a vector in shared memory: ||v||_2, or max |v_i| for ZIPML_NORM_LINF.
+__device__ __forceinline__ float l2_norm_smem(const float* v, int count, double* red);
+__device__ __forceinline__ float vector_scale_smem(const float* v, int count, double* red, int norm) {
+    if (norm == ZIPML_NORM_L2) return l2_norm_smem(v, count, red);
+    double mx = 0.0;
+    for (int i = threadIdx.x; i < count; i += kSgdThreads) mx = fmax(mx, (double)fabsf(v[i]));
+    return (float)block_max(mx, red);
+}
 
 __device__ __forceinline__ float l2_norm_smem(const float* v, int count, double* red) {
     double ss = 0.0;

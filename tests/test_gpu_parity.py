@@ -1063,3 +1063,54 @@ def test_symmetric_grid(ctx, bits):
                            levels=torch.zeros((260, 8), device=ctx.device))
     with pytest.raises(binding.ZipmlError):
         ctx.zipml_quantize(to_dev(A, ctx), bits, seed=0, grid=2)
+
+
+def test_vector_scaling_by_the_largest_entry(ctx):
+    """ZIPML_NORM_LINF: Q3 and Q4 scaled by max |v_i| (the Supplement leaves M(v) general).  AUTO runs the
+    first-generation engine for it, the others refuse; an epoch and a single step against the oracle, and
+    zipml_sgd_apply_gradient with the same option."""
+    m, n, batch, lr = 2000, 300, 250, 2e-3
+    _, A, b, _ = workload("c2", m, n, seed=12)
+    ods = oracle.quantize(A, 4, seed=2)
+    gds, db = dev_dataset(ods, ctx), to_dev(b, ctx)
+    x0 = (np.random.default_rng(3).standard_normal(n) * 0.05).astype(np.float32)
+    kw = dict(model_bits=6, grad_bits=6, seed=5, epoch=1)
+    # one step: gradient before Q4 from the model the kernel used, then Q4's decisions
+    x, g = to_dev(x0, ctx), torch.zeros((2, n), dtype=torch.float32, device=ctx.device)
+    xq = torch.zeros(n, dtype=torch.float32, device=ctx.device)
+    ctx.zipml_sgd_epoch(gds, db, x, batch, lr, first_step=2, num_steps=1, grad_out=g, model_out=xq, vector_norm=binding.NORM_LINF, **kw)
+    ctx.zipml_sync()
+    assert ctx.zipml_last_engine() in (binding.ENGINE_STEPWISE, binding.ENGINE_PERSISTENT)
+    xq_ref, _ = oracle.quantize_vector(x0, 6, 5, 1, 2, 3, norm=oracle.NORM_LINF)
+    assert (xq.cpu().numpy() != xq_ref).sum() <= 2
+    _, g_ref = oracle.sgd_epoch(ods, b, xq.cpu().numpy(), batch, lr, model_bits=0, grad_bits=6, seed=5, epoch=1, first_step=2,
+                                num_steps=1, want_grad=True, vector_norm=oracle.NORM_LINF)
+    gg = g.cpu().numpy()
+    assert rel(gg[0], g_ref[0]) <= GRAD_TOL
+    unit = np.abs(g_ref[0]).max() / 31
+    flips = np.abs(gg[1] - g_ref[1]) > 0.5 * unit
+    assert flips.sum() <= 2 and np.abs(gg[1] - g_ref[1])[~flips].max() <= 1e-5 * unit + 1e-12
+    assert np.abs(gg[1]).max() <= np.abs(gg[0]).max() * (1 + 1e-6)          # nothing beyond the largest entry
+    # whole epoch
+    x = to_dev(x0, ctx)
+    ctx.zipml_sgd_epoch(gds, db, x, batch, lr, vector_norm=binding.NORM_LINF, **kw)
+    ctx.zipml_sync()
+    x_ref, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, vector_norm=oracle.NORM_LINF, **kw)
+    assert rel(x.cpu().numpy(), x_ref) <= 20 * MODEL_TOL
+    x_l2, _ = oracle.sgd_epoch(ods, b, x0, batch, lr, **kw)
+    assert rel(x_l2, x_ref) > 1e-3                                           # the option does change the trajectory
+    # the end of a step on its own
+    xa = to_dev(x0, ctx)
+    ctx.zipml_sgd_apply_gradient(xa, to_dev(g_ref[0], ctx), 2, lr, grad_bits=6, seed=5, epoch=1, vector_norm=binding.NORM_LINF)
+    ctx.zipml_sync()
+    want = x0 - np.float32(lr) * g_ref[1]
+    assert (np.abs(xa.cpu().numpy() - want) > 1e-6).sum() <= 2
+    # other engines refuse; without Q3/Q4 the option means nothing and every engine runs
+    for engine in (binding.ENGINE_CLUSTER, binding.ENGINE_LEAN, binding.ENGINE_RING):
+        with pytest.raises(binding.ZipmlError) as e:
+            ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=engine, vector_norm=binding.NORM_LINF, **kw)
+        assert e.value.code == binding.ERR_UNSUPPORTED
+    ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, engine=binding.ENGINE_CLUSTER, vector_norm=binding.NORM_LINF)
+    ctx.zipml_sync()
+    with pytest.raises(binding.ZipmlError):
+        ctx.zipml_sgd_epoch(gds, db, to_dev(x0, ctx), batch, lr, vector_norm=2)

@@ -543,3 +543,30 @@ def test_symmetric_grid_of_the_supplements_column_scaling():
     assert np.abs(acc / N - A).max() < 5 * (2 * M.max() / s / 2) / np.sqrt(N) + 1e-6
     with pytest.raises(oracle.OracleError):
         oracle.quantize_pair(A, bits, 0, 0, mode=oracle.TABLE, levels=np.zeros((5, 8), np.float32), symmetric=True)
+
+
+def test_vector_quantizer_scaled_by_the_largest_entry():
+    """M(v) = max |v_i| instead of ||v||_2 (the Supplement leaves M general): the largest entry is reproduced exactly,
+    nothing exceeds it, the mean over draws is v, and the variance is below the l2-scaled quantizer's."""
+    rng = np.random.default_rng(8)
+    v = rng.standard_normal(40).astype(np.float32)
+    bits, N = 4, 4000
+    big = int(np.argmax(np.abs(v)))
+    acc = np.zeros(40)
+    var_inf = var_l2 = 0.0
+    for step in range(N):
+        q, codes = oracle.quantize_vector(v, bits, 5, 1, step, 4, norm=oracle.NORM_LINF)
+        assert q[big] == v[big] and abs(int(codes[big])) == 7
+        assert np.abs(q).max() <= np.abs(v).max()
+        acc += q
+        var_inf += ((q - v) ** 2).sum()
+        var_l2 += ((oracle.quantize_vector(v, bits, 5, 1, step, 4)[0] - v) ** 2).sum()
+    unit = np.abs(v).max() / 7
+    assert np.abs(acc / N - v).max() < 5 * (unit / 2) / np.sqrt(N) + 1e-6
+    assert var_inf < 0.5 * var_l2
+    # the default is the l2 scaling, unchanged
+    a, _ = oracle.quantize_vector(v, bits, 5, 1, 0, 4)
+    b, _ = oracle.quantize_vector(v, bits, 5, 1, 0, 4, norm=oracle.NORM_L2)
+    assert np.array_equal(a, b) and np.abs(a).max() <= np.linalg.norm(v) * (1 + 1e-6)
+    z, zc = oracle.quantize_vector(np.zeros(5, np.float32), bits, 0, 0, 0, 3, norm=oracle.NORM_LINF)
+    assert not z.any() and not zc.any()
