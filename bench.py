@@ -62,7 +62,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -142,7 +142,7 @@ def oracle_sample_rows(w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", help="c1..c5, c4u (see paper_1611_05402_b200/synth.py)")
@@ -268,13 +268,15 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
+    # (the sampler starts before the warm-up passes -- the same work as the timed ones -- so that its first samples
+    # do not wait for nvidia-smi to come up inside a timed region of a fraction of a second)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(max(args.warmup, 0)):
         ds, x = one_pass(False)
     ctx.zipml_sync()
-    sampler = ClockSampler(local_rank)
     fence()
     launches0 = ctx.zipml_kernel_launches()
-    sampler.start()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(args.steps):
