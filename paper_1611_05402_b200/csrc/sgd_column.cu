@@ -284,7 +284,9 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     const int rstride = R + 32;                        // bytes between the residual digit vectors
     signed char* rdig = reinterpret_cast<signed char*>(tiles_b + (size_t)a.slots_b * slot_bytes);  // [R warps][2 operands][8 digits][rstride]
     signed char* wdig = rdig + (size_t)kColRWarps * 2 * NRD * rstride;                             // [NG][4 k-blocks][4 digits][32 B]
-    ColShared* sh = reinterpret_cast<ColShared*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * NS * 32) + 15) & ~(uintptr_t)15);
+    // the A warps' hand-over of a task's digit sums from the lanes that hold them to a lane per row ([A warps][2 planes][32 rows][2])
+    int* ascr = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * NS * 32) + 15) & ~(uintptr_t)15);
+    ColShared* sh = reinterpret_cast<ColShared*>(ascr + (size_t)kColAWarps * 2 * 32 * 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gl = lane >> 2, tl = lane & 3;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -479,8 +481,12 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     }
                 }
                 // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3]) of each tile.  Integers all
-                // the way: the groups' sums (multiples of 2^(g CB), shifted back exactly) in 32 bits, two digits per
-                // lane and then the neighbour's two in 64, the shift into the dots' unit, the own part of lo^T x.
+                // the way: the groups' sums (multiples of 2^(g CB), shifted back exactly) and two digits per lane in
+                // 32 bits; through a few words of shared memory every lane then takes one row: the two lanes' pairs
+                // in 64 bits, the shift into the dots' unit, the own part of lo^T x, and one addition per plane whose
+                // 32 lanes cover 256 consecutive bytes (the fewer and wider the requests, the sooner L2 is through
+                // with a chunk's additions).
+                int* as = ascr + (size_t)aw * 2 * 32 * 2;
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -491,16 +497,23 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                             x10 += c1[h][g][2 * e] >> (g * CB); x11 += c1[h][g][2 * e + 1] >> (g * CB);
                             x20 += c2[h][g][2 * e] >> (g * CB); x21 += c2[h][g][2 * e + 1] >> (g * CB);
                         }
-                        const long long q1 = (long long)x10 + ((long long)x11 << 7), q2 = (long long)x20 + ((long long)x21 << 7);
-                        const long long v1 = q1 + (__shfl_down_sync(0xffffffffu, q1, 1) << 14);
-                        const long long v2 = q2 + (__shfl_down_sync(0xffffffffu, q2, 1) << 14);
-                        const int k = k0 + 16 * h + gl + 8 * e;
-                        if (tl == 0 && k < st.bt) {
-                            // the word's upper 56 bits take the sum, its low byte counts this CTA in
-                            red_add_u64(dots + k, ((unsigned long long)((v1 << kshift) + bint) << 8) + 1ull);
-                            red_add_u64(dots + a.bpad + k, ((unsigned long long)((v2 << kshift) + bint) << 8) + 1ull);
+                        if (tl < 2) {
+                            const int row = 16 * h + 8 * e + gl;
+                            as[row * 2 + tl] = x10 + (x11 << 7);
+                            as[64 + row * 2 + tl] = x20 + (x21 << 7);
                         }
                     }
+                __syncwarp();
+                {
+                    const int2 p1 = *reinterpret_cast<const int2*>(as + 2 * lane), p2 = *reinterpret_cast<const int2*>(as + 64 + 2 * lane);
+                    const long long v1 = (long long)p1.x + ((long long)p1.y << 14), v2 = (long long)p2.x + ((long long)p2.y << 14);
+                    const int k = k0 + lane;
+                    if (k < st.bt) {
+                        // the word's upper 56 bits take the sum, its low byte counts this CTA in
+                        red_add_u64(dots + k, ((unsigned long long)((v1 << kshift) + bint) << 8) + 1ull);
+                        red_add_u64(dots + a.bpad + k, ((unsigned long long)((v2 << kshift) + bint) << 8) + 1ull);
+                    }
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty_a + ring.slot));
@@ -952,7 +965,8 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     while (ngrp > 1 && (int64_t)(ngrp - 1) * gsize >= G) --ngrp;       // no empty group
 
     const size_t slot_bytes = (size_t)2 * R * kColBlockBytes;
-    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 4 * 32 + 16 + sizeof(ColShared);
+    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 4 * 32 + 16 +
+                         (size_t)kColAWarps * 2 * 32 * 2 * sizeof(int) + sizeof(ColShared);
     if (fixed + 4 * slot_bytes > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
     int slots = (int)(((size_t)ctx->smem_optin - fixed) / slot_bytes);
     if (slots > 2 * kColMaxSlots) slots = 2 * kColMaxSlots;
