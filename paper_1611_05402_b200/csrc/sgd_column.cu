@@ -41,8 +41,9 @@
 // relative precision is touched.  w of the own features: four digits (27 bits) whose unit is U times a power
 // of two, at most twice what the CTA's own max |w| needs, so that a digit sum becomes a multiple of U by a
 // shift; the own part of lo^T x is rounded to a multiple of U once per step: the path from the tensor-core
-// sums to the atomic is integer arithmetic only.  Residuals: eight digits (55 bits) relative to D(t) +
-// max |b| of the step; all eight columns of the tensor-core tile carry a digit.  Digits are balanced
+// sums to the atomic is integer arithmetic only.  Residuals: eight digits (55 bits) whose unit is a power of two
+// as well, at most twice what D(t) + max |b| of the step needs, so that a dot becomes a residual by a shift and
+// the label's fixed-point value (one conversion per row); all eight columns of the tensor-core tile carry a digit.  Digits are balanced
 // (-64..63) and found without a carry chain: with 64 added to every digit the number is plain base 128.
 // Results do not depend on timing: every sum is an integer sum or has a fixed order.
 //
@@ -724,9 +725,14 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
 #pragma unroll
             for (int w = 0; w < kColRWarps; ++w) bm = fmaxf(bm, sh->red_f[1][w]);
             const double rbound = (dbound + (double)bm) * 1.0001;
-            const double inv_r = rbound > 0.0 ? (double)kColQmaxR / rbound : 0.0;
-            const double U = sp.U;
-            double rmax = 0.0;
+            // The residuals' unit is a power of two as well (at most twice what the bound needs), so that a dot becomes
+            // a residual by a shift and the label's own fixed-point value: integers only on the way to the digits.
+            const int ed = rbound > 0.0 ? max(-900, min(900, col_exponent(rbound * (1.0 / (double)kColQmaxR)) + 1)) : 0;
+            const double delta_r = col_pow2(ed), inv_delta = col_pow2(-ed);
+            const int sft = col_exponent(sp.U) - ed;     // dot unit over residual unit: 2^sft (at most 2^4 by construction)
+            const int lsh = max(0, min(sft, 8)), rsh = min(63, max(0, -sft));
+            const long long half = rsh > 0 ? (1ll << (rsh - 1)) : 0;
+            long long amax = 0;                          // largest |fixed-point residual| of the lane
             long long rs_hi = 0, rs_lo = 0;              // sum of the fixed-point residuals: high parts and low 28 bits
             const int c_last = st.nch - 1;
 #pragma unroll 1
@@ -813,10 +819,10 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     for (int i = 0; i < 4; ++i) {
                         long long R1 = 0, R2 = 0;
                         if (kA + (i & 1) + 8 * (i >> 1) < st.bt) {
-                            const double r1 = (double)D1[i] * U - (double)bk[i], r2 = (double)D2[i] * U - (double)bk[i];
-                            rmax = fmax(rmax, fmax(fabs(r1), fabs(r2)));
-                            R1 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r1 * inv_r)));
-                            R2 = max(-kColQmaxR, min(kColQmaxR, __double2ll_rn(r2 * inv_r)));
+                            const long long bfix = __double2ll_rn((double)bk[i] * inv_delta);
+                            R1 = max(-kColQmaxR, min(kColQmaxR, (((D1[i] + half) >> rsh) << lsh) - bfix));
+                            R2 = max(-kColQmaxR, min(kColQmaxR, (((D2[i] + half) >> rsh) << lsh) - bfix));
+                            amax = max(amax, max(llabs(R1), llabs(R2)));
                             rs_hi += (R1 >> 28) + (R2 >> 28);
                             rs_lo += (R1 & 0xFFFFFFFll) + (R2 & 0xFFFFFFFll);
                         }
@@ -863,11 +869,11 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             // ---- the step's residuals are all known: their sum for the B warps, the next step's bound and unit
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-                rmax = fmax(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+                amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
                 rs_hi += __shfl_xor_sync(0xffffffffu, rs_hi, o);
                 rs_lo += __shfl_xor_sync(0xffffffffu, rs_lo, o);
             }
-            if (lane == 0) { sh->red_d[1][rw] = rmax; sh->red_l[0][rw] = rs_hi; sh->red_l[1][rw] = rs_lo; }
+            if (lane == 0) { sh->red_d[1][rw] = (double)amax * delta_r; sh->red_l[0][rw] = rs_hi; sh->red_l[1][rw] = rs_lo; }
             named_barrier(kColNamedR, kColRThreads);     // (the next step's barrier keeps these slots from being rewritten early)
             double rm = 0.0;
             long long hi = 0, lo = 0;
@@ -877,8 +883,8 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             if (((q0 + c_last) & (kColRWarps - 1)) == rw) {      // the warp that holds the step's last chunk
                 if (lane == 0) {
                     ColStepParams& cur = sh->sp[t_rel & 1];
-                    cur.inv_r = inv_r;
-                    cur.delta_r = rbound / (double)kColQmaxR;
+                    cur.inv_r = inv_delta;
+                    cur.delta_r = delta_r;
                     cur.rsum = (double)hi * 268435456.0 + (double)lo;
                     col_unit_of(dbound, sh->sp[(t_rel + 1) & 1].U, sh->sp[(t_rel + 1) & 1].invU);
                 }
