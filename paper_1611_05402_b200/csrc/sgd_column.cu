@@ -165,7 +165,7 @@ __device__ __noinline__ bool col_wait(unsigned long long* bar, uint32_t parity, 
 #pragma unroll 1
     for (int spin = 0;; ++spin) {
         if (mbar_try_wait_parked(bar, parity)) return true;
-        if (spin >= 4) __nanosleep(spin < 16 ? 100 : 400);       // a warp that waits long should stay out of the others' way
+        if (spin >= 4) __nanosleep(spin < 16 ? 200 : 800);       // a warp that waits long should stay out of the others' way
         if ((spin & 15) == 15) {
             if (col_aborted(sh)) return false;
             if (clock64() - t0 > kColWaitCycles) break;
@@ -202,7 +202,7 @@ __device__ __noinline__ bool col_wait_version(const int* version, int want, ColS
     const long long t0 = clock64();
 #pragma unroll 1
     for (int spin = 0; ld_acquire_cta(version) < want; ++spin) {
-        __nanosleep(100);
+        __nanosleep(400);
         if ((spin & 15) == 15) {
             if (col_aborted(sh)) return false;
             if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(status, ZIPML_ERR_TIMEOUT, where); return false; }
@@ -768,7 +768,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                                 if (col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0) { sh->abort_flag = 1; break; }
                                 if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 75); break; }
                             }
-                            __nanosleep(200);
+                            __nanosleep(400);
                         }
                     }
                 }
@@ -800,7 +800,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         }
                     }
                     if (__all_sync(0xffffffffu, done) || !ok) break;
-                    __nanosleep(100);
+                    __nanosleep(200);
                     if ((spin & 7) == 7) {
                         bool give_up = col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0;
                         if (clock64() - t0 > kColWaitCycles) { set_status(a.status, ZIPML_ERR_TIMEOUT, 77); give_up = true; }
