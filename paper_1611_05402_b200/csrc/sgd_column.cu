@@ -65,6 +65,8 @@
 #include <cuda.h>
 #include <string.h>
 
+#include <type_traits>
+
 #include "int_digits.cuh"
 #include "sgd_common.cuh"
 
@@ -452,15 +454,9 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             const int k0 = c * R + j * 32;                                // first row of the task within the step
             if (k0 < st.bt) {
                 int c1[2][NG][4], c2[2][NG][4];                          // [tile][group][fragment]: plane 1, plane 2
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int g = 0; g < NG; ++g)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) { c1[h][g][e] = 0; c2[h][g][e] = 0; }
                 const uint32_t row_addr = tile + (uint32_t)(j * 32 + a_row) * kColBlockBytes;
-#pragma unroll 1
-                for (int kb = 0; kb < 4; ++kb) {
+                // one 32-byte k-block of the two tiles and planes; the first one starts the sums (no cleared registers)
+                auto kblock = [&](int kb, auto first) {
                     uint32_t f1[2][4], f2[2][4];
                     const uint32_t off = row_addr + (((uint32_t)(2 * kb) + a_piece) ^ a_x) * 16u;
 #pragma unroll
@@ -476,11 +472,19 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         const uint32_t mk = kLow << (g * CB);
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            mma_u8s8(c1[h][g], f1[h][0] & mk, f1[h][1] & mk, f1[h][2] & mk, f1[h][3] & mk, b0, b1);
-                            mma_u8s8(c2[h][g], f2[h][0] & mk, f2[h][1] & mk, f2[h][2] & mk, f2[h][3] & mk, b0, b1);
+                            if constexpr (decltype(first)::value) {
+                                mma_u8s8_first(c1[h][g], f1[h][0] & mk, f1[h][1] & mk, f1[h][2] & mk, f1[h][3] & mk, b0, b1);
+                                mma_u8s8_first(c2[h][g], f2[h][0] & mk, f2[h][1] & mk, f2[h][2] & mk, f2[h][3] & mk, b0, b1);
+                            } else {
+                                mma_u8s8(c1[h][g], f1[h][0] & mk, f1[h][1] & mk, f1[h][2] & mk, f1[h][3] & mk, b0, b1);
+                                mma_u8s8(c2[h][g], f2[h][0] & mk, f2[h][1] & mk, f2[h][2] & mk, f2[h][3] & mk, b0, b1);
+                            }
                         }
                     }
-                }
+                };
+                kblock(0, std::true_type{});
+#pragma unroll 1
+                for (int kb = 1; kb < 4; ++kb) kblock(kb, std::false_type{});      // (unrolled it was no faster: more machine code)
                 // lane t < 2 holds digits 2t, 2t+1 of rows g (c[0], c[1]) and g+8 (c[2], c[3]) of each tile.  Integers all
                 // the way: the groups' sums (multiples of 2^(g CB), shifted back exactly) and two digits per lane in
                 // 32 bits; through a few words of shared memory every lane then takes one row: the two lanes' pairs
