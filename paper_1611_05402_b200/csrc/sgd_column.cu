@@ -49,7 +49,7 @@
 //
 // The machine code is kept small on purpose (four roles share the instruction cache): 32-bit counters kept up
 // step by step instead of 64-bit divisions, waits as functions with one copy, loops unrolled only where
-// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 25.2 us per step (stream engine:
+// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 24.7 us per step (stream engine:
 // 29.8), DRAM reads 1.00 x the packed bytes.  Not HBM bounds it but the chain of a step: the first chunk's dots
 // have to cross L2 and become digits before pass B can start (about 9 k cycles), pass B then follows the R
 // warps (about 2 k cycles per chunk for the four of them together) rather than the copies, and the next
