@@ -617,7 +617,10 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 }
                 if (a.trace && p == 0 && lane == 0) { col_tally(a, t_rel, 4, w1c - w0c); col_tally(a, t_rel, 5, clock64() - w1c); }
                 const uint32_t tile = smem_u32(tiles_b) + (uint32_t)ring.slot * slot_bytes + b_off;
-                const int nrb = ok ? (min(R, st.bt - c * R) + 31) >> 5 : 0;
+                // Rows past the step's last one carry zero digits, so whole chunks are contracted: all R / 32 blocks, and
+                // for the usual R = 128 without a test per block.
+                const int nrb = ok ? R >> 5 : 0;
+                auto blocks = [&](auto whole) {
 #pragma unroll
                 for (int rb2 = 0; rb2 < kColMaxChunkRows / 32; rb2 += 2) {
                     // the four operand pairs of two 32-row blocks are fetched together, then used: one wait for shared
@@ -628,7 +631,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
 #pragma unroll
                         for (int pl = 0; pl < 2; ++pl) {
                             const int rb = rb2 + h;
-                            if (rb < nrb) {
+                            if (decltype(whole)::value || rb < nrb) {
                                 ldsm_x4_trans(r4[h][pl], tile + (uint32_t)pl * plane_bytes + (uint32_t)rb * 32u * kColBlockBytes);
                                 asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0[h][pl]), "=r"(b1[h][pl])
                                              : "r"(rdig_lane + (uint32_t)(((rbuf * 2 + pl) * NRD) * rstride + rb * 32)));
@@ -638,7 +641,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     for (int pl = 0; pl < 2; ++pl)                   // (neighbouring MMAs go to different accumulators)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            if (rb2 + h < nrb) {
+                            if (decltype(whole)::value || rb2 + h < nrb) {
                                 // bytes {2g, 2g+1} of rows {2t, 2t+1} of the four 8-row groups -> byte 2g (and 2g+1) of rows
                                 // {2t, 2t+1, 8+2t, 9+2t} (+16): features x rows, in the row order of the residual digits
                                 const uint32_t* r = r4[h][pl];
@@ -655,6 +658,9 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                             }
                         }
                 }
+                };
+                if (nrb == kColMaxChunkRows / 32) blocks(std::true_type{});
+                else blocks(std::false_type{});
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(reinterpret_cast<uint64_t*>(sh->empty_b + ring.slot));
