@@ -286,9 +286,9 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     unsigned char* tiles_b = tiles + (size_t)a.slots_a * slot_bytes;
     const int rstride = R + 32;                        // bytes between the residual digit vectors
     signed char* rdig = reinterpret_cast<signed char*>(tiles_b + (size_t)a.slots_b * slot_bytes);  // [R warps][2 operands][8 digits][rstride]
-    signed char* wdig = rdig + (size_t)kColRWarps * 2 * NRD * rstride;                             // [NG][4 k-blocks][4 digits][32 B]
+    signed char* wdig = rdig + (size_t)kColRWarps * 2 * NRD * rstride;                             // [NG][4 k-blocks][8 columns: 4 digits, 4 x zero][32 B]
     // the A warps' hand-over of a task's digit sums from the lanes that hold them to a lane per row ([A warps][2 planes][32 rows][2])
-    int* ascr = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * NS * 32) + 15) & ~(uintptr_t)15);
+    int* ascr = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * 8 * 32) + 15) & ~(uintptr_t)15);
     ColShared* sh = reinterpret_cast<ColShared*>(ascr + (size_t)kColAWarps * 2 * 32 * 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gl = lane >> 2, tl = lane & 3;
@@ -300,6 +300,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     const int x_own = a.blocked ? 0 : (int)byte0;
     const int64_t y_own = a.blocked ? (int64_t)cta * a.m : 0;
 
+    for (int i = tid; i < NG * 4 * 8 * 32 / 4; i += kColThreads) reinterpret_cast<uint32_t*>(wdig)[i] = 0u;     // (digit columns 4..7 stay zero)
     if (tid == 0) {
         for (int s = 0; s < kColMaxSlots; ++s) {
             mbar_init(reinterpret_cast<uint64_t*>(sh->full_a + s), 1);
@@ -466,8 +467,8 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     }
 #pragma unroll
                     for (int g = 0; g < NG; ++g) {
-                        uint32_t b0 = 0u, b1 = 0u;
-                        if (gl < NS) asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(wdig_lane + (uint32_t)((g * 4 + kb) * NS * 32)));
+                        uint32_t b0, b1;                         // (columns 4..7 of the operand are zeros that stay in place)
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(wdig_lane + (uint32_t)((g * 4 + kb) * 8 * 32)));
                         // group g's codes stay where they are in the byte: its sums come out 2^(g CB) times too large
                         const uint32_t mk = kLow << (g * CB);
 #pragma unroll
@@ -585,7 +586,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         const int byte = 16 * p + 2 * gl + h, kb = byte >> 5, bb = byte & 31;
                         // balanced digits without a carry chain: with 64 added to every digit the number is plain base 128
                         const uint32_t u = (uint32_t)((have[e] ? max(-QMAXW, min(QMAXW, __float2int_rn(st_o[e] * xo[e] * inv))) : 0) + kColBiasW);
-                        signed char* dst = wdig + (size_t)((gi * 4 + kb) * NS) * 32 + ((bb & 15) >> 2) * 8 + (bb >> 4) * 4 + (bb & 3);
+                        signed char* dst = wdig + (size_t)((gi * 4 + kb) * 8) * 32 + ((bb & 15) >> 2) * 8 + (bb >> 4) * 4 + (bb & 3);
 #pragma unroll
                         for (int s = 0; s < NS; ++s) dst[s * 32] = (signed char)((int)((u >> (7 * s)) & 127u) - 64);
                     }
@@ -981,7 +982,7 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     while (ngrp > 1 && (int64_t)(ngrp - 1) * gsize >= G) --ngrp;       // no empty group
 
     const size_t slot_bytes = (size_t)2 * R * kColBlockBytes;
-    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 4 * 32 + 16 +
+    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 8 * 32 + 16 +
                          (size_t)kColAWarps * 2 * 32 * 2 * sizeof(int) + sizeof(ColShared);
     if (fixed + 4 * slot_bytes > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
     int slots = (int)(((size_t)ctx->smem_optin - fixed) / slot_bytes);
