@@ -746,6 +746,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             long long amax = 0;                          // largest |fixed-point residual| of the lane
             long long rs_hi = 0, rs_lo = 0;              // sum of the fixed-point residuals: high parts and low 28 bits
             const int c_last = st.nch - 1;
+            bool behind = false;                         // (a step's first chunks are never complete yet)
 #pragma unroll 1
             for (int c = (rw - q0) & (kColRWarps - 1); c < st.nch; c += kColRWarps) {
                 const int q = q0 + c;
@@ -764,8 +765,11 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 // ---- the chunk's dots.  First a few lanes watch the last row of each 32-row task and group (one request
                 // per look, with a pause: five hundred warps looking at L2 as fast as it answers would take a good part
                 // of its bandwidth), then every lane reads its own rows' words until their counts are complete too.
+                // A warp that found its previous chunk complete at the first look is behind pass A: it skips the watch
+                // (a round trip to L2) and reads the words at once.
                 const long long t0 = clock64();
-                if (lane < 4 * ngrp && ok) {
+                bool first_look = true;
+                if (lane < 4 * ngrp && ok && !behind) {
                     const int g = lane >> 2, first = c * R + 32 * (lane & 3);
                     if (first < st.bt && 32 * (lane & 3) < R) {
                         const long long* wl = dots + ((size_t)g * 2 + 1) * a.bpad + min(st.bt, first + 32) - 1;
@@ -775,6 +779,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                             long long v0;
                             asm volatile("ld.global.cg.s64 %0, [%1];" : "=l"(v0) : "l"(wl) : "memory");
                             if ((int)(v0 & 0xFF) >= want) break;
+                            first_look = false;
                             if ((spin & 15) == 15) {
                                 if (col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0) { sh->abort_flag = 1; break; }
                                 if (clock64() - t0 > kColWaitCycles) { sh->abort_flag = 1; set_status(a.status, ZIPML_ERR_TIMEOUT, 75); break; }
@@ -811,6 +816,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         }
                     }
                     if (__all_sync(0xffffffffu, done) || !ok) break;
+                    first_look = false;
                     __nanosleep(200);
                     if ((spin & 7) == 7) {
                         bool give_up = col_aborted(sh) || *reinterpret_cast<volatile int*>(&a.status->code) != 0;
@@ -818,6 +824,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                         if (__any_sync(0xffffffffu, give_up)) { sh->abort_flag = 1; ok = false; }
                     }
                 }
+                behind = __all_sync(0xffffffffu, first_look);
                 const long long e0c = (a.trace && rw == 0) ? clock64() : 0;
                 if (ok && q >= kColRWarps) ok = col_wait(sh->rempty + rw, (uint32_t)(((q >> kColRShift) - 1) & 1), sh, a.status, 76);
                 ok = __all_sync(0xffffffffu, ok);
