@@ -72,7 +72,10 @@
 
 namespace zipml {
 
-constexpr int kColAWarps = 8, kColBWarps = 8, kColRWarps = 4, kColRShift = 2;     // (kColRWarps = 2^kColRShift)
+constexpr int kColAWarps = 8, kColBWarps = 8, kColRWarps = 4;
+// Digit buffers: two per R warp (chunk q goes to buffer q mod kColRBufs), so that a warp can write its next chunk's
+// digits while pass B still reads its previous ones.
+constexpr int kColRBufs = 2 * kColRWarps, kColRBufShift = 3;                        // (kColRBufs = 2^kColRBufShift)
 constexpr int kColWarpA0 = 1, kColWarpB0 = kColWarpA0 + kColAWarps, kColWarpR0 = kColWarpB0 + kColBWarps;
 constexpr int kColWarpS2 = kColWarpR0 + kColRWarps;             // the second service warp (second visits)
 constexpr int kColThreads = 32 * (kColWarpS2 + 1);
@@ -125,7 +128,7 @@ struct ColStepParams {       // by step parity
 struct ColShared {
     unsigned long long full_a[kColMaxSlots], empty_a[kColMaxSlots];     // A ring: copies landed / the A warps are done
     unsigned long long full_b[kColMaxSlots], empty_b[kColMaxSlots];     // B ring: copies landed / the B warps are done
-    unsigned long long rfull[kColRWarps], rempty[kColRWarps];   // residual digits of a chunk (one buffer per R warp): written / consumed
+    unsigned long long rfull[kColRBufs], rempty[kColRBufs];     // residual digits of a chunk (buffer q mod kColRBufs): written / consumed
     int w_version;                             // steps (+1) whose digits of w are in place
     ColStepParams sp[2];
     double red_d[2][32];
@@ -286,7 +289,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
     unsigned char* tiles_b = tiles + (size_t)a.slots_a * slot_bytes;
     const int rstride = R + 32;                        // bytes between the residual digit vectors
     signed char* rdig = reinterpret_cast<signed char*>(tiles_b + (size_t)a.slots_b * slot_bytes);  // [R warps][2 operands][8 digits][rstride]
-    signed char* wdig = rdig + (size_t)kColRWarps * 2 * NRD * rstride;                             // [NG][4 k-blocks][8 columns: 4 digits, 4 x zero][32 B]
+    signed char* wdig = rdig + (size_t)kColRBufs * 2 * NRD * rstride;                             // [NG][4 k-blocks][8 columns: 4 digits, 4 x zero][32 B]
     // the A warps' hand-over of a task's digit sums from the lanes that hold them to a lane per row ([A warps][2 planes][32 rows][2])
     int* ascr = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(wdig + NG * 4 * 8 * 32) + 15) & ~(uintptr_t)15);
     ColShared* sh = reinterpret_cast<ColShared*>(ascr + (size_t)kColAWarps * 2 * 32 * 2);
@@ -308,7 +311,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             mbar_init(reinterpret_cast<uint64_t*>(sh->full_b + s), 1);
             mbar_init(reinterpret_cast<uint64_t*>(sh->empty_b + s), kColBWarps);
         }
-        for (int s = 0; s < kColRWarps; ++s) {
+        for (int s = 0; s < kColRBufs; ++s) {
             mbar_init(reinterpret_cast<uint64_t*>(sh->rfull + s), 1);
             mbar_init(reinterpret_cast<uint64_t*>(sh->rempty + s), kColBWarps);
         }
@@ -604,14 +607,14 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     for (int e = 0; e < 4; ++e) acc2[h][g][e] = 0;
 #pragma unroll 1
             for (int c = 0; c < st.nch; ++c, ++q) {
-                const int rbuf = q & (kColRWarps - 1);
+                const int rbuf = q & (kColRBufs - 1);
                 const long long w0c = (a.trace && p == 0) ? clock64() : 0;
                 long long w1c = w0c;
                 // both are usually there already: one look at each, side by side, before the waiting routine is called
-                const bool have_r = mbar_test_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1));
+                const bool have_r = mbar_test_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRBufShift) & 1));
                 const bool have_c = mbar_test_wait(sh->full_b + ring.slot, ring.phase);
                 if (!__all_sync(0xffffffffu, ok && have_r && have_c)) {
-                    ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRShift) & 1), sh, a.status, 73);
+                    ok = ok && col_wait(sh->rfull + rbuf, (uint32_t)((q >> kColRBufShift) & 1), sh, a.status, 73);
                     w1c = (a.trace && p == 0) ? clock64() : 0;
                     ok = ok && col_wait(sh->full_b + ring.slot, ring.phase, sh, a.status, 74);
                     ok = __all_sync(0xffffffffu, ok);                  // the warp acts as one
@@ -718,7 +721,6 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
         const int zper = (a.bpad + G - 1) / G;           // rows of a buffer of dot words that this CTA clears
         const int ngrp = a.ngrp;
         const int last_size = G - (ngrp - 1) * a.gsize;  // CTAs of the last group
-        signed char* rd = rdig + (size_t)rw * 2 * NRD * rstride;
 #pragma unroll 1
         for (int t_rel = 0; t_rel < steps; ++t_rel) {
             const ColStep st = col_step(a, a.first_step + t_rel);
@@ -749,7 +751,8 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
             bool behind = false;                         // (a step's first chunks are never complete yet)
 #pragma unroll 1
             for (int c = (rw - q0) & (kColRWarps - 1); c < st.nch; c += kColRWarps) {
-                const int q = q0 + c;
+                const int q = q0 + c, rbuf = q & (kColRBufs - 1);
+                signed char* rd = rdig + (size_t)rbuf * 2 * NRD * rstride;
                 // A lane takes the four rows whose digits make one 32-bit word of pass B's operand: rows 2t, 2t+1, 8+2t,
                 // 9+2t of half `hf` of the 32-row block `blk` (k index 4t + i <-> row 2t + (i & 1) + 8 (i >> 1)).
                 const int blk = lane >> 3, hf = (lane >> 2) & 1;
@@ -826,7 +829,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 }
                 behind = __all_sync(0xffffffffu, first_look);
                 const long long e0c = (a.trace && rw == 0) ? clock64() : 0;
-                if (ok && q >= kColRWarps) ok = col_wait(sh->rempty + rw, (uint32_t)(((q >> kColRShift) - 1) & 1), sh, a.status, 76);
+                if (ok && q >= kColRBufs) ok = col_wait(sh->rempty + rbuf, (uint32_t)(((q >> kColRBufShift) - 1) & 1), sh, a.status, 76);
                 ok = __all_sync(0xffffffffu, ok);
                 if (a.trace && rw == 0 && lane == 0) col_tally(a, t_rel, 3, clock64() - e0c);
                 if (kkA < R && ok) {
@@ -871,7 +874,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 }
                 if (c != c_last) {                       // (the step's last chunk is released below, after the step's sums)
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rw));
+                    if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rbuf));
                 }
                 // (off the chunk's path) every CTA has left step t - 1 behind, as chunk 0's complete dots showed: its buffer of dot words is cleared for step t + 2 (this CTA's share)
                 if (c == 0 && ok) {
@@ -907,7 +910,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                     col_unit_of(dbound, sh->sp[(t_rel + 1) & 1].U, sh->sp[(t_rel + 1) & 1].invU);
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + rw));
+                if (lane == 0) mbar_arrive(reinterpret_cast<uint64_t*>(sh->rfull + ((q0 + c_last) & (kColRBufs - 1))));
             }
             q0 += st.nch;
         }
@@ -989,7 +992,7 @@ int launch_sgd_column(zipml_ctx* ctx, const zipml_dataset* d, const float* b, fl
     while (ngrp > 1 && (int64_t)(ngrp - 1) * gsize >= G) --ngrp;       // no empty group
 
     const size_t slot_bytes = (size_t)2 * R * kColBlockBytes;
-    const size_t fixed = 1024 + (size_t)kColRWarps * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 8 * 32 + 16 +
+    const size_t fixed = 1024 + (size_t)kColRBufs * 2 * kColRDigits * (R + 32) + (size_t)ng * 4 * 8 * 32 + 16 +
                          (size_t)kColAWarps * 2 * 32 * 2 * sizeof(int) + sizeof(ColShared);
     if (fixed + 4 * slot_bytes > (size_t)ctx->smem_optin) return ZIPML_ERR_WORKSPACE;
     int slots = (int)(((size_t)ctx->smem_optin - fixed) / slot_bytes);
