@@ -22,7 +22,7 @@
 //                        s8 digits of w), converted to a fixed-point unit common to all CTAs and added to
 //                        the row's word with one 64-bit integer atomic, whose low byte counts the CTAs
 //   R warps   (4)        poll a chunk's words until their counts are complete, read the labels, turn the
-//                        residuals into eight balanced base-128 int8 digits; each warp takes every fourth
+//                        residuals into eight balanced base-256 int8 digits; each warp takes every fourth
 //                        chunk, so four exchanges are in flight at a time
 //   B warps   (8)        gradient of the CTA's own features (transposing ldmatrix, residual digits as the
 //                        other operand), accumulated in registers over the step; at the step's end: update
@@ -44,7 +44,8 @@
 // sums to the atomic is integer arithmetic only.  Residuals: eight digits (55 bits) whose unit is a power of two
 // as well, at most twice what D(t) + max |b| of the step needs, so that a dot becomes a residual by a shift and
 // the label's fixed-point value (one conversion per row); all eight columns of the tensor-core tile carry a digit.  Digits are balanced
-// (-64..63) and found without a carry chain: with 64 added to every digit the number is plain base 128.
+// and found without a carry chain: with half the base added to every digit the number is plain base 128 (w,
+// -64..63) or plain base 256 (residuals, -128..127: the digits are the number's own bytes, xor 0x80).
 // Results do not depend on timing: every sum is an integer sum or has a fixed order.
 //
 // The machine code is kept small on purpose (four roles share the instruction cache): 32-bit counters kept up
@@ -87,8 +88,10 @@ constexpr int kColMaxSlots = 16;            // per ring
 constexpr int kColMaxChunkRows = 128;       // a lane of an R warp takes four rows of a chunk
 constexpr int kColMaxGroups = 4;            // words per row and plane
 constexpr int kColRDigits = 8;              // digits of a residual
-constexpr long long kColQmaxR = 35000000000000000LL;     // below 63 * (128^8 - 1) / 127
-constexpr long long kColBiasR = 64ll * 567382630219905ll;    // 64 * (128^8 - 1) / 127: digit s of W + bias is balanced digit s of W, plus 64
+constexpr long long kColQmaxR = 35000000000000000LL;     // below 2^55: eight balanced base-256 digits hold it with room
+// Residual digits are balanced base-256 digits (-128..127), found without a carry chain: with 128 added to every digit
+// the number is plain base 256, i.e. the bytes of R + bias; a byte xor 0x80 is the digit as a signed byte.
+constexpr unsigned long long kColBiasR = 0x8080808080808080ull;
 constexpr int kColBiasW = 64 * 2113665;                      // 64 * (128^4 - 1) / 127
 constexpr long long kColWaitCycles = 6000000000LL;       // a wait gives up after about three seconds
 constexpr int kColNamedR = 1, kColNamedB = 2;            // named barriers of the R and B warps
@@ -682,7 +685,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 for (int e = 0; e < 4; ++e) acc[g][e] = acc2[0][g][e] + acc2[1][g][e];
             const ColStepParams& sp = sh->sp[t_rel & 1];
             const double delta_r = sp.delta_r, lo_term = sp.delta_r * sp.rsum, scale = 1.0 / (2.0 * (double)st.bt);
-            const double w0 = (tl == 0) ? 1.0 : (tl == 1) ? 16384.0 : (tl == 2) ? 268435456.0 : 4398046511104.0;     // 128^(2t)
+            const double w0 = (tl == 0) ? 1.0 : (tl == 1) ? 65536.0 : (tl == 2) ? 4294967296.0 : 281474976710656.0;  // 256^(2t)
             double Sf[NF];
 #pragma unroll
             for (int e = 0; e < NF; ++e) Sf[e] = 0.0;
@@ -692,7 +695,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 const int lo_d = acc[gi][2 * h] - (gi + 1 < NG ? acc[gi + 1 < NG ? gi + 1 : gi][2 * h] : 0);
                 const int hi_d = acc[gi][2 * h + 1] - (gi + 1 < NG ? acc[gi + 1 < NG ? gi + 1 : gi][2 * h + 1] : 0);
                 // (exact: the differences are 2^(gi CB) times the group's digit sums)
-                double v = ((double)(lo_d >> (gi * CB)) + 128.0 * (double)(hi_d >> (gi * CB))) * w0;
+                double v = ((double)(lo_d >> (gi * CB)) + 256.0 * (double)(hi_d >> (gi * CB))) * w0;
                 v += __shfl_xor_sync(0xffffffffu, v, 1);
                 v += __shfl_xor_sync(0xffffffffu, v, 2);
                 if ((fi & 3) == tl) Sf[fi >> 2] = v;
@@ -834,7 +837,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                 if (a.trace && rw == 0 && lane == 0) col_tally(a, t_rel, 3, clock64() - e0c);
                 if (kkA < R && ok) {
                     // residuals r = U * dot - label in fixed point, then their digits: with 64 added to every digit the
-                    // number is plain base 128 (no carry chain); four rows' digits make a word
+                    // number is plain base 256 (no carry chain); four rows' digits make a word
                     unsigned long long u1[4], u2[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -847,11 +850,10 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
                             rs_hi += (R1 >> 28) + (R2 >> 28);
                             rs_lo += (R1 & 0xFFFFFFFll) + (R2 & 0xFFFFFFFll);
                         }
-                        u1[i] = (unsigned long long)(R1 + kColBiasR);
-                        u2[i] = (unsigned long long)(R2 + kColBiasR);
+                        u1[i] = ((unsigned long long)R1 + kColBiasR) ^ kColBiasR;      // eight digits as signed bytes
+                        u2[i] = ((unsigned long long)R2 + kColBiasR) ^ kColBiasR;
                     }
-                    // a 28-bit half becomes four 7-bit digits, a byte each, minus 64 as signed bytes; the four rows' words are
-                    // then transposed into one word per digit
+                    // the four rows' words (four digits each) are transposed into one word per digit
                     signed char* dst = rd + blk * 32 + tl * 8 + hf * 4;
 #pragma unroll
                     for (int h = 0; h < 4; ++h) {                        // digits 0..3, 4..7 of r2 (meets plane 1), then of r1
@@ -859,10 +861,7 @@ __global__ void __launch_bounds__(kColThreads, 1) sgd_column_kernel(const Column
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const unsigned long long u = h < 2 ? u2[i] : u1[i];
-                            const uint32_t x = (h & 1) ? (uint32_t)(u >> 28) : ((uint32_t)u & 0xFFFFFFFu);
-                            uint32_t v = (x & 0x7Fu) | ((x & 0x3F80u) << 1) | ((x & 0x1FC000u) << 2) | ((x & 0xFE00000u) << 3);
-                            v ^= 0x40404040u; v |= (v & 0x40404040u) << 1;
-                            e[i] = v;
+                            e[i] = (h & 1) ? (uint32_t)(u >> 32) : (uint32_t)u;
                         }
                         const uint32_t t0 = __byte_perm(e[0], e[1], 0x5140), t1 = __byte_perm(e[2], e[3], 0x5140);
                         const uint32_t t2 = __byte_perm(e[0], e[1], 0x7362), t3 = __byte_perm(e[2], e[3], 0x7362);
