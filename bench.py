@@ -37,7 +37,7 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_TRAFFIC = {
     ("c2", 5): (203.04e6 + 3.76e6, "profiles/sgd_cluster_kernel_c2_full.md"),
     ("c5", 6): (4 * (591.80e6 + 6.29e6), "profiles/sgd_stream_kernel_c5_full.md, 16,384-row capture scaled x4 by the rows"),
-    ("c5", 7): (4 * (538.85e6 + 6.89e6), "profiles/sgd_column_kernel_c5_full.md, 16,384-row capture scaled x4 by the rows"),
+    ("c5", 7): (4 * (538.45e6 + 4.86e6), "profiles/sgd_column_kernel_c5_full.md, 16,384-row capture scaled x4 by the rows"),
 }
 ENGINE_KERNELS = {1: "sgd_kernel (stepwise launches)", 2: "sgd_kernel (persistent)", 3: "sgd_ring_kernel", 4: "sgd_lean_kernel",
                   5: "sgd_cluster_kernel", 6: "sgd_stream_kernel", 7: "sgd_column_kernel"}

@@ -50,13 +50,13 @@
 //
 // The machine code is kept small on purpose (four roles share the instruction cache): 32-bit counters kept up
 // step by step instead of 64-bit divisions, waits as functions with one copy, loops unrolled only where
-// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 24.7 us per step (stream engine:
+// registers demand it.  Measured on 65,536 x 32,768 4-bit rows, B = 2,048: 23.0 us per step (stream engine:
 // 29.8), DRAM reads 1.00 x the packed bytes.  Not HBM bounds it but the chain of a step: the first chunk's dots
-// have to cross L2 and become digits before pass B can start (about 9 k cycles), pass B then follows the R
-// warps (about 2 k cycles per chunk for the four of them together) rather than the copies, and the next
-// step's first dots come 6 k cycles after the last chunk's gradient.  With pass B's arithmetic taken out the
-// step is 13 % shorter, with pass A's arithmetic taken out not at all; more warps for any one role slow the
-// others by as much (the SM issues about two instructions per cycle in every variant tried).
+// have to cross L2 and become digits before pass B can start, pass B (about 1.2 k cycles per chunk on its own, 2 k
+// while pass A runs beside it) ends about 9 k cycles after pass A, and the next step's first dots come 5 k cycles
+// after the last chunk's gradient.  The SM issues about two instructions per cycle in every variant tried, so a
+// role given more warps slows the others by as much; what helped was taking instructions and tests out of the
+// loops and keeping the R warps from waiting for pass B (two digit buffers each).
 //
 // Memory order.  A buffer of dot words serves every third step and is cleared in between by the R warp that
 // has seen the first chunk of step t complete (then every CTA has left step t-1, the buffer's last use,
